@@ -1,0 +1,254 @@
+"""Pin checks for the float64 oracle, each written against something other than
+the oracle itself: a separately written AdamW, closed forms, invariants of the
+update rule, exact rational arithmetic on tiny cases.
+
+Every check takes the loaded oracle library, so the same checks can be pointed
+at deliberately broken copies of the oracle (see test_oracle_mutants.py).
+"""
+from __future__ import annotations
+
+import itertools
+import math
+from fractions import Fraction
+
+import numpy as np
+
+from oracle import adamw_ref, exact, partition_ref, step as ostep
+
+HP = dict(lr=1e-3, beta1=0.9, beta2=0.95, eps=1e-8, weight_decay=0.1)
+
+
+def run(lib, p0, g_steps, L, hp=HP, apply_wd=True):
+    """Run the oracle over len(g_steps) steps; returns float64 p, m, v."""
+    p = np.array(p0, dtype=np.float64)
+    m = np.zeros_like(p)
+    v = np.zeros(p.size // L, dtype=np.float64)
+    for t, g in enumerate(g_steps, start=1):
+        ostep.adammini_step(p, m, v, np.asarray(g, dtype=np.float64), L, step=t,
+                            apply_wd=apply_wd, lib=lib, **hp)
+    return p, m, v
+
+
+def _rel(a, b, floor=1e-300):
+    a, b = np.asarray(a, float), np.asarray(b, float)
+    return float(np.max(np.abs(a - b) / np.maximum(np.abs(b), floor))) if a.size else 0.0
+
+
+# -- P1: block length 1 is AdamW, bit for bit (paper: Adam-mini "replaces g*g by
+#    its mean"; the mean of one element is that element) -----------------------
+def check_reduces_to_adamw(lib):
+    rng = np.random.default_rng(11)
+    n = 257
+    p0 = rng.normal(0, 0.02, n)
+    gs = [rng.normal(0, 1, n) * 10.0 ** rng.uniform(-4, 0, n) for _ in range(7)]
+    gs[3][::5] = 0.0
+    p, m, v = run(lib, p0, gs, 1)
+    pa, ma, va = p0.copy(), np.zeros(n), np.zeros(n)
+    for t, g in enumerate(gs, start=1):
+        adamw_ref.adamw_step(pa, ma, va, g, step=t, **HP)
+    assert np.array_equal(p.view(np.int64), pa.view(np.int64))
+    assert np.array_equal(m.view(np.int64), ma.view(np.int64))
+    assert np.array_equal(v.view(np.int64), va.view(np.int64))
+
+
+# -- I1 / five-parameter example: v_b is the block mean of AdamW's v, m is
+#    AdamW's m, and the step uses eta / sqrt(mean of Adam's v over the block) ---
+def check_block_mean_of_adam_v(lib, blocks=((0, 1, 2), (3, 4))):
+    rng = np.random.default_rng(5)
+    n = sum(len(b) for b in blocks)
+    p0 = rng.normal(0, 0.02, n)
+    T = 6
+    gs = [rng.normal(0, 1, n) * np.array([1e-3, 1.0, 30.0, 0.2, 5e-2][:n]) for _ in range(T)]
+    # Adam-mini: every block is its own tensor (blocks here differ in length)
+    state = []
+    for idx in blocks:
+        idx = list(idx)
+        state.append([p0[idx].copy(), np.zeros(len(idx)), np.zeros(1)])
+    pa, ma, va = p0.copy(), np.zeros(n), np.zeros(n)
+    for t, g in enumerate(gs, start=1):
+        p_before = [s[0].copy() for s in state]
+        adamw_ref.adamw_step(pa, ma, va, g, step=t, **HP)
+        for s, idx in zip(state, blocks):
+            idx = list(idx)
+            ostep.adammini_step(s[0], s[1], s[2], g[idx], len(idx), step=t, lib=lib, **HP)
+        for s, idx, pb in zip(state, blocks, p_before):
+            idx = list(idx)
+            assert np.array_equal(s[1], ma[idx])                       # m is Adam's m
+            assert _rel(s[2][0], va[idx].mean()) < 1e-13               # v_b = mean of Adam's v
+            bc1 = 1 - HP["beta1"] ** t
+            bc2 = 1 - HP["beta2"] ** t
+            u_mini = HP["lr"] / (math.sqrt(va[idx].mean() / bc2) + HP["eps"])
+            want = pb * (1 - HP["lr"] * HP["weight_decay"]) - u_mini * ma[idx] / bc1
+            assert _rel(s[0], want) < 1e-12
+
+
+# -- P2: constant gradient.  m_hat = g and v_hat = mean(g_b^2) at every step, so
+#    with a = 1 - eta*lambda and c_i = g_i / (rms(g_b) + eps):
+#    p_T = a^T p_0 - eta c_i (1 - a^T) / (1 - a) --------------------------------
+def check_constant_gradient_closed_form(lib):
+    rng = np.random.default_rng(3)
+    L, nb, T = 6, 4, 25
+    p0 = rng.normal(0, 0.02, L * nb)
+    g = rng.normal(0, 1, L * nb) * np.repeat(10.0 ** rng.uniform(-3, 1, nb), L)
+    p, m, v = run(lib, p0, [g] * T, L)
+    ms = (g.reshape(nb, L) ** 2).mean(axis=1)
+    a = 1 - HP["lr"] * HP["weight_decay"]
+    c = g / (np.repeat(np.sqrt(ms), L) + HP["eps"])
+    want = a ** T * p0 - HP["lr"] * c * (1 - a ** T) / (1 - a)
+    assert _rel(p, want) < 1e-11
+    assert _rel(m, g * (1 - HP["beta1"] ** T)) < 1e-12
+    assert _rel(v, ms * (1 - HP["beta2"] ** T)) < 1e-12
+    # lambda = 0: p_T = p_0 - T eta c_i
+    hp0 = dict(HP, weight_decay=0.0)
+    p, _, _ = run(lib, p0, [g] * T, L, hp=hp0)
+    assert _rel(p, p0 - T * HP["lr"] * c) < 1e-11
+    # decay switched off per tensor behaves like lambda = 0
+    p2, _, _ = run(lib, p0, [g] * T, L, apply_wd=False)
+    assert np.array_equal(p, p2)
+
+
+# -- P2': zero gradient.  m = v = 0 and the Adam term is 0/(0+eps) = 0 ----------
+def check_zero_gradient(lib):
+    p0 = np.linspace(-1, 1, 12)
+    T = 9
+    p, m, v = run(lib, p0, [np.zeros(12)] * T, 4)
+    assert not m.any() and not v.any()
+    assert _rel(p, (1 - HP["lr"] * HP["weight_decay"]) ** T * p0) < 1e-14
+
+
+# -- I2, I3: the first step, p_1 = a p_0 - eta g / (rms(g_b) + eps); if |g| = c on
+#    the block the Adam term is eta sign(g) c / (c + eps) ------------------------
+def check_first_step(lib):
+    rng = np.random.default_rng(8)
+    L, nb = 8, 3
+    p0 = rng.normal(0, 0.02, L * nb)
+    g = rng.normal(0, 2, L * nb)
+    p, m, v = run(lib, p0, [g], L)
+    rms = np.repeat(np.sqrt((g.reshape(nb, L) ** 2).mean(axis=1)), L)
+    a = 1 - HP["lr"] * HP["weight_decay"]
+    assert _rel(p, a * p0 - HP["lr"] * g / (rms + HP["eps"])) < 1e-12
+    c = 0.37
+    s = np.sign(rng.normal(size=L * nb))
+    p, _, _ = run(lib, p0, [c * s], L)
+    assert _rel(p, a * p0 - HP["lr"] * s * c / (c + HP["eps"])) < 1e-12
+    # eps sits outside the root: with a large eps the step is eta g / (rms + eps)
+    hp = dict(HP, eps=0.5)
+    p, _, _ = run(lib, p0, [g], L, hp=hp)
+    assert _rel(p, a * p0 - HP["lr"] * g / (rms + 0.5)) < 1e-12
+
+
+# -- I4: scaling a block's gradients by k > 0 leaves p unchanged as eps -> 0 -----
+def check_scale_invariance(lib):
+    rng = np.random.default_rng(21)
+    L, nb, T = 5, 3, 6
+    hp = dict(HP, eps=1e-300)
+    p0 = rng.normal(0, 0.02, L * nb)
+    gs = [rng.normal(0, 1, L * nb) for _ in range(T)]
+    k = np.repeat([1.0, 1024.0, 2.0 ** -20], L)          # powers of two: exact scaling
+    p_a, _, _ = run(lib, p0, gs, L, hp=hp)
+    p_b, _, _ = run(lib, p0, [g * k for g in gs], L, hp=hp)
+    assert _rel(p_b, p_a) < 1e-13
+
+
+# -- I5: permuting elements inside blocks permutes m and p and leaves v ---------
+def check_permutation_invariance(lib):
+    rng = np.random.default_rng(22)
+    L, nb, T = 7, 4, 5
+    p0 = rng.normal(0, 0.02, L * nb)
+    gs = [rng.normal(0, 1, L * nb) for _ in range(T)]
+    perm = np.concatenate([b * L + rng.permutation(L) for b in range(nb)])
+    p_a, m_a, v_a = run(lib, p0, gs, L)
+    p_b, m_b, v_b = run(lib, p0[perm], [g[perm] for g in gs], L)
+    assert _rel(v_b, v_a) < 1e-14
+    assert _rel(p_b, p_a[perm]) < 1e-12
+    assert np.array_equal(m_b, m_a[perm])
+
+
+# -- I6: blocks evolve independently ---------------------------------------------
+def check_block_independence(lib):
+    rng = np.random.default_rng(23)
+    L, nb, T = 4, 5, 4
+    p0 = rng.normal(0, 0.02, L * nb)
+    gs = [rng.normal(0, 1, L * nb) for _ in range(T)]
+    gs2 = [g.copy() for g in gs]
+    for g in gs2:
+        g[2 * L:3 * L] *= -3.0                              # disturb block 2 only
+    a = run(lib, p0, gs, L)
+    b = run(lib, p0, gs2, L)
+    keep = np.ones(L * nb, bool)
+    keep[2 * L:3 * L] = False
+    assert np.array_equal(a[0][keep], b[0][keep]) and np.array_equal(a[1][keep], b[1][keep])
+    assert np.array_equal(np.delete(a[2], 2), np.delete(b[2], 2))
+    assert not np.array_equal(a[0][~keep], b[0][~keep])
+    # a tensor run alone equals the same blocks run inside a longer tensor
+    c = run(lib, p0[L:3 * L], [g[L:3 * L] for g in gs], L)
+    assert np.array_equal(c[0], a[0][L:3 * L]) and np.array_equal(c[2], a[2][1:3])
+
+
+# -- P4: brute force against exact rational arithmetic ---------------------------
+GRAD_VALUES = (-2.0, -0.5, 0.0, 0.25, 1.5)
+
+
+def _compare_exact(lib, p0, g_steps, L):
+    n = len(p0)
+    p, m, v = run(lib, p0, g_steps, L)
+    descs = [partition_ref.TensorDesc(1, n, partition_ref.FIXED, fixed_block_len=L)]
+    blocks = partition_ref.blocks_as_index_lists(descs)
+    pe, me, ve = exact.adammini_exact(p0, g_steps, blocks, **HP)
+    for got, want in ((p, pe), (m, me), (v, ve)):
+        for x, y in zip(got, want):
+            y = float(y)
+            assert abs(x - y) <= 4e-15 * max(abs(y), 1e-3 if got is p else 0.0) + 1e-300, (x, y, L, g_steps)
+
+
+def check_brute_force_exact(lib):
+    # every gradient pattern on up to 4 elements, every divisor as block length
+    for n in (1, 2, 3, 4):
+        p0 = [0.02 * ((-1) ** i) * (i + 1) for i in range(n)]
+        for L in [d for d in range(1, n + 1) if n % d == 0]:
+            for g in itertools.product(GRAD_VALUES, repeat=n):
+                _compare_exact(lib, p0, [list(g)], L)
+    # three steps on up to 12 elements, every divisor, sampled patterns
+    rng = np.random.default_rng(99)
+    for n in (6, 8, 12):
+        p0 = list(rng.normal(0, 0.02, n))
+        for L in [d for d in range(1, n + 1) if n % d == 0]:
+            for _ in range(6):
+                gs = [list(rng.choice(GRAD_VALUES, n)) for _ in range(3)]
+                _compare_exact(lib, p0, gs, L)
+
+
+# -- widening: bfloat16 / float32 bits reach the oracle exactly ------------------
+def check_widening(lib):
+    import ctypes
+    bits = np.arange(65536, dtype=np.uint16)
+    out = np.empty(65536, dtype=np.float64)
+    lib.oracle_widen_bf16(bits.ctypes.data, out.ctypes.data, 65536)
+    with np.errstate(invalid="ignore"):
+        want = (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    ok = ~np.isnan(want)
+    assert np.array_equal(out[ok], want[ok]) and np.isnan(out[~ok]).all()
+    # the step reads bf16 gradients as those values: 1.0 is 0x3F80, -2.5 is 0xC020
+    p = np.zeros(2); m = np.zeros(2); v = np.zeros(1)
+    g = np.array([0x3F80, 0xC020], dtype=np.uint16)
+    ostep.adammini_step(p, m, v, g, 2, step=1, lib=lib, **HP)
+    assert _rel(m, [0.1, -0.25]) < 1e-15 and _rel(v, [0.05 * (1 + 6.25) / 2]) < 1e-15
+    g32 = np.array([1.0, -2.5], dtype=np.float32)
+    p2 = np.zeros(2); m2 = np.zeros(2); v2 = np.zeros(1)
+    ostep.adammini_step(p2, m2, v2, g32, 2, step=1, lib=lib, **HP)
+    assert np.array_equal(p, p2) and np.array_equal(m, m2) and np.array_equal(v, v2)
+    del ctypes
+
+
+ALL_CHECKS = (
+    check_reduces_to_adamw,
+    check_block_mean_of_adam_v,
+    check_constant_gradient_closed_form,
+    check_zero_gradient,
+    check_first_step,
+    check_scale_invariance,
+    check_permutation_invariance,
+    check_block_independence,
+    check_brute_force_exact,
+    check_widening,
+)
