@@ -1,0 +1,186 @@
+/*
+ * adammini.h -- C ABI of the B200 Adam-mini optimizer-step library.
+ *
+ * The library performs, on one GPU, the per-step update of Adam-mini
+ * (Algorithm 1 of the paper, "Adam-mini (General form)"; the boxed v_b rule of
+ * the introduction) over all parameter tensors of a model:
+ *
+ *   for every block b (L contiguous elements of one tensor), at step t >= 1:
+ *     v_b   <- (1-beta2) * mean(g_b * g_b) + beta2 * v_b          one scalar per block
+ *     p_i   <- p_i - eta_t * lambda * p_i                          decoupled decay
+ *     m_i   <- (1-beta1) * g_i + beta1 * m_i
+ *     p_i   <- p_i - eta_t * (m_i / (1-beta1^t)) / (sqrt(v_b / (1-beta2^t)) + eps)
+ *
+ * Blocks follow the paper's partition rules (Algorithm 2, "Partition for
+ * non-Transformers"; Algorithm 3, "Partition for Transformers"): token rows for
+ * embedding/output, heads for query/key, output neurons for value /
+ * attention projection / MLP, the whole tensor otherwise.
+ *
+ * Conventions
+ *   - Weights are [out_features, in_features], row-major, contiguous.  Layouts
+ *     that are transposed or flattened differently (the paper's appendix notes
+ *     that they need re-ordering) are the caller's to re-order: the library
+ *     sees only rows x cols.
+ *   - Parameters (master copy), m and v are float32; gradients are float32 or
+ *     bfloat16 per tensor.  m and v must be zero before step 1.
+ *   - Every function returns an am_status (0 = success, negative = error) and
+ *     never throws or aborts.  Pointers marked "device" are device addresses
+ *     on the GPU that was current when adammini_create ran; "host" pointers
+ *     are ordinary host addresses.
+ *   - The caller owns params, grads, m, v.  The library owns its handle, the
+ *     device copy of the block table and a small scratch area.
+ */
+#ifndef ADAMMINI_H_
+#define ADAMMINI_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* How a tensor is cut into blocks (Algorithm 3 branches). */
+typedef enum {
+    AM_WHOLE  = 0,  /* one block: the ELSE branch of Algorithm 3, and Algorithm 2 */
+    AM_ROWS   = 1,  /* value, attn.proj, mlp: one block per output neuron (row)    */
+    AM_HEADS  = 2,  /* query, key: one block per head = rows/n_heads rows          */
+    AM_TOKENS = 3,  /* embed, output: one block per token row                      */
+    AM_FIXED  = 4   /* explicit block length (any divisor of numel)                */
+} am_kind;
+
+typedef enum { AM_F32 = 0, AM_BF16 = 1 } am_dtype;
+
+typedef enum {
+    AM_OK                   =  0,
+    AM_ERR_INVALID_ARGUMENT = -1,  /* null pointer, step < 1, eps <= 0, beta outside [0,1), ... */
+    AM_ERR_SHAPE            = -2,  /* rows/cols <= 0, rows % n_heads != 0, numel % block_len != 0 */
+    AM_ERR_MISALIGNED       = -3,  /* a device pointer is not 16-byte aligned */
+    AM_ERR_CUDA             = -4,  /* a CUDA call failed; see adammini_last_cuda_error */
+    AM_ERR_TIMEOUT          = -5,  /* a bounded device-side wait gave up (reported by adammini_sync_status) */
+    AM_ERR_ALLOC            = -6,  /* host or device allocation failed */
+    AM_ERR_TOO_LARGE        = -7   /* a size exceeds what the entry point supports */
+} am_status;
+
+/* One parameter tensor as the caller describes it.  1-D tensors: rows = 1. */
+typedef struct am_tensor_desc {
+    int64_t rows, cols;
+    int32_t kind;               /* am_kind */
+    int32_t n_heads;            /* AM_HEADS only; rows % n_heads == 0 */
+    int64_t fixed_block_len;    /* AM_FIXED only; (rows*cols) % fixed_block_len == 0 */
+    int32_t grad_dtype;         /* am_dtype of this tensor's gradient */
+    int32_t apply_weight_decay; /* 0: skip the decay line for this tensor */
+} am_tensor_desc;
+
+/* One row of the flat block table (one per tensor, caller's order).  Block b of
+ * the tensor is elements [b*block_len, (b+1)*block_len); its second moment is
+ * v[v_offset + b]. */
+typedef struct am_table_row {
+    int64_t numel, block_len, n_blocks, v_offset;
+    int32_t kind, grad_dtype, wd, pad;
+} am_table_row;
+
+/* eta, beta1, beta2, eps, lambda of Algorithm 1.  Doubles, so the caller's
+ * values reach the library unrounded; the kernels compute in float32. */
+typedef struct am_hparams {
+    double lr, beta1, beta2, eps, weight_decay;
+} am_hparams;
+
+typedef struct am_partition am_partition;
+typedef struct am_handle am_handle;
+
+/* ---- partitioner (host only; Algorithm 2 / Algorithm 3) ------------------------
+ * Builds the flat block table from `n_tensors` descriptors (host array, read
+ * during the call only).  On success *out owns the table; free it with
+ * adammini_partition_free.  AM_ERR_SHAPE if a descriptor does not divide. */
+int adammini_partition_build(const am_tensor_desc *descs, int32_t n_tensors, am_partition **out);
+
+/* Number of tensors in the table. */
+int32_t adammini_partition_num_tensors(const am_partition *part);
+
+/* Copies the table into `rows` (host array of n_tensors entries, may be NULL)
+ * and the total number of blocks (= length of v) into *total_blocks (may be NULL). */
+int adammini_partition_export(const am_partition *part, am_table_row *rows, int64_t *total_blocks);
+
+void adammini_partition_free(am_partition *part);
+
+/* Algorithm 3's name tests in its order of precedence: "embed"/"output" ->
+ * AM_TOKENS, "query"/"key" -> AM_HEADS, "value"/"attn.proj"/"mlp" -> AM_ROWS,
+ * anything else AM_WHOLE.  `name` is a host C string.  Returns the am_kind. */
+int32_t adammini_kind_from_name(const char *name);
+
+/* ---- optimizer handle ----------------------------------------------------------
+ * Creates a handle on the current CUDA device: copies the table (the partition
+ * may be freed afterwards), plans the kernel launches, uploads the device
+ * tables and allocates scratch.  Hyper-parameters are validated:
+ * lr >= 0, 0 <= beta < 1, eps > 0, weight_decay >= 0. */
+int adammini_create(const am_partition *part, const am_hparams *hp, am_handle **out);
+
+/* eta_t of Algorithm 1 is time-varying: set it before the step it applies to. */
+int adammini_set_lr(am_handle *h, double lr);
+int adammini_set_hparams(am_handle *h, const am_hparams *hp);
+
+/* One Adam-mini step (Algorithm 1) over every tensor of the table.
+ *   params, grads, m : host arrays of n_tensors DEVICE pointers, in table order;
+ *                      tensor i holds rows*cols contiguous elements
+ *                      (params/m float32, grads of the tensor's grad_dtype).
+ *                      All must be 16-byte aligned.  grads are only read.
+ *   v                : DEVICE pointer, float32[total_blocks], 16-byte aligned.
+ *   step             : t, 1-based.
+ *   cuda_stream      : a cudaStream_t (NULL = the legacy default stream).
+ * Asynchronous: work is enqueued on the stream and the call returns without
+ * synchronising.  params, m and v are updated in place.  Calls on one handle
+ * must be issued from one thread at a time and ordered on one stream (or
+ * otherwise serialised), because they share the handle's scratch. */
+int adammini_step(am_handle *h, void *const *params, const void *const *grads, void *const *m,
+                  float *v, int64_t step, void *cuda_stream);
+
+/* The same step for callers whose state lives in HOST memory (offloaded
+ * optimizer state): params, grads, m are host arrays of HOST pointers, v is a
+ * HOST pointer.  The library streams groups of tensors through device staging
+ * buffers (host->device copies, the kernels above, device->host copies) on
+ * internal streams and returns after everything has landed back in host
+ * memory.  Pinned host memory gives full copy bandwidth; pageable works.
+ * `staging_bytes` bounds the device memory used for staging (0 = default). */
+int adammini_step_host(am_handle *h, void *const *params, const void *const *grads, void *const *m,
+                       float *v, int64_t step, int64_t staging_bytes);
+
+/* Waits for the stream and returns AM_OK, or AM_ERR_TIMEOUT if a device-side
+ * bounded wait gave up during any step since the last call, or AM_ERR_CUDA. */
+int adammini_sync_status(am_handle *h, void *cuda_stream);
+
+/* Options and queries (keys below).  Unknown keys: AM_ERR_INVALID_ARGUMENT. */
+typedef enum {
+    AM_OPT_PATH          = 0, /* 0 = automatic; 1 = force the three-launch two-pass path for every
+                                 tensor with block_len > 16 (correctness anchor) */
+    AM_OPT_STREAM_CTAS   = 1, /* persistent CTAs of the streaming kernel (0 = one per SM) */
+    AM_OPT_CLUSTER_SIZE  = 2, /* CTAs per cluster for head-sized blocks (0 = default) */
+    AM_OPT_STREAM_THREADS = 3 /* consumer threads per CTA of the streaming kernels (0 = default) */
+} am_option;
+int adammini_set_option(am_handle *h, int32_t key, int64_t value);
+
+typedef enum {
+    AM_Q_LAUNCHES_PER_STEP = 0, /* kernels one adammini_step enqueues */
+    AM_Q_SCRATCH_BYTES     = 1, /* device scratch owned by the handle */
+    AM_Q_TOTAL_BLOCKS      = 2,
+    AM_Q_TOTAL_ELEMENTS    = 3,
+    AM_Q_ELEMENTS_SMALL    = 4, /* elements routed to the thread-per-block kernel (block_len <= 16) */
+    AM_Q_ELEMENTS_STREAM   = 5, /* ... to the single-launch streaming kernel */
+    AM_Q_ELEMENTS_CLUSTER  = 6, /* ... to the cluster kernel (head-sized blocks) */
+    AM_Q_ELEMENTS_TWOPASS  = 7, /* ... to the two-pass path (blocks beyond on-chip/L2 reach, or unaligned) */
+    AM_Q_ALGORITHMIC_BYTES = 8  /* bytes one step must move: per tensor g once (twice on the two-pass
+                                   path), m and p read+written, v read+written */
+} am_query;
+int adammini_query(const am_handle *h, int32_t what, int64_t *value);
+
+/* The CUDA error code (cudaError_t as int) of the last AM_ERR_CUDA on this handle. */
+int adammini_last_cuda_error(const am_handle *h);
+
+int adammini_destroy(am_handle *h);
+
+/* Static string for a status code. */
+const char *adammini_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ADAMMINI_H_ */
