@@ -1,0 +1,312 @@
+// Device helpers, the thread-per-block kernel for tiny blocks and the two-pass
+// kernels (partial sums -> finalize -> update) that handle any block length and
+// any alignment.  Update rule: Algorithm 1 of the paper.
+#ifndef ADAMMINI_KERNELS_BASIC_CUH_
+#define ADAMMINI_KERNELS_BASIC_CUH_
+
+#include <cuda_runtime.h>
+
+#include "adammini_internal.h"
+
+namespace am {
+
+constexpr int kThreads = 256;            // CTA size of the kernels in this file
+constexpr int kSmallMaxL = 16;           // thread-per-block kernel handles L <= 16
+constexpr int kSmallUnitBlocks = 1024;   // blocks per CTA unit (general L)
+constexpr int kSmallUnitVec = 4096;      // elements per CTA unit (L == 1, float4 path)
+constexpr int64_t kPieceMax = 32768;     // elements per partial sum, two-pass path
+constexpr int64_t kMaxPiecesPerBlock = 16384;
+
+// ---------------------------------------------------------------------------
+// small helpers
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+// Four consecutive gradients, widened exactly to float.
+template <int GD>
+__device__ __forceinline__ float4 load_g4(const void *g, int64_t i) {
+    if (GD == AM_BF16) {
+        const uint2 u = *reinterpret_cast<const uint2 *>(static_cast<const uint16_t *>(g) + i);
+        return make_float4(bf16_lo(u.x), bf16_hi(u.x), bf16_lo(u.y), bf16_hi(u.y));
+    } else {
+        return *reinterpret_cast<const float4 *>(static_cast<const float *>(g) + i);
+    }
+}
+
+template <int GD>
+__device__ __forceinline__ float load_g1(const void *g, int64_t i) {
+    if (GD == AM_BF16)
+        return __uint_as_float(static_cast<uint32_t>(static_cast<const uint16_t *>(g)[i]) << 16);
+    return static_cast<const float *>(g)[i];
+}
+
+// Elementwise part of Algorithm 1: first moment, decoupled decay on the old
+// parameter, then the Adam term with the block's step size
+//   step = eta_t / ((1-beta1^t) (sqrt(v_hat) + eps)).
+// lr_wd is eta_t*lambda, or 0 for tensors exempt from decay (then p stays p exactly).
+__device__ __forceinline__ void update_one(float g, float &m, float &p, float beta1, float omb1,
+                                           float lr_wd, float step) {
+    m = fmaf(omb1, g, beta1 * m);
+    const float decayed = fmaf(-lr_wd, p, p);
+    p = fmaf(-step, m, decayed);
+}
+
+__device__ __forceinline__ void update_four(const float4 &g, float4 &m, float4 &p, float beta1, float omb1,
+                                            float lr_wd, float step) {
+    update_one(g.x, m.x, p.x, beta1, omb1, lr_wd, step);
+    update_one(g.y, m.y, p.y, beta1, omb1, lr_wd, step);
+    update_one(g.z, m.z, p.z, beta1, omb1, lr_wd, step);
+    update_one(g.w, m.w, p.w, beta1, omb1, lr_wd, step);
+}
+
+// Per-block scalars in double: new v_b and the step size (see update_one).
+__device__ __forceinline__ float block_step(double sum_sq, double L, float v_old,
+                                            const StepScalars &s, float *v_new) {
+    const double vn = s.omb2 * (sum_sq / L) + s.beta2 * static_cast<double>(v_old);
+    *v_new = static_cast<float>(vn);
+    const double denom = sqrt(vn * s.inv_bc2) + s.eps;
+    return static_cast<float>(s.lr_over_bc1 / denom);
+}
+
+// Segment lookup: the last segment whose unit_begin is <= unit.
+__device__ __forceinline__ int find_seg(const Seg *segs, int n_segs, int64_t unit) {
+    int lo = 0, hi = n_segs - 1;
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (segs[mid].unit_begin <= unit) lo = mid; else hi = mid - 1;
+    }
+    return lo;
+}
+
+__device__ __forceinline__ double warp_sum(double x) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    return x;
+}
+
+// ---------------------------------------------------------------------------
+// L <= 16: one thread per block, float32 scalars (at L == 1 this is AdamW)
+// ---------------------------------------------------------------------------
+struct SmallScalars {
+    float beta1, omb1, beta2, omb2, inv_bc2, lr_over_bc1, eps, lr_wd;
+};
+
+__device__ __forceinline__ float small_block_step(float mean_sq, float v_old, const SmallScalars &s,
+                                                  float *v_new) {
+    const float vn = fmaf(s.omb2, mean_sq, s.beta2 * v_old);
+    *v_new = vn;
+    const float denom = __fsqrt_rn(vn * s.inv_bc2) + s.eps;
+    return __fdiv_rn(s.lr_over_bc1, denom);
+}
+
+template <int GD>
+__device__ __forceinline__ void small_body(const DevTensor &t, const Seg &seg, int64_t local,
+                                           float *__restrict__ v, const SmallScalars &sc) {
+    const float lr_wd = t.wd ? sc.lr_wd : 0.f;
+    float *vt = v + t.v_offset;
+
+    if (seg.aux) {
+        // L == 1, everything 16-byte aligned: four blocks per thread per round.
+        const int64_t base = local * kSmallUnitVec;
+#pragma unroll
+        for (int r = 0; r < kSmallUnitVec / (kThreads * 4); ++r) {
+            const int64_t i = base + (static_cast<int64_t>(r) * kThreads + threadIdx.x) * 4;
+            if (i >= t.numel) break;
+            const float4 g = load_g4<GD>(t.g, i);
+            float4 m = *reinterpret_cast<const float4 *>(t.m + i);
+            float4 p = *reinterpret_cast<const float4 *>(t.p + i);
+            float4 vv = *reinterpret_cast<const float4 *>(vt + i);
+            float st;
+            st = small_block_step(g.x * g.x, vv.x, sc, &vv.x); update_one(g.x, m.x, p.x, sc.beta1, sc.omb1, lr_wd, st);
+            st = small_block_step(g.y * g.y, vv.y, sc, &vv.y); update_one(g.y, m.y, p.y, sc.beta1, sc.omb1, lr_wd, st);
+            st = small_block_step(g.z * g.z, vv.z, sc, &vv.z); update_one(g.z, m.z, p.z, sc.beta1, sc.omb1, lr_wd, st);
+            st = small_block_step(g.w * g.w, vv.w, sc, &vv.w); update_one(g.w, m.w, p.w, sc.beta1, sc.omb1, lr_wd, st);
+            *reinterpret_cast<float4 *>(t.m + i) = m;
+            *reinterpret_cast<float4 *>(t.p + i) = p;
+            *reinterpret_cast<float4 *>(vt + i) = vv;
+        }
+        return;
+    }
+
+    const int L = static_cast<int>(t.L);
+    const float Lf = static_cast<float>(L);
+    for (int r = 0; r < kSmallUnitBlocks / kThreads; ++r) {
+        const int64_t b = local * kSmallUnitBlocks + static_cast<int64_t>(r) * kThreads + threadIdx.x;
+        if (b >= t.n_blocks) break;
+        const int64_t e0 = b * L;
+        float gl[kSmallMaxL];
+        float sum = 0.f;
+#pragma unroll
+        for (int k = 0; k < kSmallMaxL; ++k) {
+            if (k < L) {
+                gl[k] = load_g1<GD>(t.g, e0 + k);
+                sum = fmaf(gl[k], gl[k], sum);
+            }
+        }
+        float vn;
+        const float st = small_block_step(L == 1 ? sum : __fdiv_rn(sum, Lf), vt[b], sc, &vn);
+        vt[b] = vn;
+#pragma unroll
+        for (int k = 0; k < kSmallMaxL; ++k) {
+            if (k < L) {
+                float m = t.m[e0 + k], p = t.p[e0 + k];
+                update_one(gl[k], m, p, sc.beta1, sc.omb1, lr_wd, st);
+                t.m[e0 + k] = m;
+                t.p[e0 + k] = p;
+            }
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kThreads)
+small_kernel(const DevTensor *__restrict__ tensors, const Seg *__restrict__ segs, int n_segs,
+             float *__restrict__ v, SmallScalars sc) {
+    const int64_t unit = blockIdx.x;
+    const Seg seg = segs[find_seg(segs, n_segs, unit)];
+    const DevTensor &t = tensors[seg.tensor];
+    const int64_t local = unit - seg.unit_begin;
+    if (t.gdtype == AM_BF16) small_body<AM_BF16>(t, seg, local, v, sc);
+    else small_body<AM_F32>(t, seg, local, v, sc);
+}
+
+// ---------------------------------------------------------------------------
+// two-pass path.  Units of the partial and update kernels are pieces:
+// piece (b, j) of a tensor covers elements [b*L + j*piece_len, ...) of block b.
+// ---------------------------------------------------------------------------
+struct PieceRef {
+    const DevTensor *t;
+    int64_t block, start, n, local;
+    bool vec;
+};
+
+__device__ __forceinline__ PieceRef decode_piece(const DevTensor *tensors, const Seg *segs, int n_segs,
+                                                 int64_t unit) {
+    const Seg seg = segs[find_seg(segs, n_segs, unit)];
+    PieceRef r;
+    r.t = &tensors[seg.tensor];
+    r.local = unit - seg.unit_begin;
+    r.block = r.local / r.t->pieces_per_block;
+    const int64_t j = r.local - r.block * r.t->pieces_per_block;
+    const int64_t off = j * r.t->piece_len;
+    r.start = r.block * r.t->L + off;
+    const int64_t left = r.t->L - off;
+    r.n = left < r.t->piece_len ? left : r.t->piece_len;
+    r.vec = seg.aux != 0;
+    return r;
+}
+
+// Sum of squares of one piece.  Per-thread float chains stay short (<= 64 terms
+// per accumulator); everything above a thread is double and combined in a
+// fixed order, so results do not depend on scheduling.
+template <int GD>
+__device__ __forceinline__ double piece_sum_sq(const PieceRef &r) {
+    double tot = 0.0;
+    if (r.vec) {
+        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+        int chain = 0;
+        for (int64_t i = static_cast<int64_t>(threadIdx.x) * 4; i < r.n; i += kThreads * 4) {
+            const float4 g = load_g4<GD>(r.t->g, r.start + i);
+            a0 = fmaf(g.x, g.x, a0); a1 = fmaf(g.y, g.y, a1);
+            a2 = fmaf(g.z, g.z, a2); a3 = fmaf(g.w, g.w, a3);
+            if (++chain == 64) {
+                tot += (static_cast<double>(a0) + static_cast<double>(a1)) +
+                       (static_cast<double>(a2) + static_cast<double>(a3));
+                a0 = a1 = a2 = a3 = 0.f;
+                chain = 0;
+            }
+        }
+        tot += (static_cast<double>(a0) + static_cast<double>(a1)) +
+               (static_cast<double>(a2) + static_cast<double>(a3));
+    } else {
+        float a = 0.f;
+        int chain = 0;
+        for (int64_t i = threadIdx.x; i < r.n; i += kThreads) {
+            const float g = load_g1<GD>(r.t->g, r.start + i);
+            a = fmaf(g, g, a);
+            if (++chain == 64) { tot += static_cast<double>(a); a = 0.f; chain = 0; }
+        }
+        tot += static_cast<double>(a);
+    }
+    return tot;
+}
+
+__global__ void __launch_bounds__(kThreads)
+twopass_partial_kernel(const DevTensor *__restrict__ tensors, const Seg *__restrict__ segs, int n_segs,
+                       double *__restrict__ partials) {
+    __shared__ double warp_part[kThreads / 32];
+    const PieceRef r = decode_piece(tensors, segs, n_segs, blockIdx.x);
+    const double w = warp_sum(r.t->gdtype == AM_BF16 ? piece_sum_sq<AM_BF16>(r) : piece_sum_sq<AM_F32>(r));
+    if ((threadIdx.x & 31) == 0) warp_part[threadIdx.x >> 5] = w;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double s = 0.0;
+#pragma unroll
+        for (int k = 0; k < kThreads / 32; ++k) s += warp_part[k];
+        partials[r.t->piece_base + r.local] = s;
+    }
+}
+
+// One warp per block: fixed-order sum of the block's partials, then v_b and
+// the block's step size.
+__global__ void __launch_bounds__(kThreads)
+twopass_finalize_kernel(const DevTensor *__restrict__ tensors, const Seg *__restrict__ segs, int n_segs,
+                        int64_t n_units, const double *__restrict__ partials,
+                        float *__restrict__ block_steps, float *__restrict__ v, StepScalars sc) {
+    const int64_t unit = static_cast<int64_t>(blockIdx.x) * (kThreads / 32) + (threadIdx.x >> 5);
+    if (unit >= n_units) return;
+    const int lane = threadIdx.x & 31;
+    const Seg seg = segs[find_seg(segs, n_segs, unit)];
+    const DevTensor &t = tensors[seg.tensor];
+    const int64_t b = unit - seg.unit_begin;
+    const double *src = partials + t.piece_base + b * t.pieces_per_block;
+    double s = 0.0;
+    for (int64_t j = lane; j < t.pieces_per_block; j += 32) s += src[j];
+    s = warp_sum(s);
+    if (lane == 0) {
+        float vn;
+        const float st = block_step(s, static_cast<double>(t.L), v[t.v_offset + b], sc, &vn);
+        v[t.v_offset + b] = vn;
+        block_steps[t.block_base + b] = st;
+    }
+}
+
+template <int GD>
+__device__ __forceinline__ void twopass_update_body(const PieceRef &r, const float *__restrict__ block_steps,
+                                                    const StepScalars &sc) {
+    const DevTensor &t = *r.t;
+    const float st = block_steps[t.block_base + r.block];
+    const float lr_wd = t.wd ? sc.lr_wd : 0.f;
+    if (r.vec) {
+        for (int64_t i = static_cast<int64_t>(threadIdx.x) * 4; i < r.n; i += kThreads * 4) {
+            const int64_t e = r.start + i;
+            const float4 g = load_g4<GD>(t.g, e);
+            float4 m = *reinterpret_cast<const float4 *>(t.m + e);
+            float4 p = *reinterpret_cast<const float4 *>(t.p + e);
+            update_four(g, m, p, sc.beta1, sc.omb1, lr_wd, st);
+            *reinterpret_cast<float4 *>(t.m + e) = m;
+            *reinterpret_cast<float4 *>(t.p + e) = p;
+        }
+    } else {
+        for (int64_t i = threadIdx.x; i < r.n; i += kThreads) {
+            const int64_t e = r.start + i;
+            const float g = load_g1<GD>(t.g, e);
+            float m = t.m[e], p = t.p[e];
+            update_one(g, m, p, sc.beta1, sc.omb1, lr_wd, st);
+            t.m[e] = m;
+            t.p[e] = p;
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kThreads)
+twopass_update_kernel(const DevTensor *__restrict__ tensors, const Seg *__restrict__ segs, int n_segs,
+                      const float *__restrict__ block_steps, StepScalars sc) {
+    const PieceRef r = decode_piece(tensors, segs, n_segs, blockIdx.x);
+    if (r.t->gdtype == AM_BF16) twopass_update_body<AM_BF16>(r, block_steps, sc);
+    else twopass_update_body<AM_F32>(r, block_steps, sc);
+}
+
+}  // namespace am
+
+#endif  // ADAMMINI_KERNELS_BASIC_CUH_
