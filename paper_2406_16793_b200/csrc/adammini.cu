@@ -1,0 +1,410 @@
+// Host side of the Adam-mini step library: handle, launch planning, C ABI.
+// Every step of Algorithm 1 of the paper runs in the kernels of
+// kernels_basic.cuh and kernels_stream.cuh; this file only validates, plans
+// and launches.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "adammini_internal.h"
+#include "kernels_basic.cuh"
+#include "kernels_stream.cuh"
+#include "host_state.h"
+
+using namespace am;
+
+namespace {
+
+constexpr int kNumOptions = 4;
+
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+int cuda_fail(am_handle *h, cudaError_t e) {
+    if (h) h->last_cuda_error = static_cast<int>(e);
+    return AM_ERR_CUDA;
+}
+
+#define AM_CUDA(h, call)                                   \
+    do {                                                   \
+        cudaError_t e__ = (call);                          \
+        if (e__ != cudaSuccess) return cuda_fail((h), e__); \
+    } while (0)
+
+int validate_hparams(const am_hparams *hp) {
+    if (!hp) return AM_ERR_INVALID_ARGUMENT;
+    const double vals[5] = {hp->lr, hp->beta1, hp->beta2, hp->eps, hp->weight_decay};
+    for (double x : vals)
+        if (!std::isfinite(x)) return AM_ERR_INVALID_ARGUMENT;
+    if (hp->lr < 0.0 || hp->weight_decay < 0.0 || hp->eps <= 0.0) return AM_ERR_INVALID_ARGUMENT;
+    if (hp->beta1 < 0.0 || hp->beta1 >= 1.0 || hp->beta2 < 0.0 || hp->beta2 >= 1.0)
+        return AM_ERR_INVALID_ARGUMENT;
+    return AM_OK;
+}
+
+void release_plan(am_handle *h) {
+    if (h->arena) cudaFree(h->arena);
+    h->arena = nullptr;
+    h->arena_bytes = 0;
+    h->planned = false;
+    h->ptrs_valid = false;
+}
+
+// Decide the kernel family of every tensor, build the unit tables and the
+// device arena.  Called at creation and after an option changes.
+int build_plan(am_handle *h) {
+    release_plan(h);
+    const int n = static_cast<int>(h->rows.size());
+    h->path.assign(n, PATH_TWOPASS);
+    h->host_tensors.assign(n, DevTensor{});
+    std::vector<Seg> small_segs, piece_segs, block_segs;
+    int64_t small_units = 0, piece_units = 0, block_units = 0;
+    for (int k = 0; k < 4; ++k) h->elems_by_path[k] = 0;
+    h->algorithmic_bytes = 0;
+
+    StreamPlanInput sin;
+    sin.sm_count = h->sm_count;
+    sin.ctas = static_cast<int>(h->opt[AM_OPT_STREAM_CTAS]);
+    sin.cluster_size = static_cast<int>(h->opt[AM_OPT_CLUSTER_SIZE]);
+    sin.threads = static_cast<int>(h->opt[AM_OPT_STREAM_THREADS]);
+
+    stream_probe_cluster(h->sm_count, sin.threads, sin.cluster_size, &h->cluster_size, &h->n_clusters);
+
+    for (int i = 0; i < n; ++i) {
+        const am_table_row &r = h->rows[i];
+        DevTensor &t = h->host_tensors[i];
+        t.numel = r.numel;
+        t.L = r.block_len;
+        t.n_blocks = r.n_blocks;
+        t.v_offset = r.v_offset;
+        t.gdtype = r.grad_dtype;
+        t.wd = r.wd;
+        const int64_t gsz = r.grad_dtype == AM_BF16 ? 2 : 4;
+
+        int path;
+        if (r.block_len <= kSmallMaxL) path = PATH_SMALL;
+        else if (h->opt[AM_OPT_PATH] == 1) path = PATH_TWOPASS;
+        else path = stream_classify(r.block_len, r.grad_dtype, h->n_clusters > 0);
+        h->path[i] = path;
+        h->elems_by_path[path] += r.numel;
+
+        // bytes the update must move: g once if a block can stay on chip / in
+        // L2 between its reduction and its update, twice otherwise
+        const int64_t g_reads = r.block_len * gsz > kClusterMaxBlockBytes ? 2 : 1;
+        h->algorithmic_bytes += r.numel * (g_reads * gsz + 16) + r.n_blocks * 8;
+
+        if (path == PATH_SMALL) {
+            Seg s;
+            s.unit_begin = small_units;
+            s.tensor = i;
+            s.aux = (r.block_len == 1 && r.v_offset % 4 == 0 && r.numel % 4 == 0) ? 1 : 0;
+            small_units += s.aux ? ceil_div(r.numel, kSmallUnitVec) : ceil_div(r.n_blocks, kSmallUnitBlocks);
+            small_segs.push_back(s);
+        } else if (path == PATH_TWOPASS) {
+            int64_t piece_len = r.block_len, ppb = 1;
+            if (r.block_len > kPieceMax) {
+                ppb = std::min<int64_t>(ceil_div(r.block_len, kPieceMax), kMaxPiecesPerBlock);
+                piece_len = ceil_div(ceil_div(r.block_len, ppb), 1024) * 1024;
+                ppb = ceil_div(r.block_len, piece_len);
+            }
+            t.piece_len = piece_len;
+            t.pieces_per_block = ppb;
+            t.piece_base = piece_units;
+            t.block_base = block_units;
+            Seg s;
+            s.unit_begin = piece_units;
+            s.tensor = i;
+            s.aux = (r.block_len % 4 == 0) ? 1 : 0;
+            piece_segs.push_back(s);
+            Seg b;
+            b.unit_begin = block_units;
+            b.tensor = i;
+            b.aux = 0;
+            block_segs.push_back(b);
+            piece_units += r.n_blocks * ppb;
+            block_units += r.n_blocks;
+        } else {
+            stream_add_tensor(sin, i, r, path);
+        }
+    }
+    if (small_units > 0x7fffffffLL || piece_units > 0x7fffffffLL || ceil_div(block_units, kThreads / 32) > 0x7fffffffLL)
+        return AM_ERR_TOO_LARGE;
+
+    StreamPlan &sp = h->stream;
+    stream_finish_plan(sin, h->cluster_size, h->n_clusters, &sp);
+
+    // device arena: tensor table, unit tables, scratch
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = round_up(off + bytes, 256); return o; };
+    const size_t o_tensors = take(sizeof(DevTensor) * std::max(n, 1));
+    const size_t o_small = take(sizeof(Seg) * std::max<size_t>(small_segs.size(), 1));
+    const size_t o_piece = take(sizeof(Seg) * std::max<size_t>(piece_segs.size(), 1));
+    const size_t o_block = take(sizeof(Seg) * std::max<size_t>(block_segs.size(), 1));
+    const size_t o_partials = take(sizeof(double) * std::max<int64_t>(piece_units, 1));
+    const size_t o_steps = take(sizeof(float) * std::max<int64_t>(block_units, 1));
+    const size_t o_stream = take(std::max<size_t>(sp.table_bytes(), 16));
+    h->arena_bytes = off;
+    AM_CUDA(h, cudaMalloc(&h->arena, h->arena_bytes));
+    char *base = static_cast<char *>(h->arena);
+    h->d_tensors = reinterpret_cast<DevTensor *>(base + o_tensors);
+    h->d_small_segs = reinterpret_cast<Seg *>(base + o_small);
+    h->d_piece_segs = reinterpret_cast<Seg *>(base + o_piece);
+    h->d_block_segs = reinterpret_cast<Seg *>(base + o_block);
+    h->d_partials = reinterpret_cast<double *>(base + o_partials);
+    h->d_block_steps = reinterpret_cast<float *>(base + o_steps);
+    h->n_small_segs = static_cast<int>(small_segs.size());
+    h->n_piece_segs = static_cast<int>(piece_segs.size());
+    h->n_block_segs = static_cast<int>(block_segs.size());
+    h->small_units = small_units;
+    h->piece_units = piece_units;
+    h->block_units = block_units;
+    if (!small_segs.empty())
+        AM_CUDA(h, cudaMemcpy(h->d_small_segs, small_segs.data(), sizeof(Seg) * small_segs.size(), cudaMemcpyHostToDevice));
+    if (!piece_segs.empty())
+        AM_CUDA(h, cudaMemcpy(h->d_piece_segs, piece_segs.data(), sizeof(Seg) * piece_segs.size(), cudaMemcpyHostToDevice));
+    if (!block_segs.empty())
+        AM_CUDA(h, cudaMemcpy(h->d_block_segs, block_segs.data(), sizeof(Seg) * block_segs.size(), cudaMemcpyHostToDevice));
+    {
+        cudaError_t e = sp.upload(base + o_stream);
+        if (e != cudaSuccess) return cuda_fail(h, e);
+    }
+
+    h->launches = (small_units ? 1 : 0) + (piece_units ? 3 : 0) + sp.launches();
+    h->planned = true;
+    return AM_OK;
+}
+
+// Refresh the device tensor table if any data pointer changed.
+int refresh_pointers(am_handle *h, void *const *params, const void *const *grads, void *const *m,
+                     cudaStream_t stream) {
+    const int n = static_cast<int>(h->rows.size());
+    bool changed = !h->ptrs_valid;
+    for (int i = 0; i < n; ++i) {
+        DevTensor &t = h->host_tensors[i];
+        if (t.g != grads[i] || t.m != m[i] || t.p != params[i]) {
+            t.g = grads[i];
+            t.m = static_cast<float *>(m[i]);
+            t.p = static_cast<float *>(params[i]);
+            changed = true;
+        }
+    }
+    if (!changed || n == 0) return AM_OK;
+    const int k = h->next_pinned;
+    h->next_pinned ^= 1;
+    if (h->ev_pending[k]) {
+        AM_CUDA(h, cudaEventSynchronize(h->ev[k]));   // the copy that last read this buffer
+        h->ev_pending[k] = false;
+    }
+    std::memcpy(h->pinned[k], h->host_tensors.data(), sizeof(DevTensor) * n);
+    AM_CUDA(h, cudaMemcpyAsync(h->d_tensors, h->pinned[k], sizeof(DevTensor) * n, cudaMemcpyHostToDevice, stream));
+    AM_CUDA(h, cudaEventRecord(h->ev[k], stream));
+    h->ev_pending[k] = true;
+    h->ptrs_valid = true;
+    return AM_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int adammini_create(const am_partition *part, const am_hparams *hp, am_handle **out) {
+    if (!out) return AM_ERR_INVALID_ARGUMENT;
+    *out = nullptr;
+    if (!part) return AM_ERR_INVALID_ARGUMENT;
+    int rc = validate_hparams(hp);
+    if (rc != AM_OK) return rc;
+    am_handle *h = new (std::nothrow) am_handle();
+    if (!h) return AM_ERR_ALLOC;
+    try {
+        h->rows = part->rows;
+    } catch (...) {
+        delete h;
+        return AM_ERR_ALLOC;
+    }
+    h->total_blocks = part->total_blocks;
+    for (const am_table_row &r : h->rows) h->total_elems += r.numel;
+    h->hp = *hp;
+
+    cudaError_t e = cudaGetDevice(&h->device);
+    cudaDeviceProp prop;
+    if (e == cudaSuccess) e = cudaGetDeviceProperties(&prop, h->device);
+    if (e == cudaSuccess) {
+        h->sm_count = prop.multiProcessorCount;
+        const size_t n = std::max<size_t>(h->rows.size(), 1);
+        for (int k = 0; k < 2 && e == cudaSuccess; ++k) {
+            e = cudaMallocHost(&h->pinned[k], sizeof(DevTensor) * n);
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev[k], cudaEventDisableTiming);
+        }
+    }
+    if (e == cudaSuccess) e = cudaMallocHost(&h->error_word, sizeof(int));
+    if (e == cudaSuccess) *h->error_word = 0;
+    if (e == cudaSuccess) e = stream_configure_kernels();
+    if (e != cudaSuccess) {
+        const int code = static_cast<int>(e);
+        adammini_destroy(h);
+        (void)code;
+        return AM_ERR_CUDA;
+    }
+    rc = build_plan(h);
+    if (rc != AM_OK) {
+        adammini_destroy(h);
+        return rc;
+    }
+    *out = h;
+    return AM_OK;
+}
+
+int adammini_set_lr(am_handle *h, double lr) {
+    if (!h || !std::isfinite(lr) || lr < 0.0) return AM_ERR_INVALID_ARGUMENT;
+    h->hp.lr = lr;
+    return AM_OK;
+}
+
+int adammini_set_hparams(am_handle *h, const am_hparams *hp) {
+    if (!h) return AM_ERR_INVALID_ARGUMENT;
+    const int rc = validate_hparams(hp);
+    if (rc != AM_OK) return rc;
+    h->hp = *hp;
+    return AM_OK;
+}
+
+int adammini_set_option(am_handle *h, int32_t key, int64_t value) {
+    if (!h || key < 0 || key >= kNumOptions || value < 0) return AM_ERR_INVALID_ARGUMENT;
+    if (key == AM_OPT_PATH && value > 1) return AM_ERR_INVALID_ARGUMENT;
+    if (key == AM_OPT_CLUSTER_SIZE && value != 0 && value != 1 && value != 2 && value != 4 && value != 8)
+        return AM_ERR_INVALID_ARGUMENT;
+    if (key == AM_OPT_STREAM_THREADS && value != 0 && (value % 32 != 0 || value < 64 || value > 512))
+        return AM_ERR_INVALID_ARGUMENT;
+    if (h->opt[key] == value) return AM_OK;
+    AM_CUDA(h, cudaDeviceSynchronize());    // the old tables may still be in use
+    const int64_t old = h->opt[key];
+    h->opt[key] = value;
+    int rc = build_plan(h);
+    if (rc != AM_OK) {
+        h->opt[key] = old;
+        build_plan(h);
+    }
+    return rc;
+}
+
+int adammini_query(const am_handle *h, int32_t what, int64_t *value) {
+    if (!h || !value) return AM_ERR_INVALID_ARGUMENT;
+    switch (what) {
+    case AM_Q_LAUNCHES_PER_STEP: *value = h->launches; break;
+    case AM_Q_SCRATCH_BYTES: *value = static_cast<int64_t>(h->arena_bytes); break;
+    case AM_Q_TOTAL_BLOCKS: *value = h->total_blocks; break;
+    case AM_Q_TOTAL_ELEMENTS: *value = h->total_elems; break;
+    case AM_Q_ELEMENTS_SMALL: *value = h->elems_by_path[PATH_SMALL]; break;
+    case AM_Q_ELEMENTS_STREAM: *value = h->elems_by_path[PATH_STREAM]; break;
+    case AM_Q_ELEMENTS_CLUSTER: *value = h->elems_by_path[PATH_CLUSTER]; break;
+    case AM_Q_ELEMENTS_TWOPASS: *value = h->elems_by_path[PATH_TWOPASS]; break;
+    case AM_Q_ALGORITHMIC_BYTES: *value = h->algorithmic_bytes; break;
+    default: return AM_ERR_INVALID_ARGUMENT;
+    }
+    return AM_OK;
+}
+
+int adammini_last_cuda_error(const am_handle *h) { return h ? h->last_cuda_error : 0; }
+
+int adammini_step(am_handle *h, void *const *params, const void *const *grads, void *const *m,
+                  float *v, int64_t step, void *cuda_stream) {
+    if (!h || !h->planned || step < 1) return AM_ERR_INVALID_ARGUMENT;
+    const int n = static_cast<int>(h->rows.size());
+    if (n == 0) return AM_OK;
+    if (!params || !grads || !m || !v) return AM_ERR_INVALID_ARGUMENT;
+    for (int i = 0; i < n; ++i) {
+        if (!params[i] || !grads[i] || !m[i]) return AM_ERR_INVALID_ARGUMENT;
+        if (!aligned16(params[i]) || !aligned16(grads[i]) || !aligned16(m[i])) return AM_ERR_MISALIGNED;
+    }
+    if (!aligned16(v)) return AM_ERR_MISALIGNED;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+
+    int dev = -1;
+    AM_CUDA(h, cudaGetDevice(&dev));
+    if (dev != h->device) return AM_ERR_INVALID_ARGUMENT;
+
+    int rc = refresh_pointers(h, params, grads, m, stream);
+    if (rc != AM_OK) return rc;
+
+    // scalars of this step (Algorithm 1: bias corrections use beta^t)
+    const am_hparams &hp = h->hp;
+    const double bc1 = 1.0 - std::pow(hp.beta1, static_cast<double>(step));
+    const double bc2 = 1.0 - std::pow(hp.beta2, static_cast<double>(step));
+    StepScalars sc;
+    sc.beta2 = hp.beta2;
+    sc.omb2 = 1.0 - hp.beta2;
+    sc.inv_bc2 = 1.0 / bc2;
+    sc.lr_over_bc1 = hp.lr / bc1;
+    sc.eps = hp.eps;
+    sc.beta1 = static_cast<float>(hp.beta1);
+    sc.omb1 = static_cast<float>(1.0 - hp.beta1);
+    sc.lr_wd = static_cast<float>(hp.lr * hp.weight_decay);
+    sc.pad = 0.f;
+
+    if (h->small_units) {
+        SmallScalars ss;
+        ss.beta1 = sc.beta1;
+        ss.omb1 = sc.omb1;
+        ss.beta2 = static_cast<float>(hp.beta2);
+        ss.omb2 = static_cast<float>(1.0 - hp.beta2);
+        ss.inv_bc2 = static_cast<float>(sc.inv_bc2);
+        ss.lr_over_bc1 = static_cast<float>(sc.lr_over_bc1);
+        ss.eps = static_cast<float>(hp.eps);
+        ss.lr_wd = sc.lr_wd;
+        small_kernel<<<static_cast<unsigned>(h->small_units), kThreads, 0, stream>>>(
+            h->d_tensors, h->d_small_segs, h->n_small_segs, v, ss);
+        AM_CUDA(h, cudaGetLastError());
+    }
+    {
+        cudaError_t e = h->stream.launch(h->d_tensors, v, sc, h->error_word, stream);
+        if (e != cudaSuccess) return cuda_fail(h, e);
+    }
+    if (h->piece_units) {
+        twopass_partial_kernel<<<static_cast<unsigned>(h->piece_units), kThreads, 0, stream>>>(
+            h->d_tensors, h->d_piece_segs, h->n_piece_segs, h->d_partials);
+        AM_CUDA(h, cudaGetLastError());
+        const unsigned fin_grid = static_cast<unsigned>(ceil_div(h->block_units, kThreads / 32));
+        twopass_finalize_kernel<<<fin_grid, kThreads, 0, stream>>>(
+            h->d_tensors, h->d_block_segs, h->n_block_segs, h->block_units, h->d_partials,
+            h->d_block_steps, v, sc);
+        AM_CUDA(h, cudaGetLastError());
+        twopass_update_kernel<<<static_cast<unsigned>(h->piece_units), kThreads, 0, stream>>>(
+            h->d_tensors, h->d_piece_segs, h->n_piece_segs, h->d_block_steps, sc);
+        AM_CUDA(h, cudaGetLastError());
+    }
+    return AM_OK;
+}
+
+int adammini_sync_status(am_handle *h, void *cuda_stream) {
+    if (!h) return AM_ERR_INVALID_ARGUMENT;
+    AM_CUDA(h, cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)));
+    if (h->error_word && *h->error_word != 0) {
+        *h->error_word = 0;
+        return AM_ERR_TIMEOUT;
+    }
+    return AM_OK;
+}
+
+int adammini_destroy(am_handle *h) {
+    if (!h) return AM_OK;
+    cudaDeviceSynchronize();
+    host_step_release(h);
+    release_plan(h);
+    for (int k = 0; k < 2; ++k) {
+        if (h->pinned[k]) cudaFreeHost(h->pinned[k]);
+        if (h->ev[k]) cudaEventDestroy(h->ev[k]);
+    }
+    if (h->error_word) cudaFreeHost(h->error_word);
+    delete h;
+    return AM_OK;
+}
+
+}  // extern "C"
+
+#include "host_step.inl"

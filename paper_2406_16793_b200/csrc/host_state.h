@@ -1,0 +1,56 @@
+// The optimizer handle.
+#ifndef ADAMMINI_HOST_STATE_H_
+#define ADAMMINI_HOST_STATE_H_
+
+#include <cuda_runtime.h>
+
+#include <vector>
+
+#include "adammini_internal.h"
+#include "kernels_stream.cuh"
+
+struct HostStepState;   // staging for adammini_step_host, created on first use
+
+struct am_handle {
+    int device = 0;
+    int sm_count = 0;
+    std::vector<am_table_row> rows;
+    int64_t total_blocks = 0;
+    int64_t total_elems = 0;
+    am_hparams hp{};
+    int64_t opt[4] = {0, 0, 0, 0};
+
+    // launch plan
+    bool planned = false;
+    std::vector<int32_t> path;
+    std::vector<am::DevTensor> host_tensors;
+    void *arena = nullptr;
+    size_t arena_bytes = 0;
+    am::DevTensor *d_tensors = nullptr;
+    am::Seg *d_small_segs = nullptr, *d_piece_segs = nullptr, *d_block_segs = nullptr;
+    int n_small_segs = 0, n_piece_segs = 0, n_block_segs = 0;
+    int64_t small_units = 0, piece_units = 0, block_units = 0;
+    double *d_partials = nullptr;
+    float *d_block_steps = nullptr;
+    am::StreamPlan stream;
+    int cluster_size = 0, n_clusters = 0;   // what the device can keep resident (0: no cluster path)
+    int launches = 0;
+    int64_t elems_by_path[4] = {0, 0, 0, 0};
+    int64_t algorithmic_bytes = 0;
+
+    // pinned staging of the tensor table, double buffered
+    am::DevTensor *pinned[2] = {nullptr, nullptr};
+    cudaEvent_t ev[2] = {nullptr, nullptr};
+    bool ev_pending[2] = {false, false};
+    int next_pinned = 0;
+    bool ptrs_valid = false;
+
+    int *error_word = nullptr;   // pinned; kernels write a code here when a bounded wait gives up
+    int last_cuda_error = 0;
+
+    HostStepState *host_step = nullptr;
+};
+
+void host_step_release(am_handle *h);
+
+#endif  // ADAMMINI_HOST_STATE_H_

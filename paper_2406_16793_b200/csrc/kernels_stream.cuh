@@ -1,0 +1,712 @@
+// The single-read streaming kernels.
+//
+// One persistent CTA per SM.  A producer thread walks the CTA's share of the
+// work and moves gradients, first moments and parameters from HBM into a ring
+// of shared-memory stages with bulk asynchronous copies (cp.async.bulk,
+// completion counted on an mbarrier).  The consumer warps wait for a stage,
+// reduce g*g over each block (Algorithm 1: v = (1-beta2) mean(g*g) + beta2 v),
+// turn the block's new v into a step size and apply the elementwise update,
+// writing m and p back with 16-byte stores.
+//
+// Three kinds of stage:
+//   PACKED  whole blocks (block_len <= kStageElems) with their g, m and p: g is
+//           read from HBM exactly once.
+//   SUM     gradients only, for a block longer than a stage: consumers add up
+//           g*g; the last SUM stage of a block ends with the reduction (across
+//           the CTAs of a cluster through distributed shared memory when the
+//           block is split over a cluster).
+//   APPLY   g, m, p of one chunk of that block: g is fetched a second time, a
+//           few microseconds after the first, and is served by L2.
+//
+// Every wait is bounded: a wait that gives up sets the abort flag and the
+// handle's error word, and all roles leave through the common exit.
+#ifndef ADAMMINI_KERNELS_STREAM_CUH_
+#define ADAMMINI_KERNELS_STREAM_CUH_
+
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <vector>
+
+#include "adammini_internal.h"
+#include "kernels_basic.cuh"
+
+namespace am {
+
+constexpr int kStageElems = 4096;                 // elements of g, m, p per PACKED/APPLY stage
+constexpr int kWarpBlockMaxL = 1024;              // blocks up to this length are reduced by one warp
+constexpr int kCtrlBytes = 2048;                  // barriers, stage descriptors, reduction slots
+constexpr int kMaxStages = 8;
+constexpr int kMaxConsumerWarps = 16;
+constexpr int kMaxCluster = 8;
+constexpr int64_t kStreamMaxBlockBytes = 256 << 10;   // longest block one CTA handles alone (bytes of g)
+constexpr int64_t kClusterMaxBlockBytes = 4 << 20;    // longest block a cluster handles (bytes of g)
+constexpr unsigned long long kWaitTimeoutNs = 2000000000ull;   // 2 s
+constexpr unsigned long long kDrainTimeoutNs = 50000000ull;    // 50 ms
+
+enum StageKind : int32_t { STAGE_PACKED = 0, STAGE_SUM = 1, STAGE_APPLY = 2, STAGE_DONE = 3 };
+enum StageFlag : int32_t { SF_BF16 = 1, SF_WD = 2, SF_LAST = 4, SF_WRITE_V = 8 };
+
+struct StageMeta {          // written by the producer, read by the consumers
+    float *m;               // global destination of this stage's first element
+    float *p;
+    float *v;               // v of the stage's first block
+    double inv_L;           // 1 / block length
+    int32_t n;              // elements in the stage
+    int32_t L;              // block length (PACKED)
+    int32_t kind;
+    int32_t flags;
+    int64_t pad[2];
+};
+static_assert(sizeof(StageMeta) == 64, "stage descriptor is 64 bytes");
+
+struct StreamSeg {          // a run of items of one tensor
+    int64_t item_begin;
+    int32_t tensor;
+    int32_t bpi;            // blocks per item (PACKED); 0: one long block per item
+};
+
+struct StreamParams {
+    const DevTensor *tensors;
+    const StreamSeg *segs;      // n_segs entries plus a sentinel
+    const int64_t *bounds;      // item range of CTA (or cluster) k is [bounds[k], bounds[k+1])
+    float *v;
+    int *error_word;
+    StepScalars sc;
+    int32_t n_segs;
+    int32_t n_stages;
+    int32_t stage_bytes;
+    int32_t g_region_bytes;     // m starts here inside a stage; p follows kStageElems floats later
+    int32_t consumer_threads;
+};
+
+struct Control {            // first kCtrlBytes of dynamic shared memory
+    unsigned long long full[kMaxStages];
+    unsigned long long empty[kMaxStages];
+    unsigned long long redbar;
+    unsigned long long xbar[2];
+    double red[2][kMaxConsumerWarps];
+    double xpart[2][kMaxCluster];
+    float redv[2];
+    int abort_flag;
+    int pad;
+    StageMeta meta[kMaxStages];
+};
+static_assert(sizeof(Control) <= kCtrlBytes, "control block fits its reservation");
+
+// ------------------------------- PTX wrappers -------------------------------
+__device__ __forceinline__ uint32_t smem_addr(const void *p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(void *bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(void *bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(void *bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(void *bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(void *bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bulk asynchronous copy global -> shared; bytes and both addresses are multiples of 16.
+__device__ __forceinline__ void bulk_load(void *dst_smem, const void *src_gmem, uint32_t bytes, void *bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        ::"r"(smem_addr(dst_smem)), "l"(src_gmem), "r"(bytes), "r"(smem_addr(bar)) : "memory");
+}
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r;
+}
+__device__ __forceinline__ uint32_t cluster_nctarank() {
+    uint32_t r; asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r)); return r;
+}
+__device__ __forceinline__ uint32_t cluster_id_x() {
+    uint32_t r; asm volatile("mov.u32 %0, %%clusterid.x;" : "=r"(r)); return r;
+}
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t local_smem_addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_smem_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void st_cluster_f64(uint32_t cluster_addr, double x) {
+    asm volatile("st.shared::cluster.f64 [%0], %1;" ::"r"(cluster_addr), "d"(x) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release;\n\tbarrier.cluster.wait.acquire;" ::: "memory");
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t;
+}
+
+// Bounded wait on an mbarrier phase.  Returns false (after raising the abort
+// flag) if the phase did not complete within the limit or another thread of
+// the CTA already gave up.
+template <bool CLUSTER_ACQUIRE>
+__device__ __forceinline__ bool wait_phase(void *bar, uint32_t parity, Control *ctl, int *error_word,
+                                           int code, unsigned long long limit_ns = kWaitTimeoutNs) {
+    uint32_t spins = 0;
+    unsigned long long t0 = 0;
+    for (;;) {
+        const bool ok = CLUSTER_ACQUIRE ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity);
+        if (ok) return true;
+        if ((++spins & 255u) == 0) {
+            if (*reinterpret_cast<volatile int *>(&ctl->abort_flag)) return false;
+            const unsigned long long now = global_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > limit_ns) {
+                *reinterpret_cast<volatile int *>(&ctl->abort_flag) = 1;
+                *reinterpret_cast<volatile int *>(error_word) = code;
+                return false;
+            }
+        }
+    }
+}
+
+// ------------------------- consumer-side building blocks -------------------------
+template <int GD>
+__device__ __forceinline__ float4 lds_g4(const unsigned char *gs, int i) {
+    if (GD == AM_BF16) {
+        const uint2 u = *reinterpret_cast<const uint2 *>(gs + 2 * i);
+        return make_float4(bf16_lo(u.x), bf16_hi(u.x), bf16_lo(u.y), bf16_hi(u.y));
+    } else {
+        return *reinterpret_cast<const float4 *>(gs + 4 * i);
+    }
+}
+
+// Per-block scalars in float (one per block; the sum arrives as a double).
+__device__ __forceinline__ float stream_block_step(double sum_sq, double inv_L, float v_old,
+                                                   const StepScalars &s, float *v_new) {
+    const float mean = static_cast<float>(sum_sq * inv_L);
+    const float vn = fmaf(static_cast<float>(s.omb2), mean, static_cast<float>(s.beta2) * v_old);
+    *v_new = vn;
+    const float denom = __fsqrt_rn(vn * static_cast<float>(s.inv_bc2)) + static_cast<float>(s.eps);
+    return __fdiv_rn(static_cast<float>(s.lr_over_bc1), denom);
+}
+
+// Elementwise update of n elements (n % 4 == 0) by `nthr` cooperating threads.
+template <int GD>
+__device__ __forceinline__ void apply_span(const unsigned char *gs, const float *ms, const float *ps,
+                                           float *mg, float *pg, int first, int n, int tid, int nthr,
+                                           float beta1, float omb1, float lr_wd, float step) {
+#pragma unroll 2
+    for (int i = first + tid * 4; i < first + n; i += nthr * 4) {
+        const float4 g = lds_g4<GD>(gs, i);
+        float4 m = *reinterpret_cast<const float4 *>(ms + i);
+        float4 p = *reinterpret_cast<const float4 *>(ps + i);
+        update_four(g, m, p, beta1, omb1, lr_wd, step);
+        __stcs(reinterpret_cast<float4 *>(mg + i), m);
+        __stcs(reinterpret_cast<float4 *>(pg + i), p);
+    }
+}
+
+template <int GD>
+__device__ __forceinline__ void sum_span(const unsigned char *gs, int first, int n, int tid, int nthr,
+                                         float &a0, float &a1, float &a2, float &a3) {
+#pragma unroll 2
+    for (int i = first + tid * 4; i < first + n; i += nthr * 4) {
+        const float4 g = lds_g4<GD>(gs, i);
+        a0 = fmaf(g.x, g.x, a0); a1 = fmaf(g.y, g.y, a1);
+        a2 = fmaf(g.z, g.z, a2); a3 = fmaf(g.w, g.w, a3);
+    }
+}
+
+__device__ __forceinline__ double fold4(float a0, float a1, float a2, float a3) {
+    return (static_cast<double>(a0) + static_cast<double>(a1)) +
+           (static_cast<double>(a2) + static_cast<double>(a3));
+}
+
+// State of the consumer group's own barrier (an mbarrier so that it is bounded).
+struct GroupSync {
+    uint32_t parity;
+    int buf;
+};
+
+// Sum `mine` over all consumer threads in a fixed order; also broadcasts
+// v_old read by thread 0.  Returns false on abort.
+__device__ __forceinline__ bool group_reduce(Control *ctl, GroupSync &gs, int *error_word, int ctid, int n_warps,
+                                             double mine, const float *v_ptr, double *total, float *v_old) {
+    const double w = warp_sum(mine);
+    const int lane = ctid & 31;
+    if (lane == 0) {
+        ctl->red[gs.buf][ctid >> 5] = w;
+        if (ctid == 0) ctl->redv[gs.buf] = *v_ptr;
+        mbar_arrive(&ctl->redbar);
+    }
+    if (!wait_phase<false>(&ctl->redbar, gs.parity, ctl, error_word, 3)) return false;
+    double s = 0.0;
+    for (int k = 0; k < n_warps; ++k) s += ctl->red[gs.buf][k];
+    *total = s;
+    *v_old = ctl->redv[gs.buf];
+    gs.parity ^= 1;
+    gs.buf ^= 1;
+    return true;
+}
+
+// ------------------------------------ kernel ------------------------------------
+template <bool CLUSTER>
+__global__ void __launch_bounds__(32 + kMaxConsumerWarps * 32, 1)
+stream_kernel(const __grid_constant__ StreamParams P) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    Control *ctl = reinterpret_cast<Control *>(smem);
+    unsigned char *stages = smem + kCtrlBytes;
+    const int tid = threadIdx.x;
+    const int n_cwarps = P.consumer_threads >> 5;
+    const uint32_t crank = CLUSTER ? cluster_ctarank() : 0;
+    const uint32_t csize = CLUSTER ? cluster_nctarank() : 1;
+    const uint32_t unit = CLUSTER ? cluster_id_x() : blockIdx.x;
+
+    if (tid == 0) {
+        for (int s = 0; s < P.n_stages; ++s) {
+            mbar_init(&ctl->full[s], 1);
+            mbar_init(&ctl->empty[s], n_cwarps);
+        }
+        mbar_init(&ctl->redbar, n_cwarps);
+        mbar_init(&ctl->xbar[0], csize);
+        mbar_init(&ctl->xbar[1], csize);
+        ctl->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (CLUSTER) cluster_sync_all();     // peers' barriers exist before anyone arrives on them
+
+    const int64_t item_lo = P.bounds[unit], item_hi = P.bounds[unit + 1];
+
+    if (tid < 32) {
+        // ------------------------------ producer ------------------------------
+        if (tid == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            int64_t armed = 0;              // stages armed so far
+            bool ok = true;
+            int seg = 0;
+            {
+                int lo = 0, hi = P.n_segs - 1;      // last segment starting at or before item_lo
+                while (lo < hi) {
+                    const int mid = (lo + hi + 1) >> 1;
+                    if (P.segs[mid].item_begin <= item_lo) lo = mid; else hi = mid - 1;
+                }
+                seg = lo;
+            }
+            auto acquire = [&]() -> bool {
+                return wait_phase<false>(&ctl->empty[stage], phase ^ 1u, ctl, P.error_word, 1);
+            };
+            auto advance = [&]() {
+                ++armed;
+                if (++stage == P.n_stages) { stage = 0; phase ^= 1u; }
+            };
+            for (int64_t it = item_lo; it < item_hi && ok; ++it) {
+                while (seg + 1 < P.n_segs && P.segs[seg + 1].item_begin <= it) ++seg;
+                const StreamSeg sg = P.segs[seg];
+                const DevTensor &t = P.tensors[sg.tensor];
+                const int64_t local = it - sg.item_begin;
+                const int gsz = t.gdtype == AM_BF16 ? 2 : 4;
+                const int base_flags = (t.gdtype == AM_BF16 ? SF_BF16 : 0) | (t.wd ? SF_WD : 0);
+                const unsigned char *gbase = static_cast<const unsigned char *>(t.g);
+                if (sg.bpi > 0) {
+                    const int64_t b0 = local * sg.bpi;
+                    const int64_t left = t.n_blocks - b0;
+                    const int nb = static_cast<int>(left < sg.bpi ? left : sg.bpi);
+                    const int64_t e0 = b0 * t.L;
+                    const int n = nb * static_cast<int>(t.L);
+                    if (!(ok = acquire())) break;
+                    StageMeta &mt = ctl->meta[stage];
+                    mt.m = t.m + e0; mt.p = t.p + e0; mt.v = P.v + t.v_offset + b0;
+                    mt.inv_L = 1.0 / static_cast<double>(t.L);
+                    mt.n = n; mt.L = static_cast<int>(t.L); mt.kind = STAGE_PACKED; mt.flags = base_flags | SF_WRITE_V;
+                    unsigned char *st = stages + static_cast<size_t>(stage) * P.stage_bytes;
+                    mbar_arrive_expect_tx(&ctl->full[stage], static_cast<uint32_t>(n) * (gsz + 8));
+                    bulk_load(st, gbase + e0 * gsz, n * gsz, &ctl->full[stage]);
+                    bulk_load(st + P.g_region_bytes, t.m + e0, n * 4, &ctl->full[stage]);
+                    bulk_load(st + P.g_region_bytes + kStageElems * 4, t.p + e0, n * 4, &ctl->full[stage]);
+                    advance();
+                } else {
+                    // one long block; a cluster splits it evenly over its CTAs
+                    const int64_t slice = t.L / csize;
+                    const int64_t e0 = local * t.L + crank * slice;
+                    const int sum_cap = P.stage_bytes / gsz;
+                    for (int64_t off = 0; off < slice && ok; off += sum_cap) {
+                        const int c = static_cast<int>(slice - off < sum_cap ? slice - off : sum_cap);
+                        if (!(ok = acquire())) break;
+                        StageMeta &mt = ctl->meta[stage];
+                        mt.m = nullptr; mt.p = nullptr; mt.v = P.v + t.v_offset + local;
+                        mt.inv_L = 1.0 / static_cast<double>(t.L);
+                        mt.n = c; mt.L = 0; mt.kind = STAGE_SUM;
+                        mt.flags = base_flags | (off + c == slice ? SF_LAST : 0) | (crank == 0 ? SF_WRITE_V : 0);
+                        unsigned char *st = stages + static_cast<size_t>(stage) * P.stage_bytes;
+                        mbar_arrive_expect_tx(&ctl->full[stage], static_cast<uint32_t>(c) * gsz);
+                        bulk_load(st, gbase + (e0 + off) * gsz, c * gsz, &ctl->full[stage]);
+                        advance();
+                    }
+                    for (int64_t off = 0; off < slice && ok; off += kStageElems) {
+                        const int c = static_cast<int>(slice - off < kStageElems ? slice - off : kStageElems);
+                        if (!(ok = acquire())) break;
+                        StageMeta &mt = ctl->meta[stage];
+                        mt.m = t.m + e0 + off; mt.p = t.p + e0 + off; mt.v = nullptr;
+                        mt.inv_L = 0.0;
+                        mt.n = c; mt.L = 0; mt.kind = STAGE_APPLY; mt.flags = base_flags;
+                        unsigned char *st = stages + static_cast<size_t>(stage) * P.stage_bytes;
+                        mbar_arrive_expect_tx(&ctl->full[stage], static_cast<uint32_t>(c) * (gsz + 8));
+                        bulk_load(st, gbase + (e0 + off) * gsz, c * gsz, &ctl->full[stage]);
+                        bulk_load(st + P.g_region_bytes, t.m + e0 + off, c * 4, &ctl->full[stage]);
+                        bulk_load(st + P.g_region_bytes + kStageElems * 4, t.p + e0 + off, c * 4, &ctl->full[stage]);
+                        advance();
+                    }
+                }
+            }
+            if (ok && acquire()) {
+                ctl->meta[stage].kind = STAGE_DONE;
+                mbar_arrive(&ctl->full[stage]);
+            } else {
+                // gave up: let copies that are still in flight land before the CTA retires
+                const int64_t back = armed < P.n_stages ? armed : P.n_stages;
+                int s = stage;
+                uint32_t ph = phase;
+                for (int64_t k = 0; k < back; ++k) {
+                    if (--s < 0) { s = P.n_stages - 1; ph ^= 1u; }
+                    const unsigned long long t0 = global_ns();
+                    while (!mbar_try_wait(&ctl->full[s], ph) && global_ns() - t0 < kDrainTimeoutNs) {}
+                }
+            }
+        }
+    } else {
+        // ------------------------------ consumers ------------------------------
+        const int ctid = tid - 32;
+        const int lane = ctid & 31, warp = ctid >> 5;
+        const int nthr = P.consumer_threads;
+        if (ctid < nthr) {
+            const float beta1 = P.sc.beta1, omb1 = P.sc.omb1;
+            int stage = 0;
+            uint32_t phase = 0;
+            GroupSync gsync{0u, 0};
+            float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;   // running sums of a long block
+            float long_step = 0.f;
+            uint32_t long_count = 0;                         // long blocks finished (cluster exchange slot/parity)
+            for (;;) {
+                if (!wait_phase<false>(&ctl->full[stage], phase, ctl, P.error_word, 2)) break;
+                const StageMeta mt = ctl->meta[stage];
+                if (mt.kind == STAGE_DONE) break;
+                const unsigned char *gs = stages + static_cast<size_t>(stage) * P.stage_bytes;
+                const float *ms = reinterpret_cast<const float *>(gs + P.g_region_bytes);
+                const float *ps = ms + kStageElems;
+                const bool bf16 = (mt.flags & SF_BF16) != 0;
+                const float lr_wd = (mt.flags & SF_WD) ? P.sc.lr_wd : 0.f;
+                bool alive = true;
+
+                if (mt.kind == STAGE_PACKED) {
+                    const int L = mt.L, nb = mt.n / mt.L;
+                    if (L <= kWarpBlockMaxL) {
+                        for (int b = warp; b < nb; b += n_cwarps) {
+                            const int e = b * L;
+                            float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+                            if (bf16) sum_span<AM_BF16>(gs, e, L, lane, 32, s0, s1, s2, s3);
+                            else sum_span<AM_F32>(gs, e, L, lane, 32, s0, s1, s2, s3);
+                            const double tot = warp_sum(fold4(s0, s1, s2, s3));
+                            float v_old = lane == 0 ? mt.v[b] : 0.f;
+                            v_old = __shfl_sync(0xffffffffu, v_old, 0);
+                            float vn;
+                            const float step = stream_block_step(tot, mt.inv_L, v_old, P.sc, &vn);
+                            if (lane == 0) mt.v[b] = vn;
+                            if (bf16) apply_span<AM_BF16>(gs, ms, ps, mt.m, mt.p, e, L, lane, 32, beta1, omb1, lr_wd, step);
+                            else apply_span<AM_F32>(gs, ms, ps, mt.m, mt.p, e, L, lane, 32, beta1, omb1, lr_wd, step);
+                        }
+                    } else {
+                        for (int b = 0; b < nb && alive; ++b) {
+                            const int e = b * L;
+                            float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+                            if (bf16) sum_span<AM_BF16>(gs, e, L, ctid, nthr, s0, s1, s2, s3);
+                            else sum_span<AM_F32>(gs, e, L, ctid, nthr, s0, s1, s2, s3);
+                            double tot;
+                            float v_old;
+                            alive = group_reduce(ctl, gsync, P.error_word, ctid, n_cwarps, fold4(s0, s1, s2, s3),
+                                                 mt.v + b, &tot, &v_old);
+                            if (!alive) break;
+                            float vn;
+                            const float step = stream_block_step(tot, mt.inv_L, v_old, P.sc, &vn);
+                            if (ctid == 0) mt.v[b] = vn;
+                            if (bf16) apply_span<AM_BF16>(gs, ms, ps, mt.m, mt.p, e, L, ctid, nthr, beta1, omb1, lr_wd, step);
+                            else apply_span<AM_F32>(gs, ms, ps, mt.m, mt.p, e, L, ctid, nthr, beta1, omb1, lr_wd, step);
+                        }
+                    }
+                    if (!alive) break;
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&ctl->empty[stage]);
+                } else if (mt.kind == STAGE_SUM) {
+                    if (bf16) sum_span<AM_BF16>(gs, 0, mt.n, ctid, nthr, a0, a1, a2, a3);
+                    else sum_span<AM_F32>(gs, 0, mt.n, ctid, nthr, a0, a1, a2, a3);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&ctl->empty[stage]);
+                    if (mt.flags & SF_LAST) {
+                        double tot;
+                        float v_old;
+                        if (!group_reduce(ctl, gsync, P.error_word, ctid, n_cwarps, fold4(a0, a1, a2, a3), mt.v, &tot, &v_old))
+                            break;
+                        a0 = a1 = a2 = a3 = 0.f;
+                        if (CLUSTER) {
+                            // exchange the CTAs' sums through distributed shared memory
+                            const int slot = long_count & 1u;
+                            if (ctid == 0) {
+                                const uint32_t part = smem_addr(&ctl->xpart[slot][crank]);
+                                const uint32_t bar = smem_addr(&ctl->xbar[slot]);
+                                for (uint32_t r = 0; r < csize; ++r) {
+                                    st_cluster_f64(map_to_rank(part, r), tot);
+                                    mbar_arrive_remote(map_to_rank(bar, r));
+                                }
+                            }
+                            if (!wait_phase<true>(&ctl->xbar[slot], (long_count >> 1) & 1u, ctl, P.error_word, 4)) break;
+                            tot = 0.0;
+                            for (uint32_t r = 0; r < csize; ++r) tot += ctl->xpart[slot][r];
+                        }
+                        ++long_count;
+                        float vn;
+                        long_step = stream_block_step(tot, mt.inv_L, v_old, P.sc, &vn);
+                        if (ctid == 0 && (mt.flags & SF_WRITE_V)) *mt.v = vn;
+                    }
+                } else {   // STAGE_APPLY
+                    if (bf16) apply_span<AM_BF16>(gs, ms, ps, mt.m, mt.p, 0, mt.n, ctid, nthr, beta1, omb1, lr_wd, long_step);
+                    else apply_span<AM_F32>(gs, ms, ps, mt.m, mt.p, 0, mt.n, ctid, nthr, beta1, omb1, lr_wd, long_step);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&ctl->empty[stage]);
+                }
+                if (++stage == P.n_stages) { stage = 0; phase ^= 1u; }
+            }
+        }
+    }
+    // common exit: nobody leaves a cluster while a peer may still write into it
+    if (CLUSTER) cluster_sync_all();
+}
+
+// ------------------------------- host-side planning -------------------------------
+struct StreamPlanInput {
+    int sm_count = 0, ctas = 0, cluster_size = 0, threads = 0;
+    struct Item { int tensor; am_table_row row; };
+    std::vector<Item> stream_tensors, cluster_tensors;
+};
+
+// Which path a tensor with block length L (> 16) takes.
+inline int stream_classify(int64_t L, int32_t gdtype, bool cluster_ok) {
+    const int64_t gsz = gdtype == AM_BF16 ? 2 : 4;
+    const int64_t vec = 16 / gsz;                     // elements per 16 bytes of g
+    if (L % vec != 0) return PATH_TWOPASS;            // block starts would not be 16-byte aligned
+    if (L * gsz <= kStreamMaxBlockBytes) return PATH_STREAM;
+    if (cluster_ok && L * gsz <= kClusterMaxBlockBytes && L % (kMaxCluster * vec) == 0) return PATH_CLUSTER;
+    return PATH_TWOPASS;
+}
+
+inline void stream_add_tensor(StreamPlanInput &in, int index, const am_table_row &r, int path) {
+    (path == PATH_STREAM ? in.stream_tensors : in.cluster_tensors).push_back({index, r});
+}
+
+struct StreamLaunch {
+    std::vector<StreamSeg> segs;     // with sentinel
+    std::vector<int64_t> bounds;
+    int grid = 0, cluster = 1, n_stages = 0, stage_bytes = 0, g_region_bytes = 0, threads = 0;
+    const StreamSeg *d_segs = nullptr;
+    const int64_t *d_bounds = nullptr;
+    bool active() const { return grid > 0; }
+    size_t smem_bytes() const { return kCtrlBytes + static_cast<size_t>(n_stages) * stage_bytes; }
+};
+
+constexpr size_t kSmemBudget = 227 * 1024;
+
+struct StreamPlan {
+    StreamLaunch main, clus;
+
+    size_t table_bytes() const {
+        return (main.segs.size() + clus.segs.size()) * sizeof(StreamSeg) + 256 +
+               (main.bounds.size() + clus.bounds.size()) * sizeof(int64_t) + 256;
+    }
+    int launches() const { return (main.active() ? 1 : 0) + (clus.active() ? 1 : 0); }
+
+    cudaError_t upload(char *base) {
+        size_t off = 0;
+        for (StreamLaunch *L : {&main, &clus}) {
+            if (!L->active()) continue;
+            cudaError_t e = cudaMemcpy(base + off, L->segs.data(), L->segs.size() * sizeof(StreamSeg), cudaMemcpyHostToDevice);
+            if (e != cudaSuccess) return e;
+            L->d_segs = reinterpret_cast<const StreamSeg *>(base + off);
+            off += (L->segs.size() * sizeof(StreamSeg) + 127) / 128 * 128;
+            e = cudaMemcpy(base + off, L->bounds.data(), L->bounds.size() * sizeof(int64_t), cudaMemcpyHostToDevice);
+            if (e != cudaSuccess) return e;
+            L->d_bounds = reinterpret_cast<const int64_t *>(base + off);
+            off += (L->bounds.size() * sizeof(int64_t) + 127) / 128 * 128;
+        }
+        return cudaSuccess;
+    }
+
+    cudaError_t launch_one(const StreamLaunch &L, bool cluster, const DevTensor *tensors, float *v,
+                           const StepScalars &sc, int *error_word, cudaStream_t stream) const {
+        StreamParams P;
+        P.tensors = tensors; P.segs = L.d_segs; P.bounds = L.d_bounds; P.v = v; P.error_word = error_word;
+        P.sc = sc; P.n_segs = static_cast<int>(L.segs.size()) - 1; P.n_stages = L.n_stages;
+        P.stage_bytes = L.stage_bytes; P.g_region_bytes = L.g_region_bytes; P.consumer_threads = L.threads;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(L.grid);
+        cfg.blockDim = dim3(32 + L.threads);
+        cfg.dynamicSmemBytes = L.smem_bytes();
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        if (cluster) {
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = L.cluster;
+            attr[0].val.clusterDim.y = 1;
+            attr[0].val.clusterDim.z = 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+            return cudaLaunchKernelEx(&cfg, stream_kernel<true>, P);
+        }
+        return cudaLaunchKernelEx(&cfg, stream_kernel<false>, P);
+    }
+
+    cudaError_t launch(const DevTensor *tensors, float *v, const StepScalars &sc, int *error_word,
+                       cudaStream_t stream) const {
+        if (main.active()) {
+            cudaError_t e = launch_one(main, false, tensors, v, sc, error_word, stream);
+            if (e != cudaSuccess) return e;
+        }
+        if (clus.active()) {
+            cudaError_t e = launch_one(clus, true, tensors, v, sc, error_word, stream);
+            if (e != cudaSuccess) return e;
+        }
+        return cudaSuccess;
+    }
+};
+
+// Build segment tables and balanced item ranges for one launch.
+inline void stream_build_launch(const std::vector<StreamPlanInput::Item> &tensors, bool cluster, int workers,
+                                StreamLaunch *out) {
+    out->segs.clear();
+    out->bounds.clear();
+    out->grid = 0;
+    if (tensors.empty() || workers <= 0) return;
+    bool any_f32 = false;
+    for (const auto &it : tensors) any_f32 |= it.row.grad_dtype == AM_F32;
+    out->g_region_bytes = kStageElems * (any_f32 ? 4 : 2);
+    out->stage_bytes = out->g_region_bytes + kStageElems * 8;
+    out->n_stages = std::min<int>(kMaxStages, static_cast<int>((kSmemBudget - kCtrlBytes) / out->stage_bytes));
+
+    std::vector<double> item_cost;      // per segment
+    int64_t items = 0;
+    for (const auto &it : tensors) {
+        const am_table_row &r = it.row;
+        const double gsz = r.grad_dtype == AM_BF16 ? 2 : 4;
+        StreamSeg s;
+        s.item_begin = items;
+        s.tensor = it.tensor;
+        if (!cluster && r.block_len <= kStageElems) {
+            s.bpi = static_cast<int32_t>(kStageElems / r.block_len);
+            items += (r.n_blocks + s.bpi - 1) / s.bpi;
+            item_cost.push_back(static_cast<double>(s.bpi) * r.block_len * (gsz + 16));
+        } else {
+            s.bpi = 0;
+            items += r.n_blocks;
+            item_cost.push_back(static_cast<double>(r.block_len) * (2 * gsz + 16));
+        }
+        out->segs.push_back(s);
+    }
+    StreamSeg sentinel;
+    sentinel.item_begin = items;
+    sentinel.tensor = -1;
+    sentinel.bpi = 0;
+    out->segs.push_back(sentinel);
+
+    // contiguous item ranges of (nearly) equal cost
+    double total = 0.0;
+    for (size_t k = 0; k + 1 < out->segs.size(); ++k)
+        total += item_cost[k] * static_cast<double>(out->segs[k + 1].item_begin - out->segs[k].item_begin);
+    workers = static_cast<int>(std::min<int64_t>(workers, items));
+    out->bounds.assign(workers + 1, 0);
+    out->bounds[workers] = items;
+    size_t k = 0;
+    double before = 0.0;                // cost of the segments before k
+    for (int w = 1; w < workers; ++w) {
+        const double target = total * w / workers;
+        for (;;) {
+            const double seg_cost = item_cost[k] * static_cast<double>(out->segs[k + 1].item_begin - out->segs[k].item_begin);
+            if (before + seg_cost >= target || k + 2 >= out->segs.size()) break;
+            before += seg_cost;
+            ++k;
+        }
+        int64_t idx = out->segs[k].item_begin + static_cast<int64_t>((target - before) / item_cost[k] + 0.5);
+        idx = std::max(idx, out->bounds[w - 1]);
+        idx = std::min(idx, items);
+        out->bounds[w] = idx;
+    }
+    out->grid = workers;
+}
+
+// Largest cluster size (<= wanted) the device can keep resident with this
+// kernel's shared memory, and how many such clusters fit at once.
+inline void stream_probe_cluster(int sm_count, int threads, int wanted, int *cluster_size, int *n_clusters) {
+    *cluster_size = 0;
+    *n_clusters = 0;
+    if (threads <= 0) threads = 256;
+    const size_t smem = kCtrlBytes + 5 * (kStageElems * 10);   // the larger of the two stage layouts
+    for (int cs = wanted > 0 ? wanted : kMaxCluster; cs >= 1; cs >>= 1) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(std::max(sm_count / cs, 1) * cs);
+        cfg.blockDim = dim3(32 + threads);
+        cfg.dynamicSmemBytes = smem;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = cs;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, stream_kernel<true>, &cfg) == cudaSuccess && n > 0) {
+            *cluster_size = cs;
+            *n_clusters = n;
+            return;
+        }
+        (void)cudaGetLastError();
+    }
+}
+
+inline void stream_finish_plan(const StreamPlanInput &in, int cluster_size, int n_clusters, StreamPlan *plan) {
+    const int threads = in.threads > 0 ? in.threads : 256;
+    const int ctas = in.ctas > 0 ? in.ctas : in.sm_count;
+    stream_build_launch(in.stream_tensors, false, ctas, &plan->main);
+    plan->main.threads = threads;
+    plan->main.cluster = 1;
+    plan->clus = StreamLaunch();
+    if (!in.cluster_tensors.empty() && n_clusters > 0) {
+        stream_build_launch(in.cluster_tensors, true, n_clusters, &plan->clus);
+        plan->clus.grid *= cluster_size;          // bounds are per cluster
+        plan->clus.cluster = cluster_size;
+        plan->clus.threads = threads;
+    }
+}
+
+inline cudaError_t stream_configure_kernels() {
+    cudaError_t e = cudaFuncSetAttribute(stream_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(kSmemBudget));
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(stream_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                static_cast<int>(kSmemBudget));
+}
+
+}  // namespace am
+
+#endif  // ADAMMINI_KERNELS_STREAM_CUH_
