@@ -1,0 +1,8 @@
+"""B200-native Adam-mini optimizer step (arxiv 2406.16793, Algorithm 1).
+
+binding    ctypes front end of the CUDA library (libadammini.so, C ABI in include/adammini.h)
+workloads  model-shaped tensor lists and seeded synthetic inputs
+build      in-tree nvcc build of the library for sm_100a
+"""
+from . import binding, workloads  # noqa: F401
+from .binding import AdamMini, AdamMiniError, Partition  # noqa: F401

@@ -1,0 +1,178 @@
+"""Shared test machinery: run a workload through the CUDA library and through
+the float64 oracle on the same seeded inputs, and compare.
+
+The comparison follows the acceptance rule for this library: for p and m the
+error of element i is |gpu_i - oracle_i| / max(|oracle_i|, rms of the oracle's
+values over i's block); for v it is the plain relative error with an absolute
+floor.  The bound is 1e-5 (float32 arithmetic against float64; rounding errors
+add up but do not feed back because the synthetic gradients do not depend on
+the parameters).
+"""
+from __future__ import annotations
+
+import concurrent.futures as cf
+import os
+from typing import Dict, List, Optional, Sequence
+
+import numpy as np
+import torch
+
+import paper_2406_16793_b200 as am
+from oracle import step as ostep
+from paper_2406_16793_b200 import workloads as W
+
+TOL = 1e-5
+GUARD = 64          # float32 guard words either side of every test buffer
+SENTINEL = -7.0e33
+
+
+def block_relative_error(got: np.ndarray, want: np.ndarray, L: int) -> float:
+    """max_i |got-want| / max(|want_i|, rms(want over i's block)); NaN/inf must match."""
+    got = np.asarray(got, dtype=np.float64).reshape(-1, L)
+    want = np.asarray(want, dtype=np.float64).reshape(-1, L)
+    fin = np.isfinite(want)
+    if not np.array_equal(fin, np.isfinite(got)):
+        return float("inf")
+    if not fin.all():
+        same = np.where(fin, True, (np.isnan(want) & np.isnan(got)) | (want == got))
+        if not same.all():
+            return float("inf")
+    w = np.where(fin, want, 0.0)
+    rms = np.sqrt((w * w).mean(axis=1, keepdims=True))
+    scale = np.maximum(np.abs(w), rms)
+    scale = np.where(scale > 0, scale, 1.0)
+    err = np.where(fin, np.abs(got - w) / scale, 0.0)
+    return float(err.max()) if err.size else 0.0
+
+
+def v_relative_error(got: np.ndarray, want: np.ndarray) -> float:
+    got = np.asarray(got, dtype=np.float64)
+    want = np.asarray(want, dtype=np.float64)
+    fin = np.isfinite(want)
+    if not np.array_equal(fin, np.isfinite(got)):
+        return float("inf")
+    d = np.abs(got - want)[fin]
+    return float((d / np.maximum(np.abs(want[fin]), 1e-30)).max()) if d.size else 0.0
+
+
+class Guarded:
+    """A device tensor with sentinel-filled guard zones before and after it."""
+
+    def __init__(self, numel: int, dtype: torch.dtype, device):
+        item = torch.empty((), dtype=dtype).element_size()
+        self.guard = GUARD * 4 // item
+        pad = (-numel) % (16 // item)          # keep the rear guard 16-byte aligned too
+        self.raw = torch.full((numel + pad + 2 * self.guard,), SENTINEL, dtype=dtype, device=device)
+        self.view = self.raw[self.guard:self.guard + numel]
+        self.numel = numel
+
+    def intact(self) -> bool:
+        front = self.raw[:self.guard]
+        back = self.raw[self.guard + self.numel:]
+        ref = torch.full((1,), SENTINEL, dtype=self.raw.dtype, device=self.raw.device)
+        return bool((front == ref).all() and (back == ref).all())
+
+
+class DeviceState:
+    """Parameters, moments and gradient buffers of a workload on the GPU."""
+
+    def __init__(self, w: W.Workload, device="cuda", guarded: bool = True):
+        self.w = w
+        self.device = device
+        self.guards: List[Guarded] = []
+
+        def alloc(n, dtype):
+            if guarded:
+                g = Guarded(n, dtype, device)
+                self.guards.append(g)
+                return g.view
+            return torch.empty(n, dtype=dtype, device=device)
+
+        self.p, self.m, self.g = [], [], []
+        for i, t in enumerate(w.tensors):
+            p = alloc(t.numel, torch.float32)
+            p.copy_(W.gen_param(w, i, device))
+            m = alloc(t.numel, torch.float32)
+            m.zero_()
+            g = alloc(t.numel, W.torch_dtype(t.grad_dtype))
+            g.zero_()
+            self.p.append(p); self.m.append(m); self.g.append(g)
+        self.v = alloc(max(w.n_blocks, 1), torch.float32)
+        self.v.zero_()
+        self.sigmas = [W.row_sigmas(w, i, device) for i in range(len(w.tensors))]
+
+    def draw_grads(self, step: int) -> None:
+        for i in range(len(self.w.tensors)):
+            W.gen_grad(self.w, i, step, self.device, out=self.g[i], sigmas=self.sigmas[i])
+
+    def guards_intact(self) -> bool:
+        return all(g.intact() for g in self.guards)
+
+
+def make_optimizer(w: W.Workload, options: Optional[Dict[int, int]] = None, **hp) -> am.AdamMini:
+    part = am.Partition(w.tensors)
+    opt = am.AdamMini(part, **{**w.hparams, **hp})
+    for k, val in (options or {}).items():
+        opt.set_option(k, val)
+    return opt
+
+
+def oracle_step_all(state: ostep.OracleState, grads_cpu: Sequence, step: int, hp: Dict[str, float],
+                    pool: Optional[cf.ThreadPoolExecutor] = None) -> None:
+    """One oracle step over all tensors; tensors are independent, so they may
+    run on several host threads (each call is the single-threaded C routine)."""
+    def one(i):
+        ostep.adammini_step(state.p[i], state.m[i], state.v[i], grads_cpu[i], state.block_lens[i],
+                            step=step, apply_wd=state.wd_flags[i], **hp)
+    if pool is None:
+        for i in range(len(grads_cpu)):
+            one(i)
+    else:
+        list(pool.map(one, range(len(grads_cpu))))
+
+
+def run_parity(w: W.Workload, steps: Optional[int] = None, options: Optional[Dict[int, int]] = None,
+               device="cuda", hp_override: Optional[Dict[str, float]] = None, mutate_grads=None,
+               lr_schedule=None) -> Dict[str, float]:
+    """Run `steps` steps on the GPU and in the oracle; returns the worst errors.
+
+    mutate_grads(step, list_of_device_grads) may edit the gradients in place
+    (zero rows, infinities) before both sides consume them.
+    """
+    steps = steps or w.steps
+    hp = {**w.hparams, **(hp_override or {})}
+    dev = DeviceState(w, device)
+    opt = make_optimizer(w, options, **(hp_override or {}))
+    ora = ostep.OracleState([p.cpu() for p in dev.p], [t.block_len for t in w.tensors],
+                            [bool(t.apply_weight_decay) for t in w.tensors])
+    pool = cf.ThreadPoolExecutor(max_workers=min(16, os.cpu_count() or 1))
+    try:
+        for t in range(1, steps + 1):
+            dev.draw_grads(t)
+            if mutate_grads is not None:
+                mutate_grads(t, dev.g)
+            hp_t = dict(hp)
+            if lr_schedule is not None:
+                hp_t["lr"] = lr_schedule(t)
+                opt.set_lr(hp_t["lr"])
+            opt.step(dev.p, dev.g, dev.m, dev.v, t)
+            grads_cpu = [g.cpu() for g in dev.g]
+            oracle_step_all(ora, grads_cpu, t, hp_t, pool)
+        opt.sync_status()
+    finally:
+        pool.shutdown()
+    assert dev.guards_intact(), "a kernel wrote outside its buffers"
+    worst = {"p": 0.0, "m": 0.0, "v": 0.0}
+    v_gpu = dev.v.cpu().numpy()
+    off = 0
+    for i, t in enumerate(w.tensors):
+        worst["p"] = max(worst["p"], block_relative_error(dev.p[i].cpu().numpy(), ora.p[i], t.block_len))
+        worst["m"] = max(worst["m"], block_relative_error(dev.m[i].cpu().numpy(), ora.m[i], t.block_len))
+        worst["v"] = max(worst["v"], v_relative_error(v_gpu[off:off + t.n_blocks], ora.v[i]))
+        off += t.n_blocks
+    opt.close()
+    return worst
+
+
+def assert_parity(worst: Dict[str, float], tol: float = TOL) -> None:
+    assert worst["p"] <= tol and worst["m"] <= tol and worst["v"] <= tol, worst

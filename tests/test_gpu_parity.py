@@ -1,0 +1,199 @@
+"""GPU parity: the CUDA library against the float64 oracle, element by element,
+on the same seeded inputs, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import harness as H
+import paper_2406_16793_b200 as am
+from paper_2406_16793_b200 import binding as B, workloads as W
+
+pytestmark = pytest.mark.gpu
+
+TWOPASS = {B.OPT_PATH: 1}
+
+
+def test_tiny_gpt2_ten_steps():
+    """2-layer GPT-2-style model, fp32 gradients, 10 steps."""
+    H.assert_parity(H.run_parity(W.tiny_gpt2()))
+
+
+def test_tiny_gpt2_two_pass_anchor():
+    H.assert_parity(H.run_parity(W.tiny_gpt2(), options=TWOPASS))
+
+
+def test_gpt2_small_hundred_steps():
+    """GPT-2-small shapes (two layers, vocabulary rows cut to 4096), bf16 gradients, 100 steps."""
+    w = W.scaled_rows(W.gpt2_small(n_layers=2), 4096)
+    H.assert_parity(H.run_parity(w, steps=100))
+
+
+def test_llama2_block_lengths():
+    """Every block length of Llama-2-7B (4096, 11008, 524288-element heads), rows cut to 256."""
+    w = W.scaled_rows(W.llama2_7b(n_layers=1), 256)
+    H.assert_parity(H.run_parity(w))
+
+
+def test_llama3_gqa_block_lengths():
+    """Llama-3-8B shapes with grouped KV heads and Zipf row magnitudes, rows cut to 384."""
+    w = W.scaled_rows(W.llama3_8b(n_layers=1), 384)
+    H.assert_parity(H.run_parity(w))
+
+
+@pytest.mark.parametrize("L", [1, 128, 4096, 524288, 1 << 22])
+def test_flat_partition_sweep(L):
+    """One flat fp32 tensor of 2^22 elements cut into blocks of every degenerate length."""
+    H.assert_parity(H.run_parity(W.flat_sweep(L, numel=1 << 22)))
+
+
+@pytest.mark.parametrize("L", [1, 128, 4096])
+def test_flat_sweep_two_pass_anchor(L):
+    H.assert_parity(H.run_parity(W.flat_sweep(L, numel=1 << 20), options=TWOPASS))
+
+
+def ragged_workload(grad_dtype):
+    """Block lengths that exercise every path and tail: tiny, unaligned, packed
+    with a ragged last stage, long single-CTA rows with a ragged last chunk."""
+    T = W.TensorSpec
+    gd = dict(grad_dtype=grad_dtype)
+    tensors = [
+        T("l1", 1, 1027, W.FIXED, fixed_block_len=1, **gd),
+        T("l3", 7, 3, W.ROWS, **gd),
+        T("l16", 129, 16, W.ROWS, **gd),
+        T("l17", 33, 17, W.ROWS, **gd),
+        T("l24", 1025, 24, W.ROWS, **gd),
+        T("l36", 77, 36, W.ROWS, **gd),
+        T("l40", 1031, 40, W.ROWS, **gd),
+        T("l1000", 13, 1000, W.ROWS, **gd),
+        T("l1001", 5, 1001, W.ROWS, **gd),
+        T("l1032", 9, 1032, W.ROWS, **gd),
+        T("l2056", 7, 2056, W.ROWS, **gd),
+        T("l4104", 5, 4104, W.ROWS, **gd),
+        T("l20488", 3, 20488, W.ROWS, **gd),
+        T("whole50000", 1, 50000, W.WHOLE, **gd),
+        T("whole70001", 1, 70001, W.WHOLE, **gd),
+        T("heads", 12, 1000, W.HEADS, n_heads=4, **gd),
+        T("nowd", 64, 256, W.ROWS, apply_weight_decay=0, **gd),
+        T("one", 1, 1, W.WHOLE, **gd),
+    ]
+    return W.Workload("ragged", 90 + grad_dtype, tensors, W.GradRecipe(-4.0, -1.0), steps=6)
+
+
+@pytest.mark.parametrize("grad_dtype", [W.F32, W.BF16], ids=["f32", "bf16"])
+@pytest.mark.parametrize("options", [None, TWOPASS], ids=["auto", "twopass"])
+def test_ragged_shapes(grad_dtype, options):
+    H.assert_parity(H.run_parity(ragged_workload(grad_dtype), options=options))
+
+
+@pytest.mark.parametrize("threads", [128, 512])
+def test_other_consumer_thread_counts(threads):
+    w = W.scaled_rows(W.llama2_7b(n_layers=1), 128)
+    H.assert_parity(H.run_parity(w, steps=3, options={B.OPT_STREAM_THREADS: threads}))
+
+
+@pytest.mark.parametrize("cluster", [1, 2, 4])
+def test_other_cluster_sizes(cluster):
+    w = W.Workload("heads", 77, [W.TensorSpec("q", 1024, 4096, W.HEADS, n_heads=8, grad_dtype=W.BF16)],
+                   W.GradRecipe(-5.0, -1.0), steps=3)
+    H.assert_parity(H.run_parity(w, options={B.OPT_CLUSTER_SIZE: cluster}))
+
+
+def test_zero_gradient_rows_and_an_infinity():
+    """Rows with all-zero gradients keep v = 0 and take no Adam step; an
+    infinite gradient propagates exactly as in the oracle."""
+    w = W.scaled_rows(W.llama2_7b(n_layers=1, vocab=512), 64)
+
+    def mutate(step, grads):
+        grads[0].view(-1, 4096)[3:9].zero_()          # embedding rows of unseen tokens
+        grads[4].view(-1, 4096)[5].zero_()
+        if step == 2:
+            grads[5].view(-1)[12345] = float("inf")
+
+    H.assert_parity(H.run_parity(w, steps=4, mutate_grads=mutate))
+
+
+def test_learning_rate_schedule():
+    sched = lambda t: 1e-3 * min(1.0, t / 3.0) * (0.9 ** t)
+    H.assert_parity(H.run_parity(W.tiny_gpt2(), steps=8, lr_schedule=sched))
+
+
+def test_other_hyperparameters():
+    H.assert_parity(H.run_parity(W.tiny_gpt2(), steps=5,
+                                 hp_override=dict(lr=3e-4, beta1=0.8, beta2=0.999, eps=1e-6, weight_decay=0.0)))
+
+
+def _run_steps(w, first, last, state=None, stream=None):
+    dev = state or H.DeviceState(w, guarded=False)
+    opt = H.make_optimizer(w)
+    for t in range(first, last + 1):
+        dev.draw_grads(t)
+        if stream is None:
+            opt.step(dev.p, dev.g, dev.m, dev.v, t)
+        else:
+            stream.wait_stream(torch.cuda.current_stream())
+            opt.step(dev.p, dev.g, dev.m, dev.v, t, stream=stream.cuda_stream)
+            torch.cuda.current_stream().wait_stream(stream)
+    opt.sync_status(stream.cuda_stream if stream is not None else 0)
+    opt.close()
+    return dev
+
+
+def _same(a, b):
+    return all(torch.equal(x, y) for x, y in zip(a.p + a.m + [a.v], b.p + b.m + [b.v]))
+
+
+def test_deterministic_and_resumable():
+    """Two runs give identical bits; 10 steps equal 5 steps, a new handle, 5 more
+    (the state is only p, m, v and the step number)."""
+    w = W.scaled_rows(W.llama2_7b(n_layers=1, vocab=256), 128)
+    a = _run_steps(w, 1, 10)
+    b = _run_steps(w, 1, 10)
+    assert _same(a, b)
+    c = _run_steps(w, 1, 5)
+    c = _run_steps(w, 6, 10, state=c)
+    assert _same(a, c)
+
+
+def test_runs_on_a_side_stream():
+    w = W.tiny_gpt2()
+    a = _run_steps(w, 1, 3)
+    b = _run_steps(w, 1, 3, stream=torch.cuda.Stream())
+    assert _same(a, b)
+
+
+def test_argument_errors():
+    w = W.tiny_gpt2()
+    dev = H.DeviceState(w, guarded=False)
+    opt = H.make_optimizer(w)
+    with pytest.raises(am.AdamMiniError) as e:
+        opt.step(dev.p, dev.g, dev.m, dev.v, 0)
+    assert e.value.status == -1
+    bad = list(dev.p)
+    bad[3] = dev.p[3][1:]                                  # 4-byte offset: not 16-byte aligned
+    with pytest.raises(am.AdamMiniError) as e:
+        opt.step(bad, dev.g, dev.m, dev.v, 1)
+    assert e.value.status == -3
+    nul = [t.data_ptr() for t in dev.m]
+    nul[0] = 0
+    with pytest.raises(am.AdamMiniError) as e:
+        opt.step(dev.p, dev.g, nul, dev.v, 1)
+    assert e.value.status == -1
+    for kw in (dict(eps=0.0), dict(beta1=1.0), dict(beta2=-0.1), dict(lr=-1.0), dict(weight_decay=float("nan"))):
+        with pytest.raises(am.AdamMiniError):
+            am.AdamMini(am.Partition(w.tensors), **kw)
+    opt.close()
+
+
+def test_empty_partition_and_queries():
+    opt = am.AdamMini(am.Partition([]))
+    opt.step([], [], [], 0, 1)
+    opt.close()
+    w = W.scaled_rows(W.llama2_7b(n_layers=1, vocab=256), 128)
+    opt = H.make_optimizer(w)
+    n = opt.query(B.Q_TOTAL_ELEMENTS)
+    assert n == w.numel and opt.query(B.Q_TOTAL_BLOCKS) == w.n_blocks
+    assert opt.query(B.Q_ELEMENTS_STREAM) + opt.query(B.Q_ELEMENTS_CLUSTER) == n
+    assert opt.query(B.Q_ELEMENTS_CLUSTER) == 2 * 128 * 4096
+    assert opt.query(B.Q_LAUNCHES_PER_STEP) == 2
+    assert opt.query(B.Q_ALGORITHMIC_BYTES) == 18 * n + 8 * w.n_blocks
+    opt.close()

@@ -1,0 +1,83 @@
+"""Host-side checks of the CUDA library that need no GPU: the shared object
+loads, exports every entry point the header declares, and its partitioner
+produces bit-exactly the table the Python partition rules give."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import paper_2406_16793_b200 as am
+from oracle import partition_ref as pr
+from paper_2406_16793_b200 import binding, build, workloads as W
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    build.build()
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "adammini.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(adammini_\w+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_entry_point():
+    names = declared_functions()
+    assert len(names) >= 16
+    lib = ctypes.CDLL(binding.LIBRARY)
+    for n in names:
+        assert hasattr(lib, n), n
+    assert set(binding.exported_names()) == set(names)
+
+
+def workloads():
+    return [W.tiny_gpt2(), W.gpt2_small(), W.llama2_7b(), W.llama3_8b()] + \
+           [W.flat_sweep(L) for L in (1, 128, 4096, 524288, 1 << 30)]
+
+
+@pytest.mark.parametrize("w", workloads(), ids=lambda w: w.name)
+def test_partition_table_is_bit_exact(w):
+    part = am.Partition(w.tensors)
+    rows, total = part.export()
+    want, want_total = pr.build_table([
+        pr.TensorDesc(t.rows, t.cols, t.kind, t.n_heads, t.fixed_block_len, t.grad_dtype, t.apply_weight_decay)
+        for t in w.tensors])
+    assert total == want_total and len(rows) == len(want)
+    for got, ref in zip(rows, want):
+        assert (got.numel, got.block_len, got.n_blocks, got.v_offset, got.kind, got.grad_dtype, got.wd) == \
+               (ref.numel, ref.block_len, ref.n_blocks, ref.v_offset, ref.kind, ref.grad_dtype, ref.wd)
+    part.close()
+
+
+def test_name_rule_matches_algorithm3():
+    names = ["embed_tokens.weight", "output.weight", "layers.0.attention.query.weight", "h.1.attn.key.weight",
+             "h.1.attn.value.weight", "h.3.attn.proj.weight", "h.3.mlp.fc.weight", "ln_f.weight",
+             "output_embed_query", "mlp.query", "norm"]
+    for n in names:
+        assert binding.kind_from_name(n) == pr.kind_from_name(n), n
+
+
+def test_partition_rejects_bad_descriptors():
+    bad = [
+        W.TensorSpec("heads", 10, 4, W.HEADS, n_heads=3),
+        W.TensorSpec("fixed", 1, 10, W.FIXED, fixed_block_len=4),
+        W.TensorSpec("empty", 0, 4, W.ROWS),
+    ]
+    for t in bad:
+        with pytest.raises(am.AdamMiniError) as e:
+            am.Partition([t])
+        assert e.value.status == -2
+    with pytest.raises(am.AdamMiniError) as e:
+        am.Partition([W.TensorSpec("dtype", 2, 2, W.ROWS, grad_dtype=7)])
+    assert e.value.status == -1
+
+
+def test_status_strings():
+    lib = binding.load()
+    seen = {lib.adammini_status_string(s).decode() for s in range(-7, 1)}
+    assert len(seen) == 8 and "unknown status" not in seen
+    assert lib.adammini_status_string(-99).decode() == "unknown status"
