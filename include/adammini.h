@@ -154,7 +154,9 @@ typedef enum {
                                  tensor with block_len > 16 (correctness anchor) */
     AM_OPT_STREAM_CTAS   = 1, /* persistent CTAs of the streaming kernel (0 = one per SM) */
     AM_OPT_CLUSTER_SIZE  = 2, /* CTAs per cluster for head-sized blocks (0 = default) */
-    AM_OPT_STREAM_THREADS = 3 /* consumer threads per CTA of the streaming kernels (0 = default) */
+    AM_OPT_STREAM_THREADS = 3, /* consumer threads per CTA of the streaming kernels (0 = default) */
+    AM_OPT_PROFILE       = 4  /* 1: record CUDA events around each kernel family of every step
+                                 (read them with adammini_get_profile) */
 } am_option;
 int adammini_set_option(am_handle *h, int32_t key, int64_t value);
 
@@ -167,10 +169,22 @@ typedef enum {
     AM_Q_ELEMENTS_STREAM   = 5, /* ... to the single-launch streaming kernel */
     AM_Q_ELEMENTS_CLUSTER  = 6, /* ... to the cluster kernel (head-sized blocks) */
     AM_Q_ELEMENTS_TWOPASS  = 7, /* ... to the two-pass path (blocks beyond on-chip/L2 reach, or unaligned) */
-    AM_Q_ALGORITHMIC_BYTES = 8  /* bytes one step must move: per tensor g once (twice on the two-pass
-                                   path), m and p read+written, v read+written */
+    AM_Q_ALGORITHMIC_BYTES = 8, /* bytes one step must move: per tensor g once (twice for blocks beyond
+                                   on-chip/L2 reach), m and p read+written, v read+written */
+    AM_Q_BYTES_SMALL       = 9, /* the same, split by the kernel family that handles the tensor */
+    AM_Q_BYTES_STREAM      = 10,
+    AM_Q_BYTES_CLUSTER     = 11,
+    AM_Q_BYTES_TWOPASS     = 12,
+    AM_Q_STREAM_CTAS       = 13, /* launch shape of the streaming kernel */
+    AM_Q_CLUSTER_SIZE      = 14,
+    AM_Q_CLUSTER_COUNT     = 15
 } am_query;
 int adammini_query(const am_handle *h, int32_t what, int64_t *value);
+
+/* With AM_OPT_PROFILE set: waits for the last step and writes the device time in
+ * milliseconds of its kernel families to ms[0..3] (host array): thread-per-block
+ * kernel, streaming kernel, cluster kernel, two-pass kernels (0 where none ran). */
+int adammini_get_profile(am_handle *h, float *ms);
 
 /* The CUDA error code (cudaError_t as int) of the last AM_ERR_CUDA on this handle. */
 int adammini_last_cuda_error(const am_handle *h);

@@ -17,9 +17,10 @@ LIBRARY = os.path.join(_HERE, "libadammini.so")
 WHOLE, ROWS, HEADS, TOKENS, FIXED = 0, 1, 2, 3, 4
 F32, BF16 = 0, 1
 
-OPT_PATH, OPT_STREAM_CTAS, OPT_CLUSTER_SIZE, OPT_STREAM_THREADS = 0, 1, 2, 3
+OPT_PATH, OPT_STREAM_CTAS, OPT_CLUSTER_SIZE, OPT_STREAM_THREADS, OPT_PROFILE = 0, 1, 2, 3, 4
 (Q_LAUNCHES_PER_STEP, Q_SCRATCH_BYTES, Q_TOTAL_BLOCKS, Q_TOTAL_ELEMENTS, Q_ELEMENTS_SMALL,
- Q_ELEMENTS_STREAM, Q_ELEMENTS_CLUSTER, Q_ELEMENTS_TWOPASS, Q_ALGORITHMIC_BYTES) = range(9)
+ Q_ELEMENTS_STREAM, Q_ELEMENTS_CLUSTER, Q_ELEMENTS_TWOPASS, Q_ALGORITHMIC_BYTES, Q_BYTES_SMALL,
+ Q_BYTES_STREAM, Q_BYTES_CLUSTER, Q_BYTES_TWOPASS, Q_STREAM_CTAS, Q_CLUSTER_SIZE, Q_CLUSTER_COUNT) = range(16)
 
 
 class TensorDesc(ctypes.Structure):
@@ -63,6 +64,7 @@ _SIGNATURES = {
     "adammini_sync_status": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p]),
     "adammini_set_option": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64]),
     "adammini_query": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.POINTER(ctypes.c_int64)]),
+    "adammini_get_profile": (ctypes.c_int, [ctypes.c_void_p, ctypes.POINTER(ctypes.c_float)]),
     "adammini_last_cuda_error": (ctypes.c_int, [ctypes.c_void_p]),
     "adammini_destroy": (ctypes.c_int, [ctypes.c_void_p]),
     "adammini_status_string": (ctypes.c_char_p, [ctypes.c_int]),
@@ -207,6 +209,13 @@ class AdamMini:
         pa, ga, ma = _ptr_array(_data_ptrs(params)), _ptr_array(_data_ptrs(grads)), _ptr_array(_data_ptrs(m))
         vp = int(v.data_ptr()) if hasattr(v, "data_ptr") else int(v)
         _check(load().adammini_step_host(self._h, pa, ga, ma, vp, int(step), int(staging_bytes)), self._h)
+
+    def get_profile(self):
+        """Device milliseconds of the last step's kernel families (needs
+        OPT_PROFILE): [thread-per-block, streaming, cluster, two-pass]."""
+        ms = (ctypes.c_float * 4)()
+        _check(load().adammini_get_profile(self._h, ms), self._h)
+        return [float(x) for x in ms]
 
     def sync_status(self, stream: int = 0) -> None:
         """Wait for the stream; raises if a device-side bounded wait gave up."""

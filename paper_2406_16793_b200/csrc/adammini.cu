@@ -20,7 +20,7 @@ using namespace am;
 
 namespace {
 
-constexpr int kNumOptions = 4;
+constexpr int kNumOptions = 5;
 
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
@@ -65,7 +65,7 @@ int build_plan(am_handle *h) {
     h->host_tensors.assign(n, DevTensor{});
     std::vector<Seg> small_segs, piece_segs, block_segs;
     int64_t small_units = 0, piece_units = 0, block_units = 0;
-    for (int k = 0; k < 4; ++k) h->elems_by_path[k] = 0;
+    for (int k = 0; k < 4; ++k) h->elems_by_path[k] = h->bytes_by_path[k] = 0;
     h->algorithmic_bytes = 0;
 
     StreamPlanInput sin;
@@ -97,7 +97,9 @@ int build_plan(am_handle *h) {
         // bytes the update must move: g once if a block can stay on chip / in
         // L2 between its reduction and its update, twice otherwise
         const int64_t g_reads = r.block_len * gsz > kClusterMaxBlockBytes ? 2 : 1;
-        h->algorithmic_bytes += r.numel * (g_reads * gsz + 16) + r.n_blocks * 8;
+        const int64_t tensor_bytes = r.numel * (g_reads * gsz + 16) + r.n_blocks * 8;
+        h->algorithmic_bytes += tensor_bytes;
+        h->bytes_by_path[path] += tensor_bytes;
 
         if (path == PATH_SMALL) {
             Seg s;
@@ -276,7 +278,14 @@ int adammini_set_hparams(am_handle *h, const am_hparams *hp) {
 
 int adammini_set_option(am_handle *h, int32_t key, int64_t value) {
     if (!h || key < 0 || key >= kNumOptions || value < 0) return AM_ERR_INVALID_ARGUMENT;
-    if (key == AM_OPT_PATH && value > 1) return AM_ERR_INVALID_ARGUMENT;
+    if ((key == AM_OPT_PATH || key == AM_OPT_PROFILE) && value > 1) return AM_ERR_INVALID_ARGUMENT;
+    if (key == AM_OPT_PROFILE) {
+        if (value && !h->prof_ev[0])
+            for (int k = 0; k < 5; ++k) AM_CUDA(h, cudaEventCreate(&h->prof_ev[k]));
+        h->opt[key] = value;
+        h->prof_recorded = false;
+        return AM_OK;
+    }
     if (key == AM_OPT_CLUSTER_SIZE && value != 0 && value != 1 && value != 2 && value != 4 && value != 8)
         return AM_ERR_INVALID_ARGUMENT;
     if (key == AM_OPT_STREAM_THREADS && value != 0 && (value % 32 != 0 || value < 64 || value > 512))
@@ -305,6 +314,13 @@ int adammini_query(const am_handle *h, int32_t what, int64_t *value) {
     case AM_Q_ELEMENTS_CLUSTER: *value = h->elems_by_path[PATH_CLUSTER]; break;
     case AM_Q_ELEMENTS_TWOPASS: *value = h->elems_by_path[PATH_TWOPASS]; break;
     case AM_Q_ALGORITHMIC_BYTES: *value = h->algorithmic_bytes; break;
+    case AM_Q_BYTES_SMALL: *value = h->bytes_by_path[PATH_SMALL]; break;
+    case AM_Q_BYTES_STREAM: *value = h->bytes_by_path[PATH_STREAM]; break;
+    case AM_Q_BYTES_CLUSTER: *value = h->bytes_by_path[PATH_CLUSTER]; break;
+    case AM_Q_BYTES_TWOPASS: *value = h->bytes_by_path[PATH_TWOPASS]; break;
+    case AM_Q_STREAM_CTAS: *value = h->stream.main.grid; break;
+    case AM_Q_CLUSTER_SIZE: *value = h->stream.clus.active() ? h->stream.clus.cluster : 0; break;
+    case AM_Q_CLUSTER_COUNT: *value = h->stream.clus.active() ? h->stream.clus.grid / h->stream.clus.cluster : 0; break;
     default: return AM_ERR_INVALID_ARGUMENT;
     }
     return AM_OK;
@@ -347,6 +363,8 @@ int adammini_step(am_handle *h, void *const *params, const void *const *grads, v
     sc.lr_wd = static_cast<float>(hp.lr * hp.weight_decay);
     sc.pad = 0.f;
 
+    const bool prof = h->opt[AM_OPT_PROFILE] != 0;
+    if (prof) AM_CUDA(h, cudaEventRecord(h->prof_ev[0], stream));
     if (h->small_units) {
         SmallScalars ss;
         ss.beta1 = sc.beta1;
@@ -361,10 +379,11 @@ int adammini_step(am_handle *h, void *const *params, const void *const *grads, v
             h->d_tensors, h->d_small_segs, h->n_small_segs, v, ss);
         AM_CUDA(h, cudaGetLastError());
     }
-    {
-        cudaError_t e = h->stream.launch(h->d_tensors, v, sc, h->error_word, stream);
-        if (e != cudaSuccess) return cuda_fail(h, e);
-    }
+    if (prof) AM_CUDA(h, cudaEventRecord(h->prof_ev[1], stream));
+    AM_CUDA(h, h->stream.launch_main(h->d_tensors, v, sc, h->error_word, stream));
+    if (prof) AM_CUDA(h, cudaEventRecord(h->prof_ev[2], stream));
+    AM_CUDA(h, h->stream.launch_cluster(h->d_tensors, v, sc, h->error_word, stream));
+    if (prof) AM_CUDA(h, cudaEventRecord(h->prof_ev[3], stream));
     if (h->piece_units) {
         twopass_partial_kernel<<<static_cast<unsigned>(h->piece_units), kThreads, 0, stream>>>(
             h->d_tensors, h->d_piece_segs, h->n_piece_segs, h->d_partials);
@@ -378,6 +397,17 @@ int adammini_step(am_handle *h, void *const *params, const void *const *grads, v
             h->d_tensors, h->d_piece_segs, h->n_piece_segs, h->d_block_steps, sc);
         AM_CUDA(h, cudaGetLastError());
     }
+    if (prof) {
+        AM_CUDA(h, cudaEventRecord(h->prof_ev[4], stream));
+        h->prof_recorded = true;
+    }
+    return AM_OK;
+}
+
+int adammini_get_profile(am_handle *h, float *ms) {
+    if (!h || !ms || !h->prof_recorded) return AM_ERR_INVALID_ARGUMENT;
+    AM_CUDA(h, cudaEventSynchronize(h->prof_ev[4]));
+    for (int k = 0; k < 4; ++k) AM_CUDA(h, cudaEventElapsedTime(&ms[k], h->prof_ev[k], h->prof_ev[k + 1]));
     return AM_OK;
 }
 
@@ -400,6 +430,8 @@ int adammini_destroy(am_handle *h) {
         if (h->pinned[k]) cudaFreeHost(h->pinned[k]);
         if (h->ev[k]) cudaEventDestroy(h->ev[k]);
     }
+    for (int k = 0; k < 5; ++k)
+        if (h->prof_ev[k]) cudaEventDestroy(h->prof_ev[k]);
     if (h->error_word) cudaFreeHost(h->error_word);
     delete h;
     return AM_OK;

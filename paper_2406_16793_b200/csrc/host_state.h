@@ -18,7 +18,7 @@ struct am_handle {
     int64_t total_blocks = 0;
     int64_t total_elems = 0;
     am_hparams hp{};
-    int64_t opt[4] = {0, 0, 0, 0};
+    int64_t opt[5] = {0, 0, 0, 0, 0};
 
     // launch plan
     bool planned = false;
@@ -37,6 +37,9 @@ struct am_handle {
     int launches = 0;
     int64_t elems_by_path[4] = {0, 0, 0, 0};
     int64_t algorithmic_bytes = 0;
+    int64_t bytes_by_path[4] = {0, 0, 0, 0};
+    cudaEvent_t prof_ev[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+    bool prof_recorded = false;
 
     // pinned staging of the tensor table, double buffered
     am::DevTensor *pinned[2] = {nullptr, nullptr};

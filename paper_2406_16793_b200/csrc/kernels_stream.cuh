@@ -578,17 +578,13 @@ struct StreamPlan {
         return cudaLaunchKernelEx(&cfg, stream_kernel<false>, P);
     }
 
-    cudaError_t launch(const DevTensor *tensors, float *v, const StepScalars &sc, int *error_word,
-                       cudaStream_t stream) const {
-        if (main.active()) {
-            cudaError_t e = launch_one(main, false, tensors, v, sc, error_word, stream);
-            if (e != cudaSuccess) return e;
-        }
-        if (clus.active()) {
-            cudaError_t e = launch_one(clus, true, tensors, v, sc, error_word, stream);
-            if (e != cudaSuccess) return e;
-        }
-        return cudaSuccess;
+    cudaError_t launch_main(const DevTensor *tensors, float *v, const StepScalars &sc, int *error_word,
+                            cudaStream_t stream) const {
+        return main.active() ? launch_one(main, false, tensors, v, sc, error_word, stream) : cudaSuccess;
+    }
+    cudaError_t launch_cluster(const DevTensor *tensors, float *v, const StepScalars &sc, int *error_word,
+                               cudaStream_t stream) const {
+        return clus.active() ? launch_one(clus, true, tensors, v, sc, error_word, stream) : cudaSuccess;
     }
 };
 

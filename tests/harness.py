@@ -26,10 +26,20 @@ GUARD = 64          # float32 guard words either side of every test buffer
 SENTINEL = -7.0e33
 
 
+MIN_SCALE_RUN = 64
+
+
 def block_relative_error(got: np.ndarray, want: np.ndarray, L: int) -> float:
-    """max_i |got-want| / max(|want_i|, rms(want over i's block)); NaN/inf must match."""
-    got = np.asarray(got, dtype=np.float64).reshape(-1, L)
-    want = np.asarray(want, dtype=np.float64).reshape(-1, L)
+    """max_i |got-want| / max(|want_i|, rms(want over i's block)); NaN/inf must match.
+
+    For blocks shorter than 64 elements the RMS is taken over the aligned run
+    of 64 consecutive elements that holds the block (a one-element block has no
+    scale of its own: an entry of m or p that crosses zero would otherwise make
+    the ratio meaningless)."""
+    got = np.asarray(got, dtype=np.float64).reshape(-1)
+    want = np.asarray(want, dtype=np.float64).reshape(-1)
+    if want.size == 0:
+        return 0.0
     fin = np.isfinite(want)
     if not np.array_equal(fin, np.isfinite(got)):
         return float("inf")
@@ -38,11 +48,14 @@ def block_relative_error(got: np.ndarray, want: np.ndarray, L: int) -> float:
         if not same.all():
             return float("inf")
     w = np.where(fin, want, 0.0)
-    rms = np.sqrt((w * w).mean(axis=1, keepdims=True))
-    scale = np.maximum(np.abs(w), rms)
+    run = L if L >= MIN_SCALE_RUN else MIN_SCALE_RUN
+    starts = np.arange(0, w.size, run)
+    counts = np.diff(np.append(starts, w.size))
+    rms = np.sqrt(np.add.reduceat(w * w, starts) / counts)
+    scale = np.maximum(np.abs(w), np.repeat(rms, counts))
     scale = np.where(scale > 0, scale, 1.0)
     err = np.where(fin, np.abs(got - w) / scale, 0.0)
-    return float(err.max()) if err.size else 0.0
+    return float(err.max())
 
 
 def v_relative_error(got: np.ndarray, want: np.ndarray) -> float:
