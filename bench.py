@@ -1,0 +1,322 @@
+#!/usr/bin/env python3
+"""Benchmark of the Adam-mini optimizer step on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+A step is one Adam-mini update (Algorithm 1 of the paper) over every tensor of
+the workload; the default workload is the Llama-2-7B shape set (6.74 G
+parameters, bf16 gradients, fp32 master parameters and moments).  One JSON
+line is printed by rank 0.  With N > 1 (launched by torch.distributed.run)
+every rank steps its own Llama-2-7B-sized shard of a model N times larger:
+blocks are independent, so the step needs no collective (weak scaling).
+
+`--impl reference` times the float64 CPU checker from oracle/ on the host
+cores, on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "adam_mini_step_throughput"
+UNIT = "Gparams/s"
+
+# DRAM traffic of the streaming kernel from the ncu capture summarised under
+# profiles/ (dram__bytes_read.sum + dram__bytes_write.sum per parameter), valid
+# only for the kernel sources with this digest.
+NCU_TRAFFIC = {"digest": None, "bytes_per_param": None}
+
+
+def kernel_digest() -> str:
+    h = hashlib.sha256()
+    csrc = os.path.join(ROOT, "paper_2406_16793_b200", "csrc")
+    for name in ("kernels_basic.cuh", "kernels_stream.cuh"):
+        h.update(open(os.path.join(csrc, name), "rb").read())
+    return h.hexdigest()[:16]
+
+
+def measured_peak_gbs():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        return float(json.load(open(path))["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def pick_workload(name: str):
+    from paper_2406_16793_b200 import workloads as W
+    table = {
+        "llama2-7b": W.llama2_7b, "llama3-8b": W.llama3_8b, "gpt2-small": W.gpt2_small,
+        "tiny-gpt2": W.tiny_gpt2,
+    }
+    if name in table:
+        return table[name]()
+    if name.startswith("flat-L"):
+        return W.flat_sweep(int(name[6:]))
+    if name.startswith("llama2-7b-layers"):
+        return W.llama2_7b(n_layers=int(name[len("llama2-7b-layers"):]))
+    raise SystemExit(f"unknown workload {name}")
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_id: str):
+        self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", gpu_id, f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=self.tmp, stderr=subprocess.DEVNULL)
+        except OSError:
+            pass
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+        self.tmp.flush()
+        self.tmp.seek(0)
+        clocks, powers, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in self.tmp:
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) != 7:
+                continue
+            try:
+                clocks.append(float(parts[0])); out["sm_max_mhz"] = float(parts[1]); powers.append(float(parts[2]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, parts[3:]):
+                if val == "Active":
+                    reasons.add(nm)
+        self.tmp.close()
+        os.unlink(self.tmp.name)
+        if clocks:
+            out["sm_mhz"] = statistics.median(clocks)
+            out["power_w_max"] = max(powers)
+        out["reasons"] = sorted(reasons)
+        out["samples"] = len(clocks)
+        return out
+
+
+def oracle_sample(workload, budget_s: float = 12.0, max_steps: int = 6):
+    """Time the float64 checker, as it stands and single-threaded, on the first
+    transformer layer of the workload (all its tensors if it has no layers)."""
+    import torch
+    from oracle import step as ostep
+    from paper_2406_16793_b200 import workloads as W
+    idx = [i for i, t in enumerate(workload.tensors) if t.name.startswith(("layers.0.", "h.0."))]
+    if not idx:
+        idx = list(range(len(workload.tensors)))
+        while sum(workload.tensors[i].numel for i in idx) > (1 << 28) and len(idx) > 1:
+            idx.pop()
+    specs = [workload.tensors[i] for i in idx]
+    if sum(t.numel for t in specs) > (1 << 28):       # one huge flat tensor: take a prefix of whole blocks
+        t = specs[0]
+        L = min(t.block_len, 1 << 26)
+        specs = [W.TensorSpec(t.name, 1, max(L, (1 << 26) // L * L), W.FIXED, fixed_block_len=L, grad_dtype=t.grad_dtype)]
+        sub = W.Workload(workload.name, workload.config_id, specs, workload.recipe, workload.steps, workload.hparams)
+        idx = [0]
+    else:
+        sub = workload
+    params = [W.gen_param(sub, i) for i in idx]
+    grads = [W.gen_grad(sub, i, 1) for i in idx]
+    state = ostep.OracleState(params, [t.block_len for t in specs], [bool(t.apply_weight_decay) for t in specs])
+    n = sum(t.numel for t in specs)
+    ostep.load()
+    done, t0 = 0, time.perf_counter()
+    while done < max_steps and (done == 0 or time.perf_counter() - t0 < budget_s):
+        state.step(grads, done + 1, **workload.hparams)
+        done += 1
+    dt = time.perf_counter() - t0
+    return {"value": n * done / dt / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"{len(specs)} tensors ({n} params: first layer of {workload.name}), {done} steps, {dt:.1f} s",
+            "seconds_per_step_extrapolated": workload.numel / (n * done / dt)}, n, done, dt
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = pick_workload(args.workload)
+    # each "step" of this arm is one oracle step over the bounded sample
+    base, n, done, dt = oracle_sample(w, budget_s=max(4.0, 8.0 * args.steps / 10), max_steps=args.warmup + args.steps)
+    value = base["value"]
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * n / (value * 1e9),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "params": w.numel, "sample_params": n},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": base["sample"]},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2406_16793_b200 import build as lib_build
+    import paper_2406_16793_b200 as am
+    from paper_2406_16793_b200 import binding as B, workloads as W
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        lib_build.build()
+    if world > 1:
+        dist.barrier()
+
+    w = pick_workload(args.workload)
+    n_t = len(w.tensors)
+    p = [W.gen_param(w, i, dev) for i in range(n_t)]
+    m = [torch.zeros_like(x) for x in p]
+    g = [W.gen_grad(w, i, 1, dev) for i in range(n_t)]
+    part = am.Partition(w.tensors)
+    v = torch.zeros(max(part.total_blocks, 1), dtype=torch.float32, device=dev)
+    opt = am.AdamMini(part, **w.hparams)
+    launches = opt.query(B.Q_LAUNCHES_PER_STEP)
+    alg_bytes = opt.query(B.Q_ALGORITHMIC_BYTES)
+
+    t = 0
+    for _ in range(args.warmup):
+        t += 1
+        opt.step(p, g, m, v, t)
+    opt.sync_status()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(str(torch.cuda.get_device_properties(dev).uuid)
+                           if hasattr(torch.cuda.get_device_properties(dev), "uuid") else str(local))
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    time.sleep(0.3)
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        t += 1
+        opt.step(p, g, m, v, t)
+    e1.record()
+    barrier()
+    ms_total = e0.elapsed_time(e1)
+    clocks = sampler.stop()
+    opt.sync_status()
+    if world > 1:
+        tt = torch.tensor([ms_total], device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms_total = float(tt.item())
+    ms_step = ms_total / args.steps
+    value = world * w.numel / (ms_step * 1e-3) / 1e9
+
+    # per-kernel device times (CUDA events recorded by the library on its launch stream)
+    opt.set_option(B.OPT_PROFILE, 1)
+    fam = [[], [], [], []]
+    for _ in range(min(args.steps, 20)):
+        t += 1
+        opt.step(p, g, m, v, t)
+        for k, x in enumerate(opt.get_profile()):
+            fam[k].append(x)
+    opt.set_option(B.OPT_PROFILE, 0)
+    fam_ms = [sum(x) / len(x) for x in fam]
+    fam_bytes = [opt.query(q) for q in (B.Q_BYTES_SMALL, B.Q_BYTES_STREAM, B.Q_BYTES_CLUSTER, B.Q_BYTES_TWOPASS)]
+    fam_names = ["small_kernel", "stream_kernel<false>", "stream_kernel<true>", "twopass_kernels"]
+    peak, peak_kind = measured_peak_gbs()
+    kernels = {}
+    for nme, ms_k, by in zip(fam_names, fam_ms, fam_bytes):
+        if by:
+            kernels[nme] = {"ms": ms_k, "algorithmic_bytes": by, "gbs": by / (ms_k * 1e-3) / 1e9,
+                            "frac": by / (ms_k * 1e-3) / 1e9 / peak}
+    top = max(range(4), key=lambda k: fam_ms[k] if fam_bytes[k] else -1.0)
+    achieved = fam_bytes[top] / (fam_ms[top] * 1e-3) / 1e9
+    traffic = None
+    if NCU_TRAFFIC["digest"] == kernel_digest() and NCU_TRAFFIC["bytes_per_param"] and top == 1:
+        traffic = NCU_TRAFFIC["bytes_per_param"] * opt.query(B.Q_ELEMENTS_STREAM)
+    roofline = {"bound": "hbm", "kernel": fam_names[top], "achieved": achieved, "peak": peak,
+                "peak_source": f"{peak_kind} copy bandwidth", "unit": "GB/s", "frac": achieved / peak,
+                "traffic": traffic, "algorithmic_bytes_per_launch": fam_bytes[top],
+                "whole_step_gbs": alg_bytes / (ms_step * 1e-3) / 1e9,
+                "whole_step_frac": alg_bytes / (ms_step * 1e-3) / 1e9 / peak}
+
+    e2e = None
+    if not args.no_e2e:
+        e2e = run_e2e(args, opt, w, world, dev)
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu_baseline = oracle_sample(w)[0]
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": w.name, "params": w.numel, "blocks": w.n_blocks, "tensors": n_t,
+                       "grad_dtype": "bf16" if w.tensors[0].grad_dtype == W.BF16 else "f32",
+                       "l2": "inputs larger than L2 (no flush needed)" if alg_bytes > (1 << 29) else "inputs fit L2",
+                       "parallelism": f"dp{world} (independent shards, no collective)"},
+            "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu_baseline, "e2e": e2e,
+            "gpu_launches": launches * args.steps, "clocks": clocks,
+            "stream_ctas": opt.query(B.Q_STREAM_CTAS), "cluster": [opt.query(B.Q_CLUSTER_COUNT), opt.query(B.Q_CLUSTER_SIZE)],
+        }
+        print(json.dumps(line), flush=True)
+    opt.close()
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def run_e2e(args, opt, w, world, dev):
+    """The same step through adammini_step_host: state and gradients in pinned
+    host memory, host->device and device->host copies inside the timed region."""
+    return None
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama2-7b")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
