@@ -144,6 +144,45 @@ int adammini_step(am_handle *h, void *const *params, const void *const *grads, v
 int adammini_step_host(am_handle *h, void *const *params, const void *const *grads, void *const *m,
                        float *v, int64_t step, int64_t staging_bytes);
 
+/* One Adam-mini step on ONE tensor without any allocation.  (The paper has no
+ * counterpart: this entry point exists for callers that must not allocate.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a
+ * framework's memory-pool callback or a training loop whose allocator owns the
+ * whole device, in a process that has handed all free memory to another
+ * library, or in latency-critical sections where an allocation's implicit
+ * synchronisation is not acceptable.  adammini_create allocates device tables
+ * and scratch; this call allocates nothing, neither on the device nor through
+ * any library: its scratch (partial sums of g*g and per-block step sizes) is a
+ * fixed array compiled into the library, AM_NOALLOC_SCRATCH_BYTES of device
+ * memory that every GPU holds from the moment the library is loaded on it
+ * until the process exits.
+ *
+ *   param, m : DEVICE float32[numel], updated in place; grad: DEVICE, numel
+ *              elements of grad_dtype, read only; v: DEVICE float32[numel/block_len],
+ *              updated in place.  All 16-byte aligned.  m, v zero before step 1.
+ *   block_len must divide numel.  Limits: numel/block_len <= AM_NOALLOC_MAX_BLOCKS
+ *   and the number of partial sums, (numel/block_len) * ceil(block_len/32768)
+ *   (pieces grow beyond 32768 elements only for blocks over 2^29 elements),
+ *   <= AM_NOALLOC_MAX_PIECES; larger requests return AM_ERR_TOO_LARGE and do
+ *   nothing.
+ *
+ * The result equals adammini_step's on its two-pass path (same arithmetic).
+ * The first call on a device looks up the array's device address (once per
+ * device, with that device current); make that first call outside any stream
+ * capture.  Every call on a device shares the one array, which keeps whatever
+ * the previous call left there: each call overwrites the entries it uses before
+ * it reads them, so nothing needs clearing, but two calls whose kernels overlap
+ * on the GPU (different streams, or different threads or processes' streams on
+ * one context) race on it -- keep such calls on one stream or order them with
+ * events.  Asynchronous on cuda_stream like adammini_step. */
+#define AM_NOALLOC_MAX_BLOCKS 32768
+#define AM_NOALLOC_MAX_PIECES 32768
+#define AM_NOALLOC_SCRATCH_BYTES (AM_NOALLOC_MAX_PIECES * 8 + AM_NOALLOC_MAX_BLOCKS * 4)
+int adammini_step_tensor_noalloc(void *param, const void *grad, void *m, float *v, int64_t numel,
+                                 int64_t block_len, int32_t grad_dtype, int32_t apply_weight_decay,
+                                 const am_hparams *hp, int64_t step, void *cuda_stream);
+
 /* Waits for the stream and returns AM_OK, or AM_ERR_TIMEOUT if a device-side
  * bounded wait gave up during any step since the last call, or AM_ERR_CUDA. */
 int adammini_sync_status(am_handle *h, void *cuda_stream);

@@ -61,6 +61,9 @@ _SIGNATURES = {
                                      ctypes.POINTER(ctypes.c_void_p), ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p]),
     "adammini_step_host": (ctypes.c_int, [ctypes.c_void_p, ctypes.POINTER(ctypes.c_void_p), ctypes.POINTER(ctypes.c_void_p),
                                           ctypes.POINTER(ctypes.c_void_p), ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64]),
+    "adammini_step_tensor_noalloc": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                                    ctypes.c_int64, ctypes.c_int64, ctypes.c_int32, ctypes.c_int32,
+                                                    ctypes.POINTER(HParams), ctypes.c_int64, ctypes.c_void_p]),
     "adammini_sync_status": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p]),
     "adammini_set_option": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64]),
     "adammini_query": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.POINTER(ctypes.c_int64)]),
@@ -105,6 +108,27 @@ def _check(status: int, handle=None) -> None:
 def kind_from_name(name: str) -> int:
     """Algorithm 3's name tests (embed/output, query/key, value/attn.proj/mlp, else)."""
     return int(load().adammini_kind_from_name(name.encode()))
+
+
+NOALLOC_MAX_BLOCKS = 32768
+NOALLOC_MAX_PIECES = 32768
+
+
+def step_tensor_noalloc(param, grad, m, v, block_len: int, step: int, *, lr: float = 1e-3, beta1: float = 0.9,
+                        beta2: float = 0.95, eps: float = 1e-8, weight_decay: float = 0.1,
+                        apply_weight_decay: bool = True, stream: int = 0) -> None:
+    """One Adam-mini step on one tensor through the entry point that allocates
+    nothing (for callers that may not call cudaMalloc: allocator callbacks,
+    loops whose memory pool owns the device, latency-critical sections).  The
+    tensors are device tensors; v has numel/block_len entries.  All calls on a
+    device share one fixed scratch array inside the library, so issue them on
+    one stream (or order them); at most NOALLOC_MAX_BLOCKS blocks per call."""
+    numel = int(param.numel())
+    dtype = BF16 if str(grad.dtype) == "torch.bfloat16" else F32
+    hp = HParams(lr, beta1, beta2, eps, weight_decay)
+    _check(load().adammini_step_tensor_noalloc(
+        int(param.data_ptr()), int(grad.data_ptr()), int(m.data_ptr()), int(v.data_ptr()), numel,
+        int(block_len), dtype, int(bool(apply_weight_decay)), ctypes.byref(hp), int(step), stream or None))
 
 
 class Partition:

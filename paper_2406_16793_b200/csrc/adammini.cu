@@ -440,3 +440,147 @@ int adammini_destroy(am_handle *h) {
 }  // extern "C"
 
 #include "host_step.inl"
+
+// ---------------------------------------------------------------------------
+// adammini_step_tensor_noalloc: the two-pass update of one tensor with its
+// scratch in a fixed device array instead of allocated memory.
+// ---------------------------------------------------------------------------
+namespace {
+
+constexpr int kNoAllocMaxDevices = 64;
+
+// partial sums (double) first, per-block step sizes (float) after them
+static __device__ __align__(256) unsigned char g_noalloc_scratch[AM_NOALLOC_SCRATCH_BYTES];
+
+// Device address of the array on each device; the symbol itself is only a
+// host-side handle and must never be handed to a kernel.
+void *g_noalloc_addr[kNoAllocMaxDevices] = {};
+
+__device__ __forceinline__ PieceRef noalloc_piece(const DevTensor &t, int64_t local, bool vec) {
+    PieceRef r;
+    r.t = &t;
+    r.local = local;
+    r.block = local / t.pieces_per_block;
+    const int64_t off = (local - r.block * t.pieces_per_block) * t.piece_len;
+    r.start = r.block * t.L + off;
+    const int64_t left = t.L - off;
+    r.n = left < t.piece_len ? left : t.piece_len;
+    r.vec = vec;
+    return r;
+}
+
+__global__ void __launch_bounds__(kThreads)
+noalloc_partial_kernel(const __grid_constant__ DevTensor t, int vec, double *__restrict__ partials) {
+    __shared__ double warp_part[kThreads / 32];
+    const PieceRef r = noalloc_piece(t, blockIdx.x, vec != 0);
+    const double w = warp_sum(t.gdtype == AM_BF16 ? piece_sum_sq<AM_BF16>(r) : piece_sum_sq<AM_F32>(r));
+    if ((threadIdx.x & 31) == 0) warp_part[threadIdx.x >> 5] = w;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double s = 0.0;
+#pragma unroll
+        for (int k = 0; k < kThreads / 32; ++k) s += warp_part[k];
+        partials[r.local] = s;
+    }
+}
+
+__global__ void __launch_bounds__(kThreads)
+noalloc_finalize_kernel(const __grid_constant__ DevTensor t, const double *__restrict__ partials,
+                        float *__restrict__ block_steps, float *__restrict__ v, StepScalars sc) {
+    const int64_t b = static_cast<int64_t>(blockIdx.x) * (kThreads / 32) + (threadIdx.x >> 5);
+    if (b >= t.n_blocks) return;
+    const int lane = threadIdx.x & 31;
+    const double *src = partials + b * t.pieces_per_block;
+    double s = 0.0;
+    for (int64_t j = lane; j < t.pieces_per_block; j += 32) s += src[j];
+    s = warp_sum(s);
+    if (lane == 0) {
+        float vn;
+        const float st = block_step(s, static_cast<double>(t.L), v[b], sc, &vn);
+        v[b] = vn;
+        block_steps[b] = st;
+    }
+}
+
+__global__ void __launch_bounds__(kThreads)
+noalloc_update_kernel(const __grid_constant__ DevTensor t, int vec, const float *__restrict__ block_steps,
+                      StepScalars sc) {
+    const PieceRef r = noalloc_piece(t, blockIdx.x, vec != 0);
+    if (t.gdtype == AM_BF16) twopass_update_body<AM_BF16>(r, block_steps, sc);
+    else twopass_update_body<AM_F32>(r, block_steps, sc);
+}
+
+}  // namespace
+
+extern "C" int adammini_step_tensor_noalloc(void *param, const void *grad, void *m, float *v, int64_t numel,
+                                            int64_t block_len, int32_t grad_dtype, int32_t apply_weight_decay,
+                                            const am_hparams *hp, int64_t step, void *cuda_stream) {
+    if (!param || !grad || !m || !v || step < 1 || numel < 0) return AM_ERR_INVALID_ARGUMENT;
+    if (grad_dtype != AM_F32 && grad_dtype != AM_BF16) return AM_ERR_INVALID_ARGUMENT;
+    const int rc = validate_hparams(hp);
+    if (rc != AM_OK) return rc;
+    if (block_len <= 0 || numel % block_len != 0) return AM_ERR_SHAPE;
+    if (!aligned16(param) || !aligned16(grad) || !aligned16(m) || !aligned16(v)) return AM_ERR_MISALIGNED;
+    if (numel == 0) return AM_OK;
+
+    DevTensor t{};
+    t.g = grad;
+    t.m = static_cast<float *>(m);
+    t.p = static_cast<float *>(param);
+    t.numel = numel;
+    t.L = block_len;
+    t.n_blocks = numel / block_len;
+    t.v_offset = 0;
+    t.gdtype = grad_dtype;
+    t.wd = apply_weight_decay ? 1 : 0;
+    t.piece_len = block_len;
+    t.pieces_per_block = 1;
+    if (block_len > kPieceMax) {
+        int64_t ppb = std::min<int64_t>(ceil_div(block_len, kPieceMax), kMaxPiecesPerBlock);
+        t.piece_len = ceil_div(ceil_div(block_len, ppb), 1024) * 1024;
+        t.pieces_per_block = ceil_div(block_len, t.piece_len);
+    }
+    t.piece_base = 0;
+    t.block_base = 0;      // block_steps is indexed by block inside the array
+    if (t.n_blocks > AM_NOALLOC_MAX_BLOCKS) return AM_ERR_TOO_LARGE;
+    const int64_t pieces = t.n_blocks * t.pieces_per_block;
+    if (pieces > AM_NOALLOC_MAX_PIECES) return AM_ERR_TOO_LARGE;
+
+    // set-up, once per device: the device address of the static array
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess || dev < 0 || dev >= kNoAllocMaxDevices) return AM_ERR_CUDA;
+    if (!g_noalloc_addr[dev]) {
+        void *ptr = nullptr;
+        e = cudaGetSymbolAddress(&ptr, g_noalloc_scratch);
+        if (e != cudaSuccess || !ptr) return AM_ERR_CUDA;
+        g_noalloc_addr[dev] = ptr;
+    }
+    double *partials = static_cast<double *>(g_noalloc_addr[dev]);
+    float *block_steps = reinterpret_cast<float *>(static_cast<unsigned char *>(g_noalloc_addr[dev]) +
+                                                   AM_NOALLOC_MAX_PIECES * sizeof(double));
+
+    const double bc1 = 1.0 - std::pow(hp->beta1, static_cast<double>(step));
+    const double bc2 = 1.0 - std::pow(hp->beta2, static_cast<double>(step));
+    StepScalars sc;
+    sc.beta2 = hp->beta2;
+    sc.omb2 = 1.0 - hp->beta2;
+    sc.inv_bc2 = 1.0 / bc2;
+    sc.lr_over_bc1 = hp->lr / bc1;
+    sc.eps = hp->eps;
+    sc.beta1 = static_cast<float>(hp->beta1);
+    sc.omb1 = static_cast<float>(1.0 - hp->beta1);
+    sc.lr_wd = static_cast<float>(hp->lr * hp->weight_decay);
+    sc.pad = 0.f;
+
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const int vec = block_len % 4 == 0 ? 1 : 0;
+    noalloc_partial_kernel<<<static_cast<unsigned>(pieces), kThreads, 0, stream>>>(t, vec, partials);
+    if (cudaGetLastError() != cudaSuccess) return AM_ERR_CUDA;
+    noalloc_finalize_kernel<<<static_cast<unsigned>(ceil_div(t.n_blocks, kThreads / 32)), kThreads, 0, stream>>>(
+        t, partials, block_steps, v, sc);
+    if (cudaGetLastError() != cudaSuccess) return AM_ERR_CUDA;
+    noalloc_update_kernel<<<static_cast<unsigned>(pieces), kThreads, 0, stream>>>(t, vec, block_steps, sc);
+    if (cudaGetLastError() != cudaSuccess) return AM_ERR_CUDA;
+    return AM_OK;
+}
