@@ -36,7 +36,7 @@ UNIT = "Gparams/s"
 # DRAM traffic of the streaming kernel from the ncu capture summarised under
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum per parameter), valid
 # only for the kernel sources with this digest.
-NCU_TRAFFIC = {"digest": None, "bytes_per_param": None}
+NCU_TRAFFIC = {"digest": "5e4ac492867af903", "bytes_per_param": 17.90}
 
 
 def kernel_digest() -> str:
@@ -119,7 +119,7 @@ class ClockSampler:
         return out
 
 
-def oracle_sample(workload, budget_s: float = 12.0, max_steps: int = 6):
+def oracle_sample(workload, budget_s: float = 12.0, max_steps: int = 40):
     """Time the float64 checker, as it stands and single-threaded, on the first
     transformer layer of the workload (all its tensors if it has no layers)."""
     import torch
@@ -203,6 +203,10 @@ def run_ours(args):
     part = am.Partition(w.tensors)
     v = torch.zeros(max(part.total_blocks, 1), dtype=torch.float32, device=dev)
     opt = am.AdamMini(part, **w.hparams)
+    for key, val in ((B.OPT_STREAM_THREADS, args.stream_threads), (B.OPT_STREAM_CTAS, args.stream_ctas),
+                     (B.OPT_CLUSTER_SIZE, args.cluster_size), (B.OPT_PATH, args.path)):
+        if val:
+            opt.set_option(key, val)
     launches = opt.query(B.Q_LAUNCHES_PER_STEP)
     alg_bytes = opt.query(B.Q_ALGORITHMIC_BYTES)
 
@@ -217,8 +221,8 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    sampler = ClockSampler(str(torch.cuda.get_device_properties(dev).uuid)
-                           if hasattr(torch.cuda.get_device_properties(dev), "uuid") else str(local))
+    props = torch.cuda.get_device_properties(dev)
+    sampler = ClockSampler("GPU-" + str(props.uuid) if hasattr(props, "uuid") else str(local))
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     time.sleep(0.3)
     barrier()
@@ -308,6 +312,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama2-7b")
+    ap.add_argument("--stream-threads", type=int, default=0, help="consumer threads per CTA (0 = library default)")
+    ap.add_argument("--stream-ctas", type=int, default=0, help="persistent CTAs (0 = one per SM)")
+    ap.add_argument("--cluster-size", type=int, default=0, help="CTAs per cluster for head-sized blocks (0 = default)")
+    ap.add_argument("--path", type=int, default=0, help="1 = force the two-pass kernels")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
