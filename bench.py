@@ -273,7 +273,7 @@ def run_ours(args):
 
     e2e = None
     if not args.no_e2e:
-        e2e = run_e2e(args, opt, w, world, dev)
+        e2e = run_e2e(args, opt, w, world, dev, p, g, m, v)
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -299,10 +299,47 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-def run_e2e(args, opt, w, world, dev):
-    """The same step through adammini_step_host: state and gradients in pinned
-    host memory, host->device and device->host copies inside the timed region."""
-    return None
+def run_e2e(args, opt, w, world, dev, p, g, m, v):
+    """The same step through adammini_step_host: parameters, moments, v and
+    gradients in pinned host memory; host->device and device->host copies are
+    inside the timed region (CUDA events cannot bracket a call that blocks on
+    several internal streams, so this arm is timed with the host clock around
+    the blocking C call, max over ranks)."""
+    import torch
+    import torch.distributed as dist
+    need = sum(t.numel * (8 + (2 if t.grad_dtype else 4)) for t in w.tensors)
+    avail = 0
+    for line in open("/proc/meminfo"):
+        if line.startswith("MemAvailable"):
+            avail = int(line.split()[1]) * 1024
+    if avail < 2.2 * need * max(1, min(world, torch.cuda.device_count())):
+        return {"value": None, "unit": UNIT, "skipped": f"host memory: need {need} B pinned per rank, {avail} B available"}
+    hp = [x.to("cpu", non_blocking=False).pin_memory() for x in p]
+    hm = [x.to("cpu").pin_memory() for x in m]
+    hg = [x.to("cpu").pin_memory() for x in g]
+    hv = v.to("cpu").pin_memory()
+    h2d = sum(x.numel() * x.element_size() for x in hp + hm + hg) + hv.numel() * 4
+    d2h = sum(x.numel() * x.element_size() for x in hp + hm) + hv.numel() * 4
+    steps = max(1, min(args.e2e_steps, args.steps))
+    t = 1000
+    opt.step_host(hp, hg, hm, hv, t)          # warm-up: builds the staging pipeline
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        t += 1
+        opt.step_host(hp, hg, hm, hv, t)
+    torch.cuda.synchronize()
+    dt = time.perf_counter() - t0
+    if world > 1:
+        tt = torch.tensor([dt], device=dev, dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        dt = float(tt.item())
+    return {"value": world * w.numel * steps / dt / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
+            "d2h_bytes_per_step": d2h, "ms_per_step": 1e3 * dt / steps, "steps": steps,
+            "h2d_plus_d2h_gbs": (h2d + d2h) * steps / dt / 1e9, "workload": w.name,
+            "api": "adammini_step_host (pinned host buffers, 3 staging slots)"}
 
 
 def main():
@@ -317,6 +354,7 @@ def main():
     ap.add_argument("--cluster-size", type=int, default=0, help="CTAs per cluster for head-sized blocks (0 = default)")
     ap.add_argument("--path", type=int, default=0, help="1 = force the two-pass kernels")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

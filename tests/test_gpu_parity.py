@@ -197,3 +197,24 @@ def test_empty_partition_and_queries():
     assert opt.query(B.Q_LAUNCHES_PER_STEP) == 2
     assert opt.query(B.Q_ALGORITHMIC_BYTES) == 18 * n + 8 * w.n_blocks
     opt.close()
+
+
+@pytest.mark.parametrize("staging", [0, 3 * (24 << 20)], ids=["default-staging", "many-groups"])
+def test_host_buffer_step_matches_device_step(staging):
+    """adammini_step_host (state in host memory, streamed through staging slots)
+    gives the same bits as adammini_step on device-resident state."""
+    w = W.scaled_rows(W.llama2_7b(n_layers=1, vocab=512), 128)
+    dev = H.DeviceState(w, guarded=False)
+    opt = H.make_optimizer(w)
+    hp = [x.cpu().pin_memory() for x in dev.p]
+    hm = [x.cpu().pin_memory() for x in dev.m]
+    hv = dev.v.cpu().pin_memory()
+    for t in (1, 2, 3):
+        dev.draw_grads(t)
+        hg = [x.cpu() for x in dev.g]                       # pageable on purpose
+        opt.step(dev.p, dev.g, dev.m, dev.v, t)
+        opt.step_host(hp, hg, hm, hv, t, staging_bytes=staging)
+    opt.sync_status()
+    for a, b in zip(dev.p + dev.m + [dev.v], hp + hm + [hv]):
+        assert torch.equal(a.cpu(), b)
+    opt.close()
