@@ -189,3 +189,38 @@ def run_parity(w: W.Workload, steps: Optional[int] = None, options: Optional[Dic
 
 def assert_parity(worst: Dict[str, float], tol: float = TOL) -> None:
     assert worst["p"] <= tol and worst["m"] <= tol and worst["v"] <= tol, worst
+
+
+def run_sampled_parity(w: W.Workload, steps: int, tensor_indices: Sequence[int], blocks_per_tensor: int = 3,
+                       device="cuda") -> Dict[str, float]:
+    """Full-size run in the configuration the benchmark times (unguarded
+    buffers, default options); the oracle recomputes a sample of blocks one by
+    one: first, last and seeded-random blocks of the chosen tensors."""
+    dev = DeviceState(w, device, guarded=False)
+    opt = make_optimizer(w)
+    rng = np.random.default_rng(W.mix_seed(W.BASE_SEED, w.config_id, 4242) % (1 << 32))
+    samples = []            # (tensor, block, oracle p, m, v)
+    for i in tensor_indices:
+        t = w.tensors[i]
+        picks = {0, t.n_blocks - 1} | {int(x) for x in rng.integers(0, t.n_blocks, max(0, blocks_per_tensor - 2))}
+        for b in sorted(picks):
+            sl = slice(b * t.block_len, (b + 1) * t.block_len)
+            samples.append([i, b, sl, ostep.widen(dev.p[i][sl].cpu()), np.zeros(t.block_len), np.zeros(1)])
+    for step in range(1, steps + 1):
+        dev.draw_grads(step)
+        opt.step(dev.p, dev.g, dev.m, dev.v, step)
+        for s in samples:
+            i, b, sl = s[0], s[1], s[2]
+            t = w.tensors[i]
+            ostep.adammini_step(s[3], s[4], s[5], dev.g[i][sl].cpu(), t.block_len, step=step,
+                                apply_wd=bool(t.apply_weight_decay), **w.hparams)
+    opt.sync_status()
+    worst = {"p": 0.0, "m": 0.0, "v": 0.0, "blocks": len(samples)}
+    v_off = np.cumsum([0] + [t.n_blocks for t in w.tensors])
+    for i, b, sl, po, mo, vo in samples:
+        L = w.tensors[i].block_len
+        worst["p"] = max(worst["p"], block_relative_error(dev.p[i][sl].cpu().numpy(), po, L))
+        worst["m"] = max(worst["m"], block_relative_error(dev.m[i][sl].cpu().numpy(), mo, L))
+        worst["v"] = max(worst["v"], v_relative_error(dev.v[v_off[i] + b:v_off[i] + b + 1].cpu().numpy(), vo))
+    opt.close()
+    return worst

@@ -218,3 +218,20 @@ def test_host_buffer_step_matches_device_step(staging):
     for a, b in zip(dev.p + dev.m + [dev.v], hp + hm + [hv]):
         assert torch.equal(a.cpu(), b)
     opt.close()
+
+
+def test_full_size_llama2_7b_sampled_blocks():
+    """All 6.74 G parameters of the Llama-2-7B shape set, stepped exactly as the
+    benchmark steps them; the oracle recomputes sampled blocks of every kind
+    (token rows, heads, output-neuron rows of 4096 and 11008, norms) from the
+    first, a middle and the last layer."""
+    free, _ = torch.cuda.mem_get_info()
+    if free < 75 * (1 << 30):
+        pytest.skip("needs about 70 GB of free device memory")
+    w = W.llama2_7b()
+    picks = [0, len(w.tensors) - 1, len(w.tensors) - 2]
+    for layer in (0, 17, 31):
+        picks += list(range(1 + 9 * layer, 1 + 9 * (layer + 1)))
+    worst = H.run_sampled_parity(w, steps=4, tensor_indices=picks, blocks_per_tensor=3)
+    assert worst["blocks"] >= 60
+    H.assert_parity(worst)
