@@ -3,6 +3,7 @@
 binding    ctypes front end of the CUDA library (libadammini.so, C ABI in include/adammini.h)
 workloads  model-shaped tensor lists and seeded synthetic inputs
 build      in-tree nvcc build of the library for sm_100a
+sharding   whole-block sharding of a step over data-parallel ranks (host logic)
 """
-from . import binding, workloads  # noqa: F401
+from . import binding, sharding, workloads  # noqa: F401
 from .binding import AdamMini, AdamMiniError, Partition  # noqa: F401
