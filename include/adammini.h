@@ -194,8 +194,13 @@ typedef enum {
     AM_OPT_STREAM_CTAS   = 1, /* persistent CTAs of the streaming kernel (0 = one per SM) */
     AM_OPT_CLUSTER_SIZE  = 2, /* CTAs per cluster for head-sized blocks (0 = default) */
     AM_OPT_STREAM_THREADS = 3, /* consumer threads per CTA of the streaming kernels (0 = default) */
-    AM_OPT_PROFILE       = 4  /* 1: record CUDA events around each kernel family of every step
+    AM_OPT_PROFILE       = 4, /* 1: record CUDA events around each kernel family of every step
                                  (read them with adammini_get_profile) */
+    AM_OPT_STREAM_CHUNK  = 5  /* how the streaming kernel's CTAs share the work: 0 = automatic (CTAs take
+                                 up to 64 work items at a time from a shared counter, which evens out
+                                 bandwidth differences between SMs); 1..4096 = that many items at a
+                                 time; 1000000 = every CTA walks its own fixed, cost-balanced range.
+                                 Results are bit-identical in every mode */
 } am_option;
 int adammini_set_option(am_handle *h, int32_t key, int64_t value);
 

@@ -36,16 +36,18 @@ namespace am {
 constexpr int kStageElems = 4096;                 // elements of g, m, p per PACKED/APPLY stage
 constexpr int kWarpBlockMaxL = 1024;              // blocks up to this length are reduced by one warp
 constexpr int kCtrlBytes = 2048;                  // barriers, stage descriptors, reduction slots
+constexpr int kVAreaFloats = 272;                 // per stage: the old v of the stage's blocks (16-byte windows)
 constexpr int kMaxStages = 8;
 constexpr int kMaxConsumerWarps = 16;
 constexpr int kMaxCluster = 8;
+constexpr int kStaticRanges = 1000000;            // AM_OPT_STREAM_CHUNK value that selects static ranges
 constexpr int64_t kStreamMaxBlockBytes = 256 << 10;   // longest block one CTA handles alone (bytes of g)
 constexpr int64_t kClusterMaxBlockBytes = 4 << 20;    // longest block a cluster handles (bytes of g)
 constexpr unsigned long long kWaitTimeoutNs = 2000000000ull;   // 2 s
 constexpr unsigned long long kDrainTimeoutNs = 50000000ull;    // 50 ms
 
 enum StageKind : int32_t { STAGE_PACKED = 0, STAGE_SUM = 1, STAGE_APPLY = 2, STAGE_DONE = 3 };
-enum StageFlag : int32_t { SF_BF16 = 1, SF_WD = 2, SF_LAST = 4, SF_WRITE_V = 8 };
+enum StageFlag : int32_t { SF_BF16 = 1, SF_WD = 2, SF_LAST = 4, SF_WRITE_V = 8, SF_V_STAGED = 16 };
 
 struct StageMeta {          // written by the producer, read by the consumers
     float *m;               // global destination of this stage's first element
@@ -56,7 +58,8 @@ struct StageMeta {          // written by the producer, read by the consumers
     int32_t L;              // block length (PACKED)
     int32_t kind;
     int32_t flags;
-    int64_t pad[2];
+    int32_t v_shift;        // SF_V_STAGED: the first block's v sits at this index of the stage's v area
+    int32_t pad[3];
 };
 static_assert(sizeof(StageMeta) == 64, "stage descriptor is 64 bytes");
 
@@ -78,6 +81,10 @@ struct StreamParams {
     int32_t stage_bytes;
     int32_t g_region_bytes;     // m starts here inside a stage; p follows kStageElems floats later
     int32_t consumer_threads;
+    int32_t chunk;              // > 0: items are handed out `chunk` at a time from *counter
+    unsigned long long *counter;
+    int64_t total_items;
+    int64_t v_len;              // floats in v (staging never reads past it)
 };
 
 struct Control {            // first kCtrlBytes of dynamic shared memory
@@ -270,6 +277,7 @@ stream_kernel(const __grid_constant__ StreamParams P) {
     extern __shared__ __align__(128) unsigned char smem[];
     Control *ctl = reinterpret_cast<Control *>(smem);
     unsigned char *stages = smem + kCtrlBytes;
+    float *v_areas = reinterpret_cast<float *>(stages + static_cast<size_t>(P.n_stages) * P.stage_bytes);
     const int tid = threadIdx.x;
     const int n_cwarps = P.consumer_threads >> 5;
     const uint32_t crank = CLUSTER ? cluster_ctarank() : 0;
@@ -300,7 +308,7 @@ stream_kernel(const __grid_constant__ StreamParams P) {
             int64_t armed = 0;              // stages armed so far
             bool ok = true;
             int seg = 0;
-            {
+            if (CLUSTER || P.chunk <= 0) {
                 int lo = 0, hi = P.n_segs - 1;      // last segment starting at or before item_lo
                 while (lo < hi) {
                     const int mid = (lo + hi + 1) >> 1;
@@ -315,7 +323,33 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                 ++armed;
                 if (++stage == P.n_stages) { stage = 0; phase ^= 1u; }
             };
-            for (int64_t it = item_lo; it < item_hi && ok; ++it) {
+            // Old v of blocks [first, first+count) of v, copied as whole 16-byte
+            // windows next to the stage; skipped (consumers then read v from
+            // global memory) when the last window would reach past the end of v.
+            auto stage_v = [&](StageMeta &mt, int64_t first, int count) -> uint32_t {
+                const int64_t w0 = first & ~int64_t(3), w1 = (first + count + 3) & ~int64_t(3);
+                if (w1 > P.v_len || w1 - w0 > kVAreaFloats) return 0u;
+                mt.flags |= SF_V_STAGED;
+                mt.v_shift = static_cast<int32_t>(first - w0);
+                return static_cast<uint32_t>(w1 - w0) * 4u;
+            };
+            // Static mode: the CTA's own contiguous range.  Dynamic mode (single-CTA
+            // launches only): ranges of `chunk` items from a global counter, the
+            // next range requested while the current one is being issued.
+            const bool dynamic = !CLUSTER && P.chunk > 0;
+            int64_t it = item_lo, hi = item_hi, next = 0;
+            if (dynamic) {
+                it = static_cast<int64_t>(atomicAdd(P.counter, static_cast<unsigned long long>(P.chunk)));
+                hi = it + P.chunk < P.total_items ? it + P.chunk : P.total_items;
+                next = static_cast<int64_t>(atomicAdd(P.counter, static_cast<unsigned long long>(P.chunk)));
+            }
+            for (; ok; ++it) {
+                if (it >= hi) {
+                    if (!dynamic || next >= P.total_items) break;
+                    it = next;
+                    hi = it + P.chunk < P.total_items ? it + P.chunk : P.total_items;
+                    next = static_cast<int64_t>(atomicAdd(P.counter, static_cast<unsigned long long>(P.chunk)));
+                }
                 while (seg + 1 < P.n_segs && P.segs[seg + 1].item_begin <= it) ++seg;
                 const StreamSeg sg = P.segs[seg];
                 const DevTensor &t = P.tensors[sg.tensor];
@@ -334,8 +368,12 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                     mt.m = t.m + e0; mt.p = t.p + e0; mt.v = P.v + t.v_offset + b0;
                     mt.inv_L = 1.0 / static_cast<double>(t.L);
                     mt.n = n; mt.L = static_cast<int>(t.L); mt.kind = STAGE_PACKED; mt.flags = base_flags | SF_WRITE_V;
+                    const uint32_t vbytes = stage_v(mt, t.v_offset + b0, nb);
                     unsigned char *st = stages + static_cast<size_t>(stage) * P.stage_bytes;
-                    mbar_arrive_expect_tx(&ctl->full[stage], static_cast<uint32_t>(n) * (gsz + 8));
+                    mbar_arrive_expect_tx(&ctl->full[stage], static_cast<uint32_t>(n) * (gsz + 8) + vbytes);
+                    if (vbytes)
+                        bulk_load(v_areas + stage * kVAreaFloats, P.v + ((t.v_offset + b0) & ~int64_t(3)), vbytes,
+                                  &ctl->full[stage]);
                     bulk_load(st, gbase + e0 * gsz, n * gsz, &ctl->full[stage]);
                     bulk_load(st + P.g_region_bytes, t.m + e0, n * 4, &ctl->full[stage]);
                     bulk_load(st + P.g_region_bytes + kStageElems * 4, t.p + e0, n * 4, &ctl->full[stage]);
@@ -353,8 +391,12 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                         mt.inv_L = 1.0 / static_cast<double>(t.L);
                         mt.n = c; mt.L = 0; mt.kind = STAGE_SUM;
                         mt.flags = base_flags | (off + c == slice ? SF_LAST : 0) | (crank == 0 ? SF_WRITE_V : 0);
+                        const uint32_t vbytes = (off + c == slice) ? stage_v(mt, t.v_offset + local, 1) : 0u;
                         unsigned char *st = stages + static_cast<size_t>(stage) * P.stage_bytes;
-                        mbar_arrive_expect_tx(&ctl->full[stage], static_cast<uint32_t>(c) * gsz);
+                        mbar_arrive_expect_tx(&ctl->full[stage], static_cast<uint32_t>(c) * gsz + vbytes);
+                        if (vbytes)
+                            bulk_load(v_areas + stage * kVAreaFloats, P.v + ((t.v_offset + local) & ~int64_t(3)), vbytes,
+                                      &ctl->full[stage]);
                         bulk_load(st, gbase + (e0 + off) * gsz, c * gsz, &ctl->full[stage]);
                         advance();
                     }
@@ -410,6 +452,8 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                 const float *ms = reinterpret_cast<const float *>(gs + P.g_region_bytes);
                 const float *ps = ms + kStageElems;
                 const bool bf16 = (mt.flags & SF_BF16) != 0;
+                // where the old v of the stage's blocks is read from
+                const float *v_src = (mt.flags & SF_V_STAGED) ? v_areas + stage * kVAreaFloats + mt.v_shift : mt.v;
                 const float lr_wd = (mt.flags & SF_WD) ? P.sc.lr_wd : 0.f;
                 bool alive = true;
 
@@ -421,11 +465,14 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                             float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
                             if (bf16) sum_span<AM_BF16>(gs, e, L, lane, 32, s0, s1, s2, s3);
                             else sum_span<AM_F32>(gs, e, L, lane, 32, s0, s1, s2, s3);
-                            const double tot = warp_sum(fold4(s0, s1, s2, s3));
-                            float v_old = lane == 0 ? mt.v[b] : 0.f;
+                            // at most 8 terms per accumulator and a 5-level tree: float is enough
+                            float tot = (s0 + s1) + (s2 + s3);
+#pragma unroll
+                            for (int o = 16; o > 0; o >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, o);
+                            float v_old = lane == 0 ? v_src[b] : 0.f;
                             v_old = __shfl_sync(0xffffffffu, v_old, 0);
                             float vn;
-                            const float step = stream_block_step(tot, mt.inv_L, v_old, P.sc, &vn);
+                            const float step = stream_block_step(static_cast<double>(tot), mt.inv_L, v_old, P.sc, &vn);
                             if (lane == 0) mt.v[b] = vn;
                             if (bf16) apply_span<AM_BF16>(gs, ms, ps, mt.m, mt.p, e, L, lane, 32, beta1, omb1, lr_wd, step);
                             else apply_span<AM_F32>(gs, ms, ps, mt.m, mt.p, e, L, lane, 32, beta1, omb1, lr_wd, step);
@@ -439,7 +486,7 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                             double tot;
                             float v_old;
                             alive = group_reduce(ctl, gsync, P.error_word, ctid, n_cwarps, fold4(s0, s1, s2, s3),
-                                                 mt.v + b, &tot, &v_old);
+                                                 v_src + b, &tot, &v_old);
                             if (!alive) break;
                             float vn;
                             const float step = stream_block_step(tot, mt.inv_L, v_old, P.sc, &vn);
@@ -454,13 +501,16 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                 } else if (mt.kind == STAGE_SUM) {
                     if (bf16) sum_span<AM_BF16>(gs, 0, mt.n, ctid, nthr, a0, a1, a2, a3);
                     else sum_span<AM_F32>(gs, 0, mt.n, ctid, nthr, a0, a1, a2, a3);
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&ctl->empty[stage]);
-                    if (mt.flags & SF_LAST) {
+                    if (!(mt.flags & SF_LAST)) {
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&ctl->empty[stage]);
+                    } else {
                         double tot;
                         float v_old;
-                        if (!group_reduce(ctl, gsync, P.error_word, ctid, n_cwarps, fold4(a0, a1, a2, a3), mt.v, &tot, &v_old))
+                        if (!group_reduce(ctl, gsync, P.error_word, ctid, n_cwarps, fold4(a0, a1, a2, a3), v_src, &tot, &v_old))
                             break;
+                        __syncwarp();                       // the stage (and its v area) has been read
+                        if (lane == 0) mbar_arrive(&ctl->empty[stage]);
                         a0 = a1 = a2 = a3 = 0.f;
                         if (CLUSTER) {
                             // exchange the CTAs' sums through distributed shared memory
@@ -498,7 +548,7 @@ stream_kernel(const __grid_constant__ StreamParams P) {
 
 // ------------------------------- host-side planning -------------------------------
 struct StreamPlanInput {
-    int sm_count = 0, ctas = 0, cluster_size = 0, threads = 0;
+    int sm_count = 0, ctas = 0, cluster_size = 0, threads = 0, chunk = 0;
     struct Item { int tensor; am_table_row row; };
     std::vector<Item> stream_tensors, cluster_tensors;
 };
@@ -520,11 +570,12 @@ inline void stream_add_tensor(StreamPlanInput &in, int index, const am_table_row
 struct StreamLaunch {
     std::vector<StreamSeg> segs;     // with sentinel
     std::vector<int64_t> bounds;
-    int grid = 0, cluster = 1, n_stages = 0, stage_bytes = 0, g_region_bytes = 0, threads = 0;
+    int grid = 0, cluster = 1, n_stages = 0, stage_bytes = 0, g_region_bytes = 0, threads = 0, chunk = 0;
+    unsigned long long *d_counter = nullptr;
     const StreamSeg *d_segs = nullptr;
     const int64_t *d_bounds = nullptr;
     bool active() const { return grid > 0; }
-    size_t smem_bytes() const { return kCtrlBytes + static_cast<size_t>(n_stages) * stage_bytes; }
+    size_t smem_bytes() const { return kCtrlBytes + static_cast<size_t>(n_stages) * (stage_bytes + kVAreaFloats * 4); }
 };
 
 constexpr size_t kSmemBudget = 227 * 1024;
@@ -534,7 +585,7 @@ struct StreamPlan {
 
     size_t table_bytes() const {
         return (main.segs.size() + clus.segs.size()) * sizeof(StreamSeg) + 256 +
-               (main.bounds.size() + clus.bounds.size()) * sizeof(int64_t) + 256;
+               (main.bounds.size() + clus.bounds.size()) * sizeof(int64_t) + 256 + 512;
     }
     int launches() const { return (main.active() ? 1 : 0) + (clus.active() ? 1 : 0); }
 
@@ -550,9 +601,13 @@ struct StreamPlan {
             if (e != cudaSuccess) return e;
             L->d_bounds = reinterpret_cast<const int64_t *>(base + off);
             off += (L->bounds.size() * sizeof(int64_t) + 127) / 128 * 128;
+            L->d_counter = reinterpret_cast<unsigned long long *>(base + off);
+            off += 128;
         }
         return cudaSuccess;
     }
+
+    int64_t v_len = 0;
 
     cudaError_t launch_one(const StreamLaunch &L, bool cluster, const DevTensor *tensors, float *v,
                            const StepScalars &sc, int *error_word, cudaStream_t stream) const {
@@ -560,6 +615,12 @@ struct StreamPlan {
         P.tensors = tensors; P.segs = L.d_segs; P.bounds = L.d_bounds; P.v = v; P.error_word = error_word;
         P.sc = sc; P.n_segs = static_cast<int>(L.segs.size()) - 1; P.n_stages = L.n_stages;
         P.stage_bytes = L.stage_bytes; P.g_region_bytes = L.g_region_bytes; P.consumer_threads = L.threads;
+        P.v_len = v_len;
+        P.chunk = cluster ? 0 : L.chunk; P.counter = L.d_counter; P.total_items = L.bounds.empty() ? 0 : L.bounds.back();
+        if (P.chunk > 0) {
+            cudaError_t e = cudaMemsetAsync(L.d_counter, 0, sizeof(unsigned long long), stream);
+            if (e != cudaSuccess) return e;
+        }
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(L.grid);
         cfg.blockDim = dim3(32 + L.threads);
@@ -599,7 +660,7 @@ inline void stream_build_launch(const std::vector<StreamPlanInput::Item> &tensor
     for (const auto &it : tensors) any_f32 |= it.row.grad_dtype == AM_F32;
     out->g_region_bytes = kStageElems * (any_f32 ? 4 : 2);
     out->stage_bytes = out->g_region_bytes + kStageElems * 8;
-    out->n_stages = std::min<int>(kMaxStages, static_cast<int>((kSmemBudget - kCtrlBytes) / out->stage_bytes));
+    out->n_stages = std::min<int>(kMaxStages, static_cast<int>((kSmemBudget - kCtrlBytes) / (out->stage_bytes + kVAreaFloats * 4)));
 
     std::vector<double> item_cost;      // per segment
     int64_t items = 0;
@@ -657,7 +718,7 @@ inline void stream_probe_cluster(int sm_count, int threads, int wanted, int *clu
     *cluster_size = 0;
     *n_clusters = 0;
     if (threads <= 0) threads = 256;
-    const size_t smem = kCtrlBytes + 5 * (kStageElems * 10);   // the larger of the two stage layouts
+    const size_t smem = kCtrlBytes + 5 * (kStageElems * 10 + kVAreaFloats * 4);   // the larger of the two stage layouts
     for (int cs = wanted > 0 ? wanted : kMaxCluster; cs >= 1; cs >>= 1) {
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(std::max(sm_count / cs, 1) * cs);
@@ -686,6 +747,13 @@ inline void stream_finish_plan(const StreamPlanInput &in, int cluster_size, int 
     stream_build_launch(in.stream_tensors, false, ctas, &plan->main);
     plan->main.threads = threads;
     plan->main.cluster = 1;
+    // work distribution: ranges of `chunk` items from a shared counter unless static ranges were asked for
+    if (in.chunk == kStaticRanges) plan->main.chunk = 0;
+    else if (in.chunk > 0) plan->main.chunk = in.chunk;
+    else {
+        const int64_t items = plan->main.bounds.empty() ? 0 : plan->main.bounds.back();
+        plan->main.chunk = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(64, items / (int64_t(32) * std::max(ctas, 1)))));
+    }
     plan->clus = StreamLaunch();
     if (!in.cluster_tensors.empty() && n_clusters > 0) {
         stream_build_launch(in.cluster_tensors, true, n_clusters, &plan->clus);

@@ -235,3 +235,17 @@ def test_full_size_llama2_7b_sampled_blocks():
     worst = H.run_sampled_parity(w, steps=4, tensor_indices=picks, blocks_per_tensor=3)
     assert worst["blocks"] >= 60
     H.assert_parity(worst)
+
+
+@pytest.mark.parametrize("chunk", [1, 7, 1000000])
+def test_dynamic_work_distribution_gives_identical_bits(chunk):
+    w = W.scaled_rows(W.llama2_7b(n_layers=2, vocab=1024), 512)
+    a = _run_steps(w, 1, 3)
+    dev = H.DeviceState(w, guarded=False)
+    opt = H.make_optimizer(w, {B.OPT_STREAM_CHUNK: chunk})
+    for t in (1, 2, 3):
+        dev.draw_grads(t)
+        opt.step(dev.p, dev.g, dev.m, dev.v, t)
+    opt.sync_status()
+    opt.close()
+    assert _same(a, dev)
