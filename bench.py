@@ -205,7 +205,7 @@ def run_ours(args):
     opt = am.AdamMini(part, **w.hparams)
     for key, val in ((B.OPT_STREAM_THREADS, args.stream_threads), (B.OPT_STREAM_CTAS, args.stream_ctas),
                      (B.OPT_CLUSTER_SIZE, args.cluster_size), (B.OPT_PATH, args.path),
-                     (B.OPT_STREAM_CHUNK, args.stream_chunk)):
+                     (B.OPT_STREAM_CHUNK, args.stream_chunk), (B.OPT_CLUSTER_CHUNK, args.cluster_chunk)):
         if val:
             opt.set_option(key, val)
     launches = opt.query(B.Q_LAUNCHES_PER_STEP)
@@ -291,6 +291,7 @@ def run_ours(args):
                        "parallelism": f"dp{world} (independent shards, no collective)"},
             "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu_baseline, "e2e": e2e,
             "gpu_launches": launches * args.steps, "clocks": clocks,
+            "gpu": {"name": props.name, "uuid_tail": str(getattr(props, "uuid", ""))[-8:]},
             "stream_ctas": opt.query(B.Q_STREAM_CTAS), "cluster": [opt.query(B.Q_CLUSTER_COUNT), opt.query(B.Q_CLUSTER_SIZE)],
         }
         print(json.dumps(line), flush=True)
@@ -354,6 +355,7 @@ def main():
     ap.add_argument("--stream-ctas", type=int, default=0, help="persistent CTAs (0 = one per SM)")
     ap.add_argument("--cluster-size", type=int, default=0, help="CTAs per cluster for head-sized blocks (0 = default)")
     ap.add_argument("--stream-chunk", type=int, default=0, help="items per grab from the shared work counter (0 = automatic, 1000000 = static ranges)")
+    ap.add_argument("--cluster-chunk", type=int, default=0, help="blocks per grab of a cluster (0 = automatic, 1000000 = static)")
     ap.add_argument("--path", type=int, default=0, help="1 = force the two-pass kernels")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=3)

@@ -201,6 +201,7 @@ typedef enum {
                                  bandwidth differences between SMs); 1..4096 = that many items at a
                                  time; 1000000 = every CTA walks its own fixed, cost-balanced range.
                                  Results are bit-identical in every mode */
+    , AM_OPT_CLUSTER_CHUNK = 6 /* the same for the cluster kernel, in blocks handed to a cluster at a time */
 } am_option;
 int adammini_set_option(am_handle *h, int32_t key, int64_t value);
 

@@ -20,7 +20,7 @@ using namespace am;
 
 namespace {
 
-constexpr int kNumOptions = 6;
+constexpr int kNumOptions = 7;
 
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
@@ -74,6 +74,7 @@ int build_plan(am_handle *h) {
     sin.cluster_size = static_cast<int>(h->opt[AM_OPT_CLUSTER_SIZE]);
     sin.threads = static_cast<int>(h->opt[AM_OPT_STREAM_THREADS]);
     sin.chunk = static_cast<int>(h->opt[AM_OPT_STREAM_CHUNK]);
+    sin.cluster_chunk = static_cast<int>(h->opt[AM_OPT_CLUSTER_CHUNK]);
 
     stream_probe_cluster(h->sm_count, sin.threads, sin.cluster_size, &h->cluster_size, &h->n_clusters);
 
@@ -281,7 +282,8 @@ int adammini_set_hparams(am_handle *h, const am_hparams *hp) {
 int adammini_set_option(am_handle *h, int32_t key, int64_t value) {
     if (!h || key < 0 || key >= kNumOptions || value < 0) return AM_ERR_INVALID_ARGUMENT;
     if ((key == AM_OPT_PATH || key == AM_OPT_PROFILE) && value > 1) return AM_ERR_INVALID_ARGUMENT;
-    if (key == AM_OPT_STREAM_CHUNK && value > 4096 && value != kStaticRanges) return AM_ERR_INVALID_ARGUMENT;
+    if ((key == AM_OPT_STREAM_CHUNK || key == AM_OPT_CLUSTER_CHUNK) && value > 4096 && value != kStaticRanges)
+        return AM_ERR_INVALID_ARGUMENT;
     if (key == AM_OPT_PROFILE) {
         if (value && !h->prof_ev[0])
             for (int k = 0; k < 5; ++k) AM_CUDA(h, cudaEventCreate(&h->prof_ev[k]));

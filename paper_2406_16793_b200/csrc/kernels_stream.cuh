@@ -40,6 +40,7 @@ constexpr int kVAreaFloats = 272;                 // per stage: the old v of the
 constexpr int kMaxStages = 8;
 constexpr int kMaxConsumerWarps = 16;
 constexpr int kMaxCluster = 8;
+constexpr int kItemSlots = 8;                     // block indices in flight from a cluster's first CTA to its peers
 constexpr int kStaticRanges = 1000000;            // AM_OPT_STREAM_CHUNK value that selects static ranges
 constexpr int64_t kStreamMaxBlockBytes = 256 << 10;   // longest block one CTA handles alone (bytes of g)
 constexpr int64_t kClusterMaxBlockBytes = 4 << 20;    // longest block a cluster handles (bytes of g)
@@ -97,6 +98,8 @@ struct Control {            // first kCtrlBytes of dynamic shared memory
     float redv[2];
     int abort_flag;
     int pad;
+    unsigned long long ibar[kItemSlots];   // cluster launches: "the next block index has arrived"
+    long long next_item[kItemSlots];
     StageMeta meta[kMaxStages];
 };
 static_assert(sizeof(Control) <= kCtrlBytes, "control block fits its reservation");
@@ -155,6 +158,9 @@ __device__ __forceinline__ uint32_t map_to_rank(uint32_t local_smem_addr, uint32
 }
 __device__ __forceinline__ void st_cluster_f64(uint32_t cluster_addr, double x) {
     asm volatile("st.shared::cluster.f64 [%0], %1;" ::"r"(cluster_addr), "d"(x) : "memory");
+}
+__device__ __forceinline__ void st_cluster_s64(uint32_t cluster_addr, long long x) {
+    asm volatile("st.shared::cluster.s64 [%0], %1;" ::"r"(cluster_addr), "l"(x) : "memory");
 }
 __device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
@@ -292,6 +298,7 @@ stream_kernel(const __grid_constant__ StreamParams P) {
         mbar_init(&ctl->redbar, n_cwarps);
         mbar_init(&ctl->xbar[0], csize);
         mbar_init(&ctl->xbar[1], csize);
+        for (int k = 0; k < kItemSlots; ++k) mbar_init(&ctl->ibar[k], 1);
         ctl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -308,7 +315,7 @@ stream_kernel(const __grid_constant__ StreamParams P) {
             int64_t armed = 0;              // stages armed so far
             bool ok = true;
             int seg = 0;
-            if (CLUSTER || P.chunk <= 0) {
+            if (P.chunk <= 0) {
                 int lo = 0, hi = P.n_segs - 1;      // last segment starting at or before item_lo
                 while (lo < hi) {
                     const int mid = (lo + hi + 1) >> 1;
@@ -333,22 +340,52 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                 mt.v_shift = static_cast<int32_t>(first - w0);
                 return static_cast<uint32_t>(w1 - w0) * 4u;
             };
-            // Static mode: the CTA's own contiguous range.  Dynamic mode (single-CTA
-            // launches only): ranges of `chunk` items from a global counter, the
-            // next range requested while the current one is being issued.
+            // Static mode: the CTA's (or cluster's) own contiguous range.  Dynamic mode:
+            // a single CTA takes ranges of `chunk` items from a global counter, the next
+            // range requested while the current one is being issued; in a cluster the
+            // first CTA takes one block at a time and hands the index to every CTA of the
+            // cluster through distributed shared memory, two blocks ahead.
             const bool dynamic = !CLUSTER && P.chunk > 0;
+            const bool cdynamic = CLUSTER && P.chunk > 0;
+            uint32_t published = 0, taken = 0;
+            auto cluster_publish = [&]() {
+                const long long idx = static_cast<long long>(atomicAdd(P.counter, static_cast<unsigned long long>(P.chunk)));
+                const uint32_t slot = published & (kItemSlots - 1);
+                ++published;
+                const uint32_t item = smem_addr(&ctl->next_item[slot]), bar = smem_addr(&ctl->ibar[slot]);
+                for (uint32_t r = 0; r < csize; ++r) {
+                    st_cluster_s64(map_to_rank(item, r), idx);
+                    mbar_arrive_remote(map_to_rank(bar, r));
+                }
+            };
+            auto cluster_take = [&]() -> int64_t {
+                const uint32_t slot = taken & (kItemSlots - 1), par = (taken / kItemSlots) & 1u;
+                ++taken;
+                if (!wait_phase<true>(&ctl->ibar[slot], par, ctl, P.error_word, 5)) { ok = false; return P.total_items; }
+                return *reinterpret_cast<volatile long long *>(&ctl->next_item[slot]);
+            };
             int64_t it = item_lo, hi = item_hi, next = 0;
             if (dynamic) {
                 it = static_cast<int64_t>(atomicAdd(P.counter, static_cast<unsigned long long>(P.chunk)));
                 hi = it + P.chunk < P.total_items ? it + P.chunk : P.total_items;
                 next = static_cast<int64_t>(atomicAdd(P.counter, static_cast<unsigned long long>(P.chunk)));
+            } else if (cdynamic) {
+                if (crank == 0) { cluster_publish(); cluster_publish(); }
+                it = hi = 0;                    // the loop's first test takes the first block
             }
             for (; ok; ++it) {
                 if (it >= hi) {
-                    if (!dynamic || next >= P.total_items) break;
-                    it = next;
-                    hi = it + P.chunk < P.total_items ? it + P.chunk : P.total_items;
-                    next = static_cast<int64_t>(atomicAdd(P.counter, static_cast<unsigned long long>(P.chunk)));
+                    if (cdynamic) {
+                        it = cluster_take();
+                        if (!ok || it >= P.total_items) break;
+                        hi = it + P.chunk < P.total_items ? it + P.chunk : P.total_items;
+                        if (crank == 0) cluster_publish();
+                    } else {
+                        if (!dynamic || next >= P.total_items) break;
+                        it = next;
+                        hi = it + P.chunk < P.total_items ? it + P.chunk : P.total_items;
+                        next = static_cast<int64_t>(atomicAdd(P.counter, static_cast<unsigned long long>(P.chunk)));
+                    }
                 }
                 while (seg + 1 < P.n_segs && P.segs[seg + 1].item_begin <= it) ++seg;
                 const StreamSeg sg = P.segs[seg];
@@ -548,7 +585,7 @@ stream_kernel(const __grid_constant__ StreamParams P) {
 
 // ------------------------------- host-side planning -------------------------------
 struct StreamPlanInput {
-    int sm_count = 0, ctas = 0, cluster_size = 0, threads = 0, chunk = 0;
+    int sm_count = 0, ctas = 0, cluster_size = 0, threads = 0, chunk = 0, cluster_chunk = 0;
     struct Item { int tensor; am_table_row row; };
     std::vector<Item> stream_tensors, cluster_tensors;
 };
@@ -616,7 +653,7 @@ struct StreamPlan {
         P.sc = sc; P.n_segs = static_cast<int>(L.segs.size()) - 1; P.n_stages = L.n_stages;
         P.stage_bytes = L.stage_bytes; P.g_region_bytes = L.g_region_bytes; P.consumer_threads = L.threads;
         P.v_len = v_len;
-        P.chunk = cluster ? 0 : L.chunk; P.counter = L.d_counter; P.total_items = L.bounds.empty() ? 0 : L.bounds.back();
+        P.chunk = L.chunk; P.counter = L.d_counter; P.total_items = L.bounds.empty() ? 0 : L.bounds.back();
         if (P.chunk > 0) {
             cudaError_t e = cudaMemsetAsync(L.d_counter, 0, sizeof(unsigned long long), stream);
             if (e != cudaSuccess) return e;
@@ -756,10 +793,25 @@ inline void stream_finish_plan(const StreamPlanInput &in, int cluster_size, int 
     }
     plan->clus = StreamLaunch();
     if (!in.cluster_tensors.empty() && n_clusters > 0) {
+        // Launch shape for head-sized blocks.  Measured on B200: blocks of up to 1 MB of
+        // gradients (bf16 heads of 128 x 4096) run best on clusters of 4 that take one block
+        // at a time from the shared counter; larger blocks on clusters of 8 with fixed ranges.
+        int64_t max_block_bytes = 0;
+        for (const auto &it : in.cluster_tensors)
+            max_block_bytes = std::max(max_block_bytes, it.row.block_len * (it.row.grad_dtype == AM_BF16 ? 2 : 4));
+        const bool small_blocks = max_block_bytes <= (int64_t(1) << 20);
+        int chunk = in.cluster_chunk;
+        if (in.cluster_size == 0 && small_blocks && cluster_size > 4) {
+            int cs4 = 0, n4 = 0;
+            stream_probe_cluster(in.sm_count, threads, 4, &cs4, &n4);
+            if (cs4 == 4 && n4 > 0) { cluster_size = 4; n_clusters = n4; }
+        }
+        if (chunk == 0) chunk = (in.cluster_size == 0 && !small_blocks) ? kStaticRanges : 1;
         stream_build_launch(in.cluster_tensors, true, n_clusters, &plan->clus);
         plan->clus.grid *= cluster_size;          // bounds are per cluster
         plan->clus.cluster = cluster_size;
         plan->clus.threads = threads;
+        plan->clus.chunk = chunk == kStaticRanges ? 0 : chunk;
     }
 }
 
