@@ -134,6 +134,29 @@ int adammini_set_hparams(am_handle *h, const am_hparams *hp);
 int adammini_step(am_handle *h, void *const *params, const void *const *grads, void *const *m,
                   float *v, int64_t step, void *cuda_stream);
 
+/* Optional extras of a step: trainer-side operations that sit next to
+ * optimizer.step() in mixed-precision training and cost nothing when fused
+ * into the same pass (the paper's Algorithm 1 is silent on them).
+ *   params_bf16       host array of n_tensors DEVICE pointers (entries may be NULL), 16-byte
+ *                     aligned: the updated parameter is also written there rounded to bfloat16
+ *                     (round to nearest even) -- the working copy of a bf16 model.  NULL: none.
+ *   grad_scale        every gradient is multiplied by this before use (1.0 = off): the inverse
+ *                     loss scale and/or a global-norm clip coefficient known on the host.
+ *   grad_scale_device optional DEVICE float multiplied in as well (a clip coefficient computed
+ *                     on the device).  NULL: none.
+ *   skip_flag         optional DEVICE float; if it is non-zero when the kernels run, the step
+ *                     changes nothing (found-inf skip of dynamic loss scaling).  NULL: never skip. */
+typedef struct am_step_extras {
+    void *const *params_bf16;
+    double grad_scale;
+    const float *grad_scale_device;
+    const float *skip_flag;
+} am_step_extras;
+
+/* adammini_step with extras (`ex` may be NULL, which is adammini_step). */
+int adammini_step_ex(am_handle *h, void *const *params, const void *const *grads, void *const *m,
+                     float *v, int64_t step, void *cuda_stream, const am_step_extras *ex);
+
 /* The same step for callers whose state lives in HOST memory (offloaded
  * optimizer state): params, grads, m are host arrays of HOST pointers, v is a
  * HOST pointer.  The library streams groups of tensors through device staging

@@ -12,7 +12,7 @@ import os
 from typing import Iterable, List, Optional, Sequence
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIBRARY = os.path.join(_HERE, "libadammini.so")
+LIBRARY = os.environ.get("ADAMMINI_LIBRARY") or os.path.join(_HERE, "libadammini.so")
 
 WHOLE, ROWS, HEADS, TOKENS, FIXED = 0, 1, 2, 3, 4
 F32, BF16 = 0, 1
@@ -40,6 +40,11 @@ class HParams(ctypes.Structure):
                 ("eps", ctypes.c_double), ("weight_decay", ctypes.c_double)]
 
 
+class StepExtras(ctypes.Structure):
+    _fields_ = [("params_bf16", ctypes.POINTER(ctypes.c_void_p)), ("grad_scale", ctypes.c_double),
+                ("grad_scale_device", ctypes.c_void_p), ("skip_flag", ctypes.c_void_p)]
+
+
 class AdamMiniError(RuntimeError):
     def __init__(self, status: int, message: str):
         super().__init__(f"adammini: {message} (status {status})")
@@ -59,6 +64,9 @@ _SIGNATURES = {
     "adammini_set_hparams": (ctypes.c_int, [ctypes.c_void_p, ctypes.POINTER(HParams)]),
     "adammini_step": (ctypes.c_int, [ctypes.c_void_p, ctypes.POINTER(ctypes.c_void_p), ctypes.POINTER(ctypes.c_void_p),
                                      ctypes.POINTER(ctypes.c_void_p), ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p]),
+    "adammini_step_ex": (ctypes.c_int, [ctypes.c_void_p, ctypes.POINTER(ctypes.c_void_p), ctypes.POINTER(ctypes.c_void_p),
+                                        ctypes.POINTER(ctypes.c_void_p), ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p,
+                                        ctypes.POINTER(StepExtras)]),
     "adammini_step_host": (ctypes.c_int, [ctypes.c_void_p, ctypes.POINTER(ctypes.c_void_p), ctypes.POINTER(ctypes.c_void_p),
                                           ctypes.POINTER(ctypes.c_void_p), ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64]),
     "adammini_step_tensor_noalloc": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
@@ -89,7 +97,12 @@ def load() -> ctypes.CDLL:
                 "(there is no CPU fallback)")
         lib = ctypes.CDLL(LIBRARY)
         for name, (res, args) in _SIGNATURES.items():
-            fn = getattr(lib, name)
+            try:
+                fn = getattr(lib, name)
+            except AttributeError:
+                if os.environ.get("ADAMMINI_LIBRARY"):
+                    continue            # an older build named explicitly: its missing calls fail when used
+                raise
             fn.restype = res
             fn.argtypes = args
         _lib = lib
@@ -225,6 +238,25 @@ class AdamMini:
         pa, ga, ma = self._arrays(params, grads, m)
         vp = int(v.data_ptr()) if hasattr(v, "data_ptr") else int(v)
         _check(load().adammini_step(self._h, pa, ga, ma, vp, int(step), stream or None), self._h)
+
+    def step_ex(self, params: Sequence, grads: Sequence, m: Sequence, v, step: int, stream: int = 0, *,
+                params_bf16: Optional[Sequence] = None, grad_scale: float = 1.0, grad_scale_device=None,
+                skip_flag=None) -> None:
+        """A step with the optional extras of adammini_step_ex: bf16 copies of the
+        updated parameters, a gradient scale (host value and/or device scalar)
+        and a device flag that turns the step into a no-op."""
+        pa, ga, ma = self._arrays(params, grads, m)
+        vp = int(v.data_ptr()) if hasattr(v, "data_ptr") else int(v)
+        ex = StepExtras()
+        keep = None
+        if params_bf16 is not None:
+            keep = _ptr_array([0 if t is None else (int(t.data_ptr()) if hasattr(t, "data_ptr") else int(t))
+                               for t in params_bf16])
+            ex.params_bf16 = ctypes.cast(keep, ctypes.POINTER(ctypes.c_void_p))
+        ex.grad_scale = float(grad_scale)
+        ex.grad_scale_device = int(grad_scale_device.data_ptr()) if grad_scale_device is not None else None
+        ex.skip_flag = int(skip_flag.data_ptr()) if skip_flag is not None else None
+        _check(load().adammini_step_ex(self._h, pa, ga, ma, vp, int(step), stream or None, ctypes.byref(ex)), self._h)
 
     def step_host(self, params: Sequence, grads: Sequence, m: Sequence, v, step: int,
                   staging_bytes: int = 0) -> None:

@@ -187,12 +187,14 @@ int build_plan(am_handle *h) {
 
 // Refresh the device tensor table if any data pointer changed.
 int refresh_pointers(am_handle *h, void *const *params, const void *const *grads, void *const *m,
-                     cudaStream_t stream) {
+                     void *const *params_bf16, cudaStream_t stream) {
     const int n = static_cast<int>(h->rows.size());
     bool changed = !h->ptrs_valid;
     for (int i = 0; i < n; ++i) {
         DevTensor &t = h->host_tensors[i];
-        if (t.g != grads[i] || t.m != m[i] || t.p != params[i]) {
+        uint16_t *pb = params_bf16 ? static_cast<uint16_t *>(params_bf16[i]) : nullptr;
+        if (t.g != grads[i] || t.m != m[i] || t.p != params[i] || t.p_bf16 != pb) {
+            t.p_bf16 = pb;
             t.g = grads[i];
             t.m = static_cast<float *>(m[i]);
             t.p = static_cast<float *>(params[i]);
@@ -335,7 +337,13 @@ int adammini_last_cuda_error(const am_handle *h) { return h ? h->last_cuda_error
 
 int adammini_step(am_handle *h, void *const *params, const void *const *grads, void *const *m,
                   float *v, int64_t step, void *cuda_stream) {
+    return adammini_step_ex(h, params, grads, m, v, step, cuda_stream, nullptr);
+}
+
+int adammini_step_ex(am_handle *h, void *const *params, const void *const *grads, void *const *m,
+                     float *v, int64_t step, void *cuda_stream, const am_step_extras *ex) {
     if (!h || !h->planned || step < 1) return AM_ERR_INVALID_ARGUMENT;
+    if (ex && !(std::isfinite(ex->grad_scale))) return AM_ERR_INVALID_ARGUMENT;
     const int n = static_cast<int>(h->rows.size());
     if (n == 0) return AM_OK;
     if (!params || !grads || !m || !v) return AM_ERR_INVALID_ARGUMENT;
@@ -344,13 +352,16 @@ int adammini_step(am_handle *h, void *const *params, const void *const *grads, v
         if (!aligned16(params[i]) || !aligned16(grads[i]) || !aligned16(m[i])) return AM_ERR_MISALIGNED;
     }
     if (!aligned16(v)) return AM_ERR_MISALIGNED;
+    if (ex && ex->params_bf16)
+        for (int i = 0; i < n; ++i)
+            if (!aligned16(ex->params_bf16[i])) return AM_ERR_MISALIGNED;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
 
     int dev = -1;
     AM_CUDA(h, cudaGetDevice(&dev));
     if (dev != h->device) return AM_ERR_INVALID_ARGUMENT;
 
-    int rc = refresh_pointers(h, params, grads, m, stream);
+    int rc = refresh_pointers(h, params, grads, m, ex ? ex->params_bf16 : nullptr, stream);
     if (rc != AM_OK) return rc;
 
     // scalars of this step (Algorithm 1: bias corrections use beta^t)
@@ -366,7 +377,9 @@ int adammini_step(am_handle *h, void *const *params, const void *const *grads, v
     sc.beta1 = static_cast<float>(hp.beta1);
     sc.omb1 = static_cast<float>(1.0 - hp.beta1);
     sc.lr_wd = static_cast<float>(hp.lr * hp.weight_decay);
-    sc.pad = 0.f;
+    sc.gscale = ex ? static_cast<float>(ex->grad_scale) : 1.f;
+    sc.gscale_dev = ex ? ex->grad_scale_device : nullptr;
+    sc.skip_flag = ex ? ex->skip_flag : nullptr;
 
     const bool prof = h->opt[AM_OPT_PROFILE] != 0;
     if (prof) AM_CUDA(h, cudaEventRecord(h->prof_ev[0], stream));
@@ -380,6 +393,9 @@ int adammini_step(am_handle *h, void *const *params, const void *const *grads, v
         ss.lr_over_bc1 = static_cast<float>(sc.lr_over_bc1);
         ss.eps = static_cast<float>(hp.eps);
         ss.lr_wd = sc.lr_wd;
+        ss.gscale = sc.gscale;
+        ss.gscale_dev = sc.gscale_dev;
+        ss.skip_flag = sc.skip_flag;
         small_kernel<<<static_cast<unsigned>(h->small_units), kThreads, 0, stream>>>(
             h->d_tensors, h->d_small_segs, h->n_small_segs, v, ss);
         AM_CUDA(h, cudaGetLastError());
@@ -391,7 +407,7 @@ int adammini_step(am_handle *h, void *const *params, const void *const *grads, v
     if (prof) AM_CUDA(h, cudaEventRecord(h->prof_ev[3], stream));
     if (h->piece_units) {
         twopass_partial_kernel<<<static_cast<unsigned>(h->piece_units), kThreads, 0, stream>>>(
-            h->d_tensors, h->d_piece_segs, h->n_piece_segs, h->d_partials);
+            h->d_tensors, h->d_piece_segs, h->n_piece_segs, h->d_partials, sc.gscale, sc.gscale_dev, sc.skip_flag);
         AM_CUDA(h, cudaGetLastError());
         const unsigned fin_grid = static_cast<unsigned>(ceil_div(h->block_units, kThreads / 32));
         twopass_finalize_kernel<<<fin_grid, kThreads, 0, stream>>>(
@@ -478,7 +494,7 @@ __global__ void __launch_bounds__(kThreads)
 noalloc_partial_kernel(const __grid_constant__ DevTensor t, int vec, double *__restrict__ partials) {
     __shared__ double warp_part[kThreads / 32];
     const PieceRef r = noalloc_piece(t, blockIdx.x, vec != 0);
-    const double w = warp_sum(t.gdtype == AM_BF16 ? piece_sum_sq<AM_BF16>(r) : piece_sum_sq<AM_F32>(r));
+    const double w = warp_sum(t.gdtype == AM_BF16 ? piece_sum_sq<AM_BF16>(r, 1.f) : piece_sum_sq<AM_F32>(r, 1.f));
     if ((threadIdx.x & 31) == 0) warp_part[threadIdx.x >> 5] = w;
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -576,7 +592,9 @@ extern "C" int adammini_step_tensor_noalloc(void *param, const void *grad, void 
     sc.beta1 = static_cast<float>(hp->beta1);
     sc.omb1 = static_cast<float>(1.0 - hp->beta1);
     sc.lr_wd = static_cast<float>(hp->lr * hp->weight_decay);
-    sc.pad = 0.f;
+    sc.gscale = 1.f;
+    sc.gscale_dev = nullptr;
+    sc.skip_flag = nullptr;
 
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const int vec = block_len % 4 == 0 ? 1 : 0;

@@ -28,6 +28,7 @@ struct DevTensor {
     const void *g;
     float *m;
     float *p;
+    uint16_t *p_bf16;   // optional bf16 copy of the updated parameters (nullptr: none)
     int64_t numel;
     int64_t L;          // block length
     int64_t n_blocks;
@@ -57,7 +58,9 @@ struct StepScalars {
     double eps;
     float beta1, omb1;      // beta1, 1-beta1
     float lr_wd;            // eta_t * lambda
-    float pad;
+    float gscale;           // gradients are multiplied by this on load (1 = off) ...
+    const float *gscale_dev;  // ... and by this device scalar when not null
+    const float *skip_flag;   // device scalar; non-zero: the step leaves everything untouched
 };
 
 }  // namespace am

@@ -4,6 +4,7 @@
 #ifndef ADAMMINI_KERNELS_BASIC_CUH_
 #define ADAMMINI_KERNELS_BASIC_CUH_
 
+#include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
 #include "adammini_internal.h"
@@ -24,21 +25,45 @@ __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w 
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 
 // Four consecutive gradients, widened exactly to float.
+// (every gradient is multiplied by `gscale` as it is loaded: 1.0f leaves it bit-exact)
 template <int GD>
-__device__ __forceinline__ float4 load_g4(const void *g, int64_t i) {
+__device__ __forceinline__ float4 load_g4(const void *g, int64_t i, float gscale) {
+    float4 r;
     if (GD == AM_BF16) {
         const uint2 u = *reinterpret_cast<const uint2 *>(static_cast<const uint16_t *>(g) + i);
-        return make_float4(bf16_lo(u.x), bf16_hi(u.x), bf16_lo(u.y), bf16_hi(u.y));
+        r = make_float4(bf16_lo(u.x), bf16_hi(u.x), bf16_lo(u.y), bf16_hi(u.y));
     } else {
-        return *reinterpret_cast<const float4 *>(static_cast<const float *>(g) + i);
+        r = *reinterpret_cast<const float4 *>(static_cast<const float *>(g) + i);
     }
+    r.x *= gscale; r.y *= gscale; r.z *= gscale; r.w *= gscale;
+    return r;
 }
 
 template <int GD>
-__device__ __forceinline__ float load_g1(const void *g, int64_t i) {
+__device__ __forceinline__ float load_g1(const void *g, int64_t i, float gscale) {
     if (GD == AM_BF16)
-        return __uint_as_float(static_cast<uint32_t>(static_cast<const uint16_t *>(g)[i]) << 16);
-    return static_cast<const float *>(g)[i];
+        return __uint_as_float(static_cast<uint32_t>(static_cast<const uint16_t *>(g)[i]) << 16) * gscale;
+    return static_cast<const float *>(g)[i] * gscale;
+}
+
+__device__ __forceinline__ float effective_gscale(float gscale, const float *gscale_dev) {
+    return gscale_dev ? gscale * *gscale_dev : gscale;
+}
+__device__ __forceinline__ bool step_skipped(const float *skip_flag) {
+    return skip_flag != nullptr && *skip_flag != 0.f;
+}
+
+// bf16 copy of updated parameters, round to nearest even
+__device__ __forceinline__ void store_bf16x4(uint16_t *dst, const float4 &p) {
+    const __nv_bfloat162 lo = __floats2bfloat162_rn(p.x, p.y), hi = __floats2bfloat162_rn(p.z, p.w);
+    uint2 u;
+    u.x = *reinterpret_cast<const uint32_t *>(&lo);
+    u.y = *reinterpret_cast<const uint32_t *>(&hi);
+    *reinterpret_cast<uint2 *>(dst) = u;
+}
+__device__ __forceinline__ void store_bf16(uint16_t *dst, float p) {
+    const __nv_bfloat16 b = __float2bfloat16_rn(p);
+    *dst = *reinterpret_cast<const uint16_t *>(&b);
 }
 
 // Elementwise part of Algorithm 1: first moment, decoupled decay on the old
@@ -89,7 +114,9 @@ __device__ __forceinline__ double warp_sum(double x) {
 // L <= 16: one thread per block, float32 scalars (at L == 1 this is AdamW)
 // ---------------------------------------------------------------------------
 struct SmallScalars {
-    float beta1, omb1, beta2, omb2, inv_bc2, lr_over_bc1, eps, lr_wd;
+    float beta1, omb1, beta2, omb2, inv_bc2, lr_over_bc1, eps, lr_wd, gscale;
+    const float *gscale_dev;
+    const float *skip_flag;
 };
 
 __device__ __forceinline__ float small_block_step(float mean_sq, float v_old, const SmallScalars &s,
@@ -104,6 +131,7 @@ template <int GD>
 __device__ __forceinline__ void small_body(const DevTensor &t, const Seg &seg, int64_t local,
                                            float *__restrict__ v, const SmallScalars &sc) {
     const float lr_wd = t.wd ? sc.lr_wd : 0.f;
+    const float gscale = effective_gscale(sc.gscale, sc.gscale_dev);
     float *vt = v + t.v_offset;
 
     if (seg.aux) {
@@ -113,7 +141,7 @@ __device__ __forceinline__ void small_body(const DevTensor &t, const Seg &seg, i
         for (int r = 0; r < kSmallUnitVec / (kThreads * 4); ++r) {
             const int64_t i = base + (static_cast<int64_t>(r) * kThreads + threadIdx.x) * 4;
             if (i >= t.numel) break;
-            const float4 g = load_g4<GD>(t.g, i);
+            const float4 g = load_g4<GD>(t.g, i, gscale);
             float4 m = *reinterpret_cast<const float4 *>(t.m + i);
             float4 p = *reinterpret_cast<const float4 *>(t.p + i);
             float4 vv = *reinterpret_cast<const float4 *>(vt + i);
@@ -125,6 +153,7 @@ __device__ __forceinline__ void small_body(const DevTensor &t, const Seg &seg, i
             *reinterpret_cast<float4 *>(t.m + i) = m;
             *reinterpret_cast<float4 *>(t.p + i) = p;
             *reinterpret_cast<float4 *>(vt + i) = vv;
+            if (t.p_bf16) store_bf16x4(t.p_bf16 + i, p);
         }
         return;
     }
@@ -140,7 +169,7 @@ __device__ __forceinline__ void small_body(const DevTensor &t, const Seg &seg, i
 #pragma unroll
         for (int k = 0; k < kSmallMaxL; ++k) {
             if (k < L) {
-                gl[k] = load_g1<GD>(t.g, e0 + k);
+                gl[k] = load_g1<GD>(t.g, e0 + k, gscale);
                 sum = fmaf(gl[k], gl[k], sum);
             }
         }
@@ -154,6 +183,7 @@ __device__ __forceinline__ void small_body(const DevTensor &t, const Seg &seg, i
                 update_one(gl[k], m, p, sc.beta1, sc.omb1, lr_wd, st);
                 t.m[e0 + k] = m;
                 t.p[e0 + k] = p;
+                if (t.p_bf16) store_bf16(t.p_bf16 + e0 + k, p);
             }
         }
     }
@@ -162,6 +192,7 @@ __device__ __forceinline__ void small_body(const DevTensor &t, const Seg &seg, i
 __global__ void __launch_bounds__(kThreads)
 small_kernel(const DevTensor *__restrict__ tensors, const Seg *__restrict__ segs, int n_segs,
              float *__restrict__ v, SmallScalars sc) {
+    if (step_skipped(sc.skip_flag)) return;
     const int64_t unit = blockIdx.x;
     const Seg seg = segs[find_seg(segs, n_segs, unit)];
     const DevTensor &t = tensors[seg.tensor];
@@ -200,13 +231,13 @@ __device__ __forceinline__ PieceRef decode_piece(const DevTensor *tensors, const
 // per accumulator); everything above a thread is double and combined in a
 // fixed order, so results do not depend on scheduling.
 template <int GD>
-__device__ __forceinline__ double piece_sum_sq(const PieceRef &r) {
+__device__ __forceinline__ double piece_sum_sq(const PieceRef &r, float gscale) {
     double tot = 0.0;
     if (r.vec) {
         float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
         int chain = 0;
         for (int64_t i = static_cast<int64_t>(threadIdx.x) * 4; i < r.n; i += kThreads * 4) {
-            const float4 g = load_g4<GD>(r.t->g, r.start + i);
+            const float4 g = load_g4<GD>(r.t->g, r.start + i, gscale);
             a0 = fmaf(g.x, g.x, a0); a1 = fmaf(g.y, g.y, a1);
             a2 = fmaf(g.z, g.z, a2); a3 = fmaf(g.w, g.w, a3);
             if (++chain == 64) {
@@ -222,7 +253,7 @@ __device__ __forceinline__ double piece_sum_sq(const PieceRef &r) {
         float a = 0.f;
         int chain = 0;
         for (int64_t i = threadIdx.x; i < r.n; i += kThreads) {
-            const float g = load_g1<GD>(r.t->g, r.start + i);
+            const float g = load_g1<GD>(r.t->g, r.start + i, gscale);
             a = fmaf(g, g, a);
             if (++chain == 64) { tot += static_cast<double>(a); a = 0.f; chain = 0; }
         }
@@ -233,10 +264,13 @@ __device__ __forceinline__ double piece_sum_sq(const PieceRef &r) {
 
 __global__ void __launch_bounds__(kThreads)
 twopass_partial_kernel(const DevTensor *__restrict__ tensors, const Seg *__restrict__ segs, int n_segs,
-                       double *__restrict__ partials) {
+                       double *__restrict__ partials, float gscale_host, const float *gscale_dev,
+                       const float *skip_flag) {
     __shared__ double warp_part[kThreads / 32];
+    if (step_skipped(skip_flag)) return;
+    const float gscale = effective_gscale(gscale_host, gscale_dev);
     const PieceRef r = decode_piece(tensors, segs, n_segs, blockIdx.x);
-    const double w = warp_sum(r.t->gdtype == AM_BF16 ? piece_sum_sq<AM_BF16>(r) : piece_sum_sq<AM_F32>(r));
+    const double w = warp_sum(r.t->gdtype == AM_BF16 ? piece_sum_sq<AM_BF16>(r, gscale) : piece_sum_sq<AM_F32>(r, gscale));
     if ((threadIdx.x & 31) == 0) warp_part[threadIdx.x >> 5] = w;
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -254,7 +288,7 @@ twopass_finalize_kernel(const DevTensor *__restrict__ tensors, const Seg *__rest
                         int64_t n_units, const double *__restrict__ partials,
                         float *__restrict__ block_steps, float *__restrict__ v, StepScalars sc) {
     const int64_t unit = static_cast<int64_t>(blockIdx.x) * (kThreads / 32) + (threadIdx.x >> 5);
-    if (unit >= n_units) return;
+    if (unit >= n_units || step_skipped(sc.skip_flag)) return;
     const int lane = threadIdx.x & 31;
     const Seg seg = segs[find_seg(segs, n_segs, unit)];
     const DevTensor &t = tensors[seg.tensor];
@@ -277,24 +311,27 @@ __device__ __forceinline__ void twopass_update_body(const PieceRef &r, const flo
     const DevTensor &t = *r.t;
     const float st = block_steps[t.block_base + r.block];
     const float lr_wd = t.wd ? sc.lr_wd : 0.f;
+    const float gscale = effective_gscale(sc.gscale, sc.gscale_dev);
     if (r.vec) {
         for (int64_t i = static_cast<int64_t>(threadIdx.x) * 4; i < r.n; i += kThreads * 4) {
             const int64_t e = r.start + i;
-            const float4 g = load_g4<GD>(t.g, e);
+            const float4 g = load_g4<GD>(t.g, e, gscale);
             float4 m = *reinterpret_cast<const float4 *>(t.m + e);
             float4 p = *reinterpret_cast<const float4 *>(t.p + e);
             update_four(g, m, p, sc.beta1, sc.omb1, lr_wd, st);
             *reinterpret_cast<float4 *>(t.m + e) = m;
             *reinterpret_cast<float4 *>(t.p + e) = p;
+            if (t.p_bf16) store_bf16x4(t.p_bf16 + e, p);
         }
     } else {
         for (int64_t i = threadIdx.x; i < r.n; i += kThreads) {
             const int64_t e = r.start + i;
-            const float g = load_g1<GD>(t.g, e);
+            const float g = load_g1<GD>(t.g, e, gscale);
             float m = t.m[e], p = t.p[e];
             update_one(g, m, p, sc.beta1, sc.omb1, lr_wd, st);
             t.m[e] = m;
             t.p[e] = p;
+            if (t.p_bf16) store_bf16(t.p_bf16 + e, p);
         }
     }
 }
@@ -302,6 +339,7 @@ __device__ __forceinline__ void twopass_update_body(const PieceRef &r, const flo
 __global__ void __launch_bounds__(kThreads)
 twopass_update_kernel(const DevTensor *__restrict__ tensors, const Seg *__restrict__ segs, int n_segs,
                       const float *__restrict__ block_steps, StepScalars sc) {
+    if (step_skipped(sc.skip_flag)) return;
     const PieceRef r = decode_piece(tensors, segs, n_segs, blockIdx.x);
     if (r.t->gdtype == AM_BF16) twopass_update_body<AM_BF16>(r, block_steps, sc);
     else twopass_update_body<AM_F32>(r, block_steps, sc);

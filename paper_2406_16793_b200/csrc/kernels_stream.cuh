@@ -60,7 +60,8 @@ struct StageMeta {          // written by the producer, read by the consumers
     int32_t kind;
     int32_t flags;
     int32_t v_shift;        // SF_V_STAGED: the first block's v sits at this index of the stage's v area
-    int32_t pad[3];
+    int32_t pad;
+    uint16_t *pb;           // bf16 copy of the updated parameters (nullptr: none)
 };
 static_assert(sizeof(StageMeta) == 64, "stage descriptor is 64 bytes");
 
@@ -218,10 +219,11 @@ __device__ __forceinline__ float stream_block_step(double sum_sq, double inv_L, 
 }
 
 // Elementwise update of n elements (n % 4 == 0) by `nthr` cooperating threads.
-template <int GD>
-__device__ __forceinline__ void apply_span(const unsigned char *gs, const float *ms, const float *ps,
-                                           float *mg, float *pg, int first, int n, int tid, int nthr,
-                                           float beta1, float omb1, float lr_wd, float step) {
+// The gradient scale is folded into `omb1` (= (1-beta1) * scale) by the caller.
+template <int GD, bool BF16_COPY>
+__device__ __forceinline__ void apply_span_impl(const unsigned char *gs, const float *ms, const float *ps,
+                                                float *mg, float *pg, uint16_t *pb, int first, int n, int tid,
+                                                int nthr, float beta1, float omb1, float lr_wd, float step) {
 #pragma unroll 2
     for (int i = first + tid * 4; i < first + n; i += nthr * 4) {
         const float4 g = lds_g4<GD>(gs, i);
@@ -230,7 +232,16 @@ __device__ __forceinline__ void apply_span(const unsigned char *gs, const float 
         update_four(g, m, p, beta1, omb1, lr_wd, step);
         __stcs(reinterpret_cast<float4 *>(mg + i), m);
         __stcs(reinterpret_cast<float4 *>(pg + i), p);
+        if (BF16_COPY) store_bf16x4(pb + i, p);
     }
+}
+
+template <int GD>
+__device__ __forceinline__ void apply_span(const unsigned char *gs, const float *ms, const float *ps,
+                                           float *mg, float *pg, uint16_t *pb, int first, int n, int tid, int nthr,
+                                           float beta1, float omb1, float lr_wd, float step) {
+    if (pb) apply_span_impl<GD, true>(gs, ms, ps, mg, pg, pb, first, n, tid, nthr, beta1, omb1, lr_wd, step);
+    else apply_span_impl<GD, false>(gs, ms, ps, mg, pg, pb, first, n, tid, nthr, beta1, omb1, lr_wd, step);
 }
 
 template <int GD>
@@ -281,6 +292,7 @@ template <bool CLUSTER>
 __global__ void __launch_bounds__(32 + kMaxConsumerWarps * 32, 1)
 stream_kernel(const __grid_constant__ StreamParams P) {
     extern __shared__ __align__(128) unsigned char smem[];
+    if (step_skipped(P.sc.skip_flag)) return;      // uniform over the grid: nobody reaches a barrier
     Control *ctl = reinterpret_cast<Control *>(smem);
     unsigned char *stages = smem + kCtrlBytes;
     float *v_areas = reinterpret_cast<float *>(stages + static_cast<size_t>(P.n_stages) * P.stage_bytes);
@@ -403,6 +415,7 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                     if (!(ok = acquire())) break;
                     StageMeta &mt = ctl->meta[stage];
                     mt.m = t.m + e0; mt.p = t.p + e0; mt.v = P.v + t.v_offset + b0;
+                    mt.pb = t.p_bf16 ? t.p_bf16 + e0 : nullptr;
                     mt.inv_L = 1.0 / static_cast<double>(t.L);
                     mt.n = n; mt.L = static_cast<int>(t.L); mt.kind = STAGE_PACKED; mt.flags = base_flags | SF_WRITE_V;
                     const uint32_t vbytes = stage_v(mt, t.v_offset + b0, nb);
@@ -424,7 +437,7 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                         const int c = static_cast<int>(slice - off < sum_cap ? slice - off : sum_cap);
                         if (!(ok = acquire())) break;
                         StageMeta &mt = ctl->meta[stage];
-                        mt.m = nullptr; mt.p = nullptr; mt.v = P.v + t.v_offset + local;
+                        mt.m = nullptr; mt.p = nullptr; mt.v = P.v + t.v_offset + local; mt.pb = nullptr;
                         mt.inv_L = 1.0 / static_cast<double>(t.L);
                         mt.n = c; mt.L = 0; mt.kind = STAGE_SUM;
                         mt.flags = base_flags | (off + c == slice ? SF_LAST : 0) | (crank == 0 ? SF_WRITE_V : 0);
@@ -442,6 +455,7 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                         if (!(ok = acquire())) break;
                         StageMeta &mt = ctl->meta[stage];
                         mt.m = t.m + e0 + off; mt.p = t.p + e0 + off; mt.v = nullptr;
+                        mt.pb = t.p_bf16 ? t.p_bf16 + e0 + off : nullptr;
                         mt.inv_L = 0.0;
                         mt.n = c; mt.L = 0; mt.kind = STAGE_APPLY; mt.flags = base_flags;
                         unsigned char *st = stages + static_cast<size_t>(stage) * P.stage_bytes;
@@ -474,7 +488,11 @@ stream_kernel(const __grid_constant__ StreamParams P) {
         const int lane = ctid & 31, warp = ctid >> 5;
         const int nthr = P.consumer_threads;
         if (ctid < nthr) {
-            const float beta1 = P.sc.beta1, omb1 = P.sc.omb1;
+            // the gradient scale s enters as (1-beta1)*s in the first moment and as s*s on the
+            // sums of squares, so the per-element work is the same with or without it
+            const float gscale = effective_gscale(P.sc.gscale, P.sc.gscale_dev);
+            const float beta1 = P.sc.beta1, omb1 = P.sc.omb1 * gscale;
+            const double gscale_sq = static_cast<double>(gscale) * static_cast<double>(gscale);
             int stage = 0;
             uint32_t phase = 0;
             GroupSync gsync{0u, 0};
@@ -509,10 +527,10 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                             float v_old = lane == 0 ? v_src[b] : 0.f;
                             v_old = __shfl_sync(0xffffffffu, v_old, 0);
                             float vn;
-                            const float step = stream_block_step(static_cast<double>(tot), mt.inv_L, v_old, P.sc, &vn);
+                            const float step = stream_block_step(static_cast<double>(tot) * gscale_sq, mt.inv_L, v_old, P.sc, &vn);
                             if (lane == 0) mt.v[b] = vn;
-                            if (bf16) apply_span<AM_BF16>(gs, ms, ps, mt.m, mt.p, e, L, lane, 32, beta1, omb1, lr_wd, step);
-                            else apply_span<AM_F32>(gs, ms, ps, mt.m, mt.p, e, L, lane, 32, beta1, omb1, lr_wd, step);
+                            if (bf16) apply_span<AM_BF16>(gs, ms, ps, mt.m, mt.p, mt.pb, e, L, lane, 32, beta1, omb1, lr_wd, step);
+                            else apply_span<AM_F32>(gs, ms, ps, mt.m, mt.p, mt.pb, e, L, lane, 32, beta1, omb1, lr_wd, step);
                         }
                     } else {
                         for (int b = 0; b < nb && alive; ++b) {
@@ -526,10 +544,10 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                                                  v_src + b, &tot, &v_old);
                             if (!alive) break;
                             float vn;
-                            const float step = stream_block_step(tot, mt.inv_L, v_old, P.sc, &vn);
+                            const float step = stream_block_step(tot * gscale_sq, mt.inv_L, v_old, P.sc, &vn);
                             if (ctid == 0) mt.v[b] = vn;
-                            if (bf16) apply_span<AM_BF16>(gs, ms, ps, mt.m, mt.p, e, L, ctid, nthr, beta1, omb1, lr_wd, step);
-                            else apply_span<AM_F32>(gs, ms, ps, mt.m, mt.p, e, L, ctid, nthr, beta1, omb1, lr_wd, step);
+                            if (bf16) apply_span<AM_BF16>(gs, ms, ps, mt.m, mt.p, mt.pb, e, L, ctid, nthr, beta1, omb1, lr_wd, step);
+                            else apply_span<AM_F32>(gs, ms, ps, mt.m, mt.p, mt.pb, e, L, ctid, nthr, beta1, omb1, lr_wd, step);
                         }
                     }
                     if (!alive) break;
@@ -566,12 +584,12 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                         }
                         ++long_count;
                         float vn;
-                        long_step = stream_block_step(tot, mt.inv_L, v_old, P.sc, &vn);
+                        long_step = stream_block_step(tot * gscale_sq, mt.inv_L, v_old, P.sc, &vn);
                         if (ctid == 0 && (mt.flags & SF_WRITE_V)) *mt.v = vn;
                     }
                 } else {   // STAGE_APPLY
-                    if (bf16) apply_span<AM_BF16>(gs, ms, ps, mt.m, mt.p, 0, mt.n, ctid, nthr, beta1, omb1, lr_wd, long_step);
-                    else apply_span<AM_F32>(gs, ms, ps, mt.m, mt.p, 0, mt.n, ctid, nthr, beta1, omb1, lr_wd, long_step);
+                    if (bf16) apply_span<AM_BF16>(gs, ms, ps, mt.m, mt.p, mt.pb, 0, mt.n, ctid, nthr, beta1, omb1, lr_wd, long_step);
+                    else apply_span<AM_F32>(gs, ms, ps, mt.m, mt.p, mt.pb, 0, mt.n, ctid, nthr, beta1, omb1, lr_wd, long_step);
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&ctl->empty[stage]);
                 }
