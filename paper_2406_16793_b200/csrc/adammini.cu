@@ -400,6 +400,7 @@ int adammini_step_ex(am_handle *h, void *const *params, const void *const *grads
             h->d_tensors, h->d_small_segs, h->n_small_segs, v, ss);
         AM_CUDA(h, cudaGetLastError());
     }
+    h->stream.bf16_copies = ex && ex->params_bf16;
     if (prof) AM_CUDA(h, cudaEventRecord(h->prof_ev[1], stream));
     AM_CUDA(h, h->stream.launch_main(h->d_tensors, v, sc, h->error_word, stream));
     if (prof) AM_CUDA(h, cudaEventRecord(h->prof_ev[2], stream));

@@ -236,11 +236,11 @@ __device__ __forceinline__ void apply_span_impl(const unsigned char *gs, const f
     }
 }
 
-template <int GD>
+template <int GD, bool COPY>
 __device__ __forceinline__ void apply_span(const unsigned char *gs, const float *ms, const float *ps,
                                            float *mg, float *pg, uint16_t *pb, int first, int n, int tid, int nthr,
                                            float beta1, float omb1, float lr_wd, float step) {
-    if (pb) apply_span_impl<GD, true>(gs, ms, ps, mg, pg, pb, first, n, tid, nthr, beta1, omb1, lr_wd, step);
+    if (COPY && pb) apply_span_impl<GD, true>(gs, ms, ps, mg, pg, pb, first, n, tid, nthr, beta1, omb1, lr_wd, step);
     else apply_span_impl<GD, false>(gs, ms, ps, mg, pg, pb, first, n, tid, nthr, beta1, omb1, lr_wd, step);
 }
 
@@ -288,7 +288,12 @@ __device__ __forceinline__ bool group_reduce(Control *ctl, GroupSync &gs, int *e
 }
 
 // ------------------------------------ kernel ------------------------------------
-template <bool CLUSTER>
+// Template parameters keep the code of one launch small (the consumer loop is
+// sensitive to instruction-cache misses): GDM says which gradient dtypes the
+// launch's tensors have, COPY whether any tensor wants a bf16 copy.
+enum GradMode : int { GDM_F32 = 0, GDM_BF16 = 1, GDM_MIXED = 2 };
+
+template <bool CLUSTER, int GDM, bool COPY>
 __global__ void __launch_bounds__(32 + kMaxConsumerWarps * 32, 1)
 stream_kernel(const __grid_constant__ StreamParams P) {
     extern __shared__ __align__(128) unsigned char smem[];
@@ -506,7 +511,7 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                 const unsigned char *gs = stages + static_cast<size_t>(stage) * P.stage_bytes;
                 const float *ms = reinterpret_cast<const float *>(gs + P.g_region_bytes);
                 const float *ps = ms + kStageElems;
-                const bool bf16 = (mt.flags & SF_BF16) != 0;
+                const bool bf16 = GDM == GDM_MIXED ? (mt.flags & SF_BF16) != 0 : GDM == GDM_BF16;
                 // where the old v of the stage's blocks is read from
                 const float *v_src = (mt.flags & SF_V_STAGED) ? v_areas + stage * kVAreaFloats + mt.v_shift : mt.v;
                 const float lr_wd = (mt.flags & SF_WD) ? P.sc.lr_wd : 0.f;
@@ -529,8 +534,8 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                             float vn;
                             const float step = stream_block_step(static_cast<double>(tot) * gscale_sq, mt.inv_L, v_old, P.sc, &vn);
                             if (lane == 0) mt.v[b] = vn;
-                            if (bf16) apply_span<AM_BF16>(gs, ms, ps, mt.m, mt.p, mt.pb, e, L, lane, 32, beta1, omb1, lr_wd, step);
-                            else apply_span<AM_F32>(gs, ms, ps, mt.m, mt.p, mt.pb, e, L, lane, 32, beta1, omb1, lr_wd, step);
+                            if (bf16) apply_span<AM_BF16, COPY>(gs, ms, ps, mt.m, mt.p, mt.pb, e, L, lane, 32, beta1, omb1, lr_wd, step);
+                            else apply_span<AM_F32, COPY>(gs, ms, ps, mt.m, mt.p, mt.pb, e, L, lane, 32, beta1, omb1, lr_wd, step);
                         }
                     } else {
                         for (int b = 0; b < nb && alive; ++b) {
@@ -546,8 +551,8 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                             float vn;
                             const float step = stream_block_step(tot * gscale_sq, mt.inv_L, v_old, P.sc, &vn);
                             if (ctid == 0) mt.v[b] = vn;
-                            if (bf16) apply_span<AM_BF16>(gs, ms, ps, mt.m, mt.p, mt.pb, e, L, ctid, nthr, beta1, omb1, lr_wd, step);
-                            else apply_span<AM_F32>(gs, ms, ps, mt.m, mt.p, mt.pb, e, L, ctid, nthr, beta1, omb1, lr_wd, step);
+                            if (bf16) apply_span<AM_BF16, COPY>(gs, ms, ps, mt.m, mt.p, mt.pb, e, L, ctid, nthr, beta1, omb1, lr_wd, step);
+                            else apply_span<AM_F32, COPY>(gs, ms, ps, mt.m, mt.p, mt.pb, e, L, ctid, nthr, beta1, omb1, lr_wd, step);
                         }
                     }
                     if (!alive) break;
@@ -588,8 +593,8 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                         if (ctid == 0 && (mt.flags & SF_WRITE_V)) *mt.v = vn;
                     }
                 } else {   // STAGE_APPLY
-                    if (bf16) apply_span<AM_BF16>(gs, ms, ps, mt.m, mt.p, mt.pb, 0, mt.n, ctid, nthr, beta1, omb1, lr_wd, long_step);
-                    else apply_span<AM_F32>(gs, ms, ps, mt.m, mt.p, mt.pb, 0, mt.n, ctid, nthr, beta1, omb1, lr_wd, long_step);
+                    if (bf16) apply_span<AM_BF16, COPY>(gs, ms, ps, mt.m, mt.p, mt.pb, 0, mt.n, ctid, nthr, beta1, omb1, lr_wd, long_step);
+                    else apply_span<AM_F32, COPY>(gs, ms, ps, mt.m, mt.p, mt.pb, 0, mt.n, ctid, nthr, beta1, omb1, lr_wd, long_step);
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&ctl->empty[stage]);
                 }
@@ -622,10 +627,28 @@ inline void stream_add_tensor(StreamPlanInput &in, int index, const am_table_row
     (path == PATH_STREAM ? in.stream_tensors : in.cluster_tensors).push_back({index, r});
 }
 
+typedef void (*StreamKernelFn)(const StreamParams);
+
+template <bool CLUSTER>
+inline StreamKernelFn stream_kernel_for(int gdm, bool copy) {
+    switch (gdm * 2 + (copy ? 1 : 0)) {
+    case 0: return stream_kernel<CLUSTER, GDM_F32, false>;
+    case 1: return stream_kernel<CLUSTER, GDM_F32, true>;
+    case 2: return stream_kernel<CLUSTER, GDM_BF16, false>;
+    case 3: return stream_kernel<CLUSTER, GDM_BF16, true>;
+    case 4: return stream_kernel<CLUSTER, GDM_MIXED, false>;
+    default: return stream_kernel<CLUSTER, GDM_MIXED, true>;
+    }
+}
+inline StreamKernelFn stream_kernel_for(bool cluster, int gdm, bool copy) {
+    return cluster ? stream_kernel_for<true>(gdm, copy) : stream_kernel_for<false>(gdm, copy);
+}
+
 struct StreamLaunch {
     std::vector<StreamSeg> segs;     // with sentinel
     std::vector<int64_t> bounds;
     int grid = 0, cluster = 1, n_stages = 0, stage_bytes = 0, g_region_bytes = 0, threads = 0, chunk = 0;
+    int gdm = GDM_MIXED;
     unsigned long long *d_counter = nullptr;
     const StreamSeg *d_segs = nullptr;
     const int64_t *d_bounds = nullptr;
@@ -663,6 +686,7 @@ struct StreamPlan {
     }
 
     int64_t v_len = 0;
+    bool bf16_copies = false;      // set per step: some tensor has a bf16 copy to write
 
     cudaError_t launch_one(const StreamLaunch &L, bool cluster, const DevTensor *tensors, float *v,
                            const StepScalars &sc, int *error_word, cudaStream_t stream) const {
@@ -689,9 +713,8 @@ struct StreamPlan {
             attr[0].val.clusterDim.z = 1;
             cfg.attrs = attr;
             cfg.numAttrs = 1;
-            return cudaLaunchKernelEx(&cfg, stream_kernel<true>, P);
         }
-        return cudaLaunchKernelEx(&cfg, stream_kernel<false>, P);
+        return cudaLaunchKernelEx(&cfg, stream_kernel_for(cluster, L.gdm, bf16_copies), P);
     }
 
     cudaError_t launch_main(const DevTensor *tensors, float *v, const StepScalars &sc, int *error_word,
@@ -711,8 +734,12 @@ inline void stream_build_launch(const std::vector<StreamPlanInput::Item> &tensor
     out->bounds.clear();
     out->grid = 0;
     if (tensors.empty() || workers <= 0) return;
-    bool any_f32 = false;
-    for (const auto &it : tensors) any_f32 |= it.row.grad_dtype == AM_F32;
+    bool any_f32 = false, any_bf16 = false;
+    for (const auto &it : tensors) {
+        any_f32 |= it.row.grad_dtype == AM_F32;
+        any_bf16 |= it.row.grad_dtype == AM_BF16;
+    }
+    out->gdm = any_f32 && any_bf16 ? GDM_MIXED : (any_bf16 ? GDM_BF16 : GDM_F32);
     out->g_region_bytes = kStageElems * (any_f32 ? 4 : 2);
     out->stage_bytes = out->g_region_bytes + kStageElems * 8;
     out->n_stages = std::min<int>(kMaxStages, static_cast<int>((kSmemBudget - kCtrlBytes) / (out->stage_bytes + kVAreaFloats * 4)));
@@ -787,7 +814,7 @@ inline void stream_probe_cluster(int sm_count, int threads, int wanted, int *clu
         cfg.attrs = attr;
         cfg.numAttrs = 1;
         int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, stream_kernel<true>, &cfg) == cudaSuccess && n > 0) {
+        if (cudaOccupancyMaxActiveClusters(&n, stream_kernel<true, GDM_MIXED, true>, &cfg) == cudaSuccess && n > 0) {
             *cluster_size = cs;
             *n_clusters = n;
             return;
@@ -834,11 +861,15 @@ inline void stream_finish_plan(const StreamPlanInput &in, int cluster_size, int 
 }
 
 inline cudaError_t stream_configure_kernels() {
-    cudaError_t e = cudaFuncSetAttribute(stream_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         static_cast<int>(kSmemBudget));
-    if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(stream_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                static_cast<int>(kSmemBudget));
+    for (int cluster = 0; cluster < 2; ++cluster)
+        for (int gdm = 0; gdm < 3; ++gdm)
+            for (int copy = 0; copy < 2; ++copy) {
+                const cudaError_t e = cudaFuncSetAttribute(stream_kernel_for(cluster != 0, gdm, copy != 0),
+                                                           cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                           static_cast<int>(kSmemBudget));
+                if (e != cudaSuccess) return e;
+            }
+    return cudaSuccess;
 }
 
 }  // namespace am
