@@ -19,7 +19,9 @@ import torch
 
 import paper_2406_16793_b200 as am
 from oracle import step as ostep
-from paper_2406_16793_b200 import workloads as W
+from paper_2406_16793_b200 import build as _lib_build, workloads as W
+
+_lib_build.build()      # compile the CUDA library if the shared object is missing or older than its sources
 
 TOL = 1e-5
 GUARD = 64          # float32 guard words either side of every test buffer
@@ -222,5 +224,37 @@ def run_sampled_parity(w: W.Workload, steps: int, tensor_indices: Sequence[int],
         worst["p"] = max(worst["p"], block_relative_error(dev.p[i][sl].cpu().numpy(), po, L))
         worst["m"] = max(worst["m"], block_relative_error(dev.m[i][sl].cpu().numpy(), mo, L))
         worst["v"] = max(worst["v"], v_relative_error(dev.v[v_off[i] + b:v_off[i] + b + 1].cpu().numpy(), vo))
+    opt.close()
+    return worst
+
+
+def run_sampled_runs(w: W.Workload, steps: int, run_elems: int, n_runs: int, device="cuda") -> Dict[str, float]:
+    """Full-size run of a one-tensor workload with short blocks; the oracle
+    recomputes `n_runs` aligned runs of `run_elems` elements (whole blocks):
+    the first, the last and seeded-random ones."""
+    t = w.tensors[0]
+    L = t.block_len
+    assert len(w.tensors) == 1 and run_elems % L == 0 and t.numel % run_elems == 0
+    dev = DeviceState(w, device, guarded=False)
+    opt = make_optimizer(w)
+    rng = np.random.default_rng(W.mix_seed(W.BASE_SEED, w.config_id, L) % (1 << 32))
+    n_slots = t.numel // run_elems
+    picks = sorted({0, n_slots - 1} | {int(x) for x in rng.integers(0, n_slots, n_runs - 2)})
+    samples = []
+    for k in picks:
+        sl = slice(k * run_elems, (k + 1) * run_elems)
+        samples.append([sl, ostep.widen(dev.p[0][sl].cpu()), np.zeros(run_elems), np.zeros(run_elems // L)])
+    for step in range(1, steps + 1):
+        dev.draw_grads(step)
+        opt.step(dev.p, dev.g, dev.m, dev.v, step)
+        for sl, po, mo, vo in samples:
+            ostep.adammini_step(po, mo, vo, dev.g[0][sl].cpu(), L, step=step, **w.hparams)
+    opt.sync_status()
+    worst = {"p": 0.0, "m": 0.0, "v": 0.0, "blocks": len(samples) * (run_elems // L)}
+    for sl, po, mo, vo in samples:
+        worst["p"] = max(worst["p"], block_relative_error(dev.p[0][sl].cpu().numpy(), po, L))
+        worst["m"] = max(worst["m"], block_relative_error(dev.m[0][sl].cpu().numpy(), mo, L))
+        vs = slice(sl.start // L, sl.stop // L)
+        worst["v"] = max(worst["v"], v_relative_error(dev.v[vs].cpu().numpy(), vo))
     opt.close()
     return worst

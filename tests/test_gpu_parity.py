@@ -249,3 +249,50 @@ def test_dynamic_work_distribution_gives_identical_bits(chunk):
     opt.sync_status()
     opt.close()
     assert _same(a, dev)
+
+
+def test_gpt2_small_full_model_hundred_steps():
+    """All 124 M parameters of the GPT-2-small shape set (196 tensors, bf16
+    gradients), 100 steps, every element compared with the oracle."""
+    H.assert_parity(H.run_parity(W.gpt2_small(), steps=100))
+
+
+def _need_free_memory(gib):
+    free, _ = torch.cuda.mem_get_info()
+    if free < gib * (1 << 30):
+        pytest.skip(f"needs about {gib} GiB of free device memory")
+
+
+def test_full_size_llama3_8b_sampled_blocks():
+    """All 8.03 G parameters of the Llama-3-8B shape set (grouped KV heads,
+    14336-element rows, Zipf-scaled vocabulary rows), stepped as the benchmark
+    steps them; the oracle recomputes sampled blocks of every kind."""
+    _need_free_memory(90)
+    w = W.llama3_8b()
+    picks = [0, len(w.tensors) - 1, len(w.tensors) - 2]
+    for layer in (0, 31):
+        picks += list(range(1 + 9 * layer, 1 + 9 * (layer + 1)))
+    worst = H.run_sampled_parity(w, steps=3, tensor_indices=picks, blocks_per_tensor=3)
+    assert worst["blocks"] >= 40
+    H.assert_parity(worst)
+
+
+@pytest.mark.parametrize("L", [1, 128, 4096, 524288])
+def test_full_size_flat_sweep_sampled_blocks(L):
+    """One flat fp32 tensor of 2^30 elements at every block length of the
+    partition-degeneracy sweep; the oracle recomputes sampled runs of blocks."""
+    _need_free_memory(20)
+    w = W.flat_sweep(L)
+    if L < 4096:
+        # sample runs of 4096/L consecutive blocks by viewing them as one tensor of short blocks
+        worst = H.run_sampled_runs(w, steps=3, run_elems=4096, n_runs=24)
+    else:
+        worst = H.run_sampled_parity(w, steps=3, tensor_indices=[0], blocks_per_tensor=6)
+    H.assert_parity(worst)
+
+
+def test_full_size_whole_tensor_block():
+    """2^30 elements as ONE block (the two-pass path at full size): the oracle
+    runs the whole tensor for two steps."""
+    _need_free_memory(20)
+    H.assert_parity(H.run_parity(W.flat_sweep(1 << 30), steps=2))
