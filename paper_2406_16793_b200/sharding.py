@@ -9,9 +9,10 @@ and the tensor descriptors a rank hands to the library for its pieces.
 from __future__ import annotations
 
 from dataclasses import dataclass
+from math import gcd
 from typing import List, Sequence
 
-from .workloads import FIXED, TensorSpec
+from .workloads import BF16, FIXED, TensorSpec
 
 
 @dataclass(frozen=True)
@@ -61,6 +62,11 @@ def shard_by_blocks(tensors: Sequence[TensorSpec], world_size: int) -> List[List
             target = total * (rank + 1) // world_size
             room = target - done
             take = nb - b if rank == world_size - 1 else min(nb - b, max(0, (room + L // 2) // L))
+            if take < nb - b:
+                # a cut inside a tensor must leave every piece 16-byte aligned (8 bf16 or 4 fp32 elements)
+                step = 8 // gcd(L, 8)
+                take = ((b + take) // step) * step - b
+                take = max(take, 0)
             if take == 0:
                 if rank < world_size - 1:
                     rank += 1
@@ -73,3 +79,43 @@ def shard_by_blocks(tensors: Sequence[TensorSpec], world_size: int) -> List[List
                 rank += 1
         v_off += nb
     return out
+
+
+class ShardedStep:
+    """One rank's share of an Adam-mini step: the rank's pieces as a partition
+    of their own, stepped through the library on views of the full tensors.
+
+    Every rank holds (or can address) the full parameter, gradient and moment
+    tensors and updates only its blocks; after the step a trainer all-gathers
+    the updated parameters (outside this class).  v is sharded: the rank keeps
+    only the second moments of its own blocks.
+    """
+
+    def __init__(self, tensors: Sequence[TensorSpec], world_size: int, rank: int, **hparams):
+        from . import binding
+        self.tensors = list(tensors)
+        self.pieces = shard_by_blocks(self.tensors, world_size)[rank]
+        self.specs = [p.spec(self.tensors[p.tensor]) for p in self.pieces]
+        self.partition = binding.Partition(self.specs)
+        self.optimizer = binding.AdamMini(self.partition, **hparams)
+        self.local_blocks = sum(p.block_end - p.block_begin for p in self.pieces)
+
+    def _views(self, full, grads: bool):
+        out = []
+        for p in self.pieces:
+            t = self.tensors[p.tensor]
+            item = (2 if t.grad_dtype == BF16 else 4) if grads else 4
+            x = full[p.tensor]
+            base = int(x.data_ptr()) if hasattr(x, "data_ptr") else int(x)
+            out.append(base + p.elem_begin * item)
+        return out
+
+    def step(self, params, grads, m, v_local, step: int, stream: int = 0) -> None:
+        """params/grads/m: the FULL tensors in table order (device tensors or raw
+        addresses); v_local: float32[self.local_blocks] of this rank."""
+        self.optimizer.step(self._views(params, False), self._views(grads, True), self._views(m, False),
+                            v_local, step, stream)
+
+    def close(self) -> None:
+        self.optimizer.close()
+        self.partition.close()

@@ -296,3 +296,26 @@ def test_full_size_whole_tensor_block():
     runs the whole tensor for two steps."""
     _need_free_memory(20)
     H.assert_parity(H.run_parity(W.flat_sweep(1 << 30), steps=2))
+
+
+@pytest.mark.parametrize("world", [2, 3])
+def test_sharded_ranks_tile_the_unsharded_step(world):
+    """Whole-block sharding: every rank's share is stepped on its own (here one
+    after the other on the one GPU; the shares do not interact), and together
+    they must reproduce the unsharded step bit for bit."""
+    from paper_2406_16793_b200 import sharding
+    w = W.scaled_rows(W.llama2_7b(n_layers=1, vocab=300), 200)
+    ref = _run_steps(w, 1, 3)
+    dev = H.DeviceState(w, guarded=False)
+    ranks = [sharding.ShardedStep(w.tensors, world, r, **w.hparams) for r in range(world)]
+    v_local = [torch.zeros(max(r.local_blocks, 1), device="cuda") for r in ranks]
+    for t in (1, 2, 3):
+        dev.draw_grads(t)
+        for r, v in zip(ranks, v_local):
+            r.step(dev.p, dev.g, dev.m, v, t)
+    torch.cuda.synchronize()
+    assert all(torch.equal(a, b) for a, b in zip(ref.p + ref.m, dev.p + dev.m))
+    v_all = torch.cat([v[:r.local_blocks] for r, v in zip(ranks, v_local)])
+    assert torch.equal(v_all, ref.v)
+    for r in ranks:
+        r.close()
