@@ -98,6 +98,61 @@ int oracle_adammini_step(double *p, double *m, double *v, const void *g,
     return 0;
 }
 
+/*
+ * The paper's ablation of the block statistic (appendix "Ablation Studies on
+ * the Design of Adam-mini"): instead of the mean of g*g the block's learning
+ * rate is built from the max, the min, the 1-norm or the 2-norm.  The paper
+ * names the quantities only; the reading taken here is that the statistic of
+ * the vector g_b*g_b replaces mean(g_b*g_b) in the v rule, so that v stays
+ * one scalar per block:
+ *   statistic 0: mean(g*g)   1: max(g*g)   2: min(g*g)
+ *   statistic 3: sum(g*g)    (1-norm of a non-negative vector)
+ *   statistic 4: sqrt(sum((g*g)^2))   (2-norm)
+ * Everything else is Algorithm 1 as above.
+ */
+int oracle_adammini_step_stat(double *p, double *m, double *v, const void *g,
+                              int g_dtype, int64_t numel, int64_t L, double lr,
+                              double beta1, double beta2, double eps, double wd,
+                              int apply_wd, int64_t t, int statistic)
+{
+    if (!p || !m || !v || !g || numel < 0 || L <= 0 || numel % L != 0 || t < 1 ||
+        statistic < 0 || statistic > 4)
+        return -1;
+    const double bc1 = 1.0 - pow(beta1, (double)t);
+    const double bc2 = 1.0 - pow(beta2, (double)t);
+    const int64_t n_blocks = numel / L;
+
+    for (int64_t b = 0; b < n_blocks; ++b) {
+        const int64_t lo = b * L;
+        double acc = 0.0;
+        for (int64_t i = 0; i < L; ++i) {
+            const double gi = grad_at(g, g_dtype, lo + i);
+            const double sq = gi * gi;
+            if (statistic == 0 || statistic == 3) acc = acc + sq;
+            else if (statistic == 1) acc = (i == 0 || sq > acc) ? sq : acc;
+            else if (statistic == 2) acc = (i == 0 || sq < acc) ? sq : acc;
+            else acc = acc + sq * sq;
+        }
+        double stat = acc;
+        if (statistic == 0) stat = acc / (double)L;
+        if (statistic == 4) stat = sqrt(acc);
+        v[b] = (1.0 - beta2) * stat + beta2 * v[b];
+        const double v_hat = v[b] / bc2;
+        const double denom = sqrt(v_hat) + eps;
+
+        for (int64_t i = 0; i < L; ++i) {
+            const int64_t k = lo + i;
+            const double gi = grad_at(g, g_dtype, k);
+            if (apply_wd)
+                p[k] = p[k] - lr * wd * p[k];
+            m[k] = (1.0 - beta1) * gi + beta1 * m[k];
+            const double m_hat = m[k] / bc1;
+            p[k] = p[k] - lr * m_hat / denom;
+        }
+    }
+    return 0;
+}
+
 /* Exact widening helpers so Python callers can build float64 state from the
  * bits handed to the GPU without going through another library. */
 void oracle_widen_f32(const float *src, double *dst, int64_t n)

@@ -28,8 +28,24 @@ def sqrt_fraction(x: Fraction, bits: int = SQRT_BITS) -> Fraction:
     return Fraction(isqrt(scaled), 1 << (shift // 2))
 
 
+def block_statistic(squares: Sequence[Fraction], statistic: int) -> Fraction:
+    """mean (0), max (1), min (2), sum (3) or 2-norm (4) of a block's g*g values."""
+    if statistic == 0:
+        return sum(squares, Fraction(0)) / len(squares)
+    if statistic == 1:
+        return max(squares)
+    if statistic == 2:
+        return min(squares)
+    if statistic == 3:
+        return sum(squares, Fraction(0))
+    if statistic == 4:
+        return sqrt_fraction(sum((x * x for x in squares), Fraction(0)))
+    raise ValueError("unknown statistic")
+
+
 def adammini_exact(p: Sequence, g_steps: Sequence[Sequence], blocks: Sequence[Sequence[int]], *,
-                   lr, beta1, beta2, eps, weight_decay) -> tuple[List[Fraction], List[Fraction], List[Fraction]]:
+                   lr, beta1, beta2, eps, weight_decay,
+                   statistic: int = 0) -> tuple[List[Fraction], List[Fraction], List[Fraction]]:
     """Run len(g_steps) Adam-mini steps exactly.
 
     p: initial parameters; g_steps[t-1][i]: gradient of element i at step t;
@@ -45,7 +61,7 @@ def adammini_exact(p: Sequence, g_steps: Sequence[Sequence], blocks: Sequence[Se
     for t, g in enumerate(g_steps, start=1):
         g = [F(x) for x in g]
         for b, idx in enumerate(blocks):
-            mean_sq = sum((g[i] * g[i] for i in idx), F(0)) / len(idx)
+            mean_sq = block_statistic([g[i] * g[i] for i in idx], statistic)
             for i in idx:
                 p[i] = p[i] - lr * lam * p[i]
                 m[i] = (1 - beta1) * g[i] + beta1 * m[i]

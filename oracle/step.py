@@ -30,6 +30,8 @@ def load(path: str | None = None) -> ctypes.CDLL:
         ctypes.c_double, ctypes.c_double, ctypes.c_double, ctypes.c_double,
         ctypes.c_double, ctypes.c_int, ctypes.c_int64,
     ]
+    lib.oracle_adammini_step_stat.restype = ctypes.c_int
+    lib.oracle_adammini_step_stat.argtypes = lib.oracle_adammini_step.argtypes + [ctypes.c_int]
     lib.oracle_widen_f32.restype = None
     lib.oracle_widen_f32.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64]
     lib.oracle_widen_bf16.restype = None
@@ -66,8 +68,11 @@ def _grad_view(g) -> tuple[np.ndarray, int]:
 def adammini_step(p: np.ndarray, m: np.ndarray, v: np.ndarray, g, block_len: int, *,
                   lr: float, beta1: float, beta2: float, eps: float,
                   weight_decay: float, step: int, apply_wd: bool = True,
-                  lib: ctypes.CDLL | None = None) -> None:
-    """One Adam-mini step (Algorithm 1) on one tensor, in place, float64 state."""
+                  lib: ctypes.CDLL | None = None, statistic: int = 0) -> None:
+    """One Adam-mini step (Algorithm 1) on one tensor, in place, float64 state.
+
+    statistic != 0 selects the ablation variants of the block statistic
+    (1 max, 2 min, 3 one-norm, 4 two-norm of g*g), a separate C routine."""
     lib = lib or load()
     for a in (p, m, v):
         if a.dtype != np.float64 or not a.flags.c_contiguous:
@@ -76,10 +81,13 @@ def adammini_step(p: np.ndarray, m: np.ndarray, v: np.ndarray, g, block_len: int
     n = p.size
     if m.size != n or gv.size != n or n % block_len or v.size != n // block_len:
         raise ValueError("shape mismatch")
-    rc = lib.oracle_adammini_step(
-        p.ctypes.data, m.ctypes.data, v.ctypes.data, gv.ctypes.data, code, n,
-        int(block_len), float(lr), float(beta1), float(beta2), float(eps),
-        float(weight_decay), int(bool(apply_wd)), int(step))
+    args = (p.ctypes.data, m.ctypes.data, v.ctypes.data, gv.ctypes.data, code, n,
+            int(block_len), float(lr), float(beta1), float(beta2), float(eps),
+            float(weight_decay), int(bool(apply_wd)), int(step))
+    if statistic:
+        rc = lib.oracle_adammini_step_stat(*args, int(statistic))
+    else:
+        rc = lib.oracle_adammini_step(*args)
     if rc != 0:
         raise ValueError(f"oracle_adammini_step rejected its arguments (rc={rc})")
 

@@ -252,3 +252,98 @@ ALL_CHECKS = (
     check_brute_force_exact,
     check_widening,
 )
+
+
+# =============================================================================
+# The ablation variants of the block statistic (max, min, 1-norm, 2-norm of g*g)
+# =============================================================================
+STATS = (1, 2, 3, 4)
+
+
+def run_stat(lib, p0, g_steps, L, statistic, hp=HP):
+    p = np.array(p0, dtype=np.float64)
+    m = np.zeros_like(p)
+    v = np.zeros(p.size // L, dtype=np.float64)
+    for t, g in enumerate(g_steps, start=1):
+        ostep.adammini_step(p, m, v, np.asarray(g, dtype=np.float64), L, step=t, lib=lib,
+                            statistic=statistic, **hp)
+    return p, m, v
+
+
+# -- with one element per block every statistic of {g*g} is g*g: AdamW again, bit for bit
+#    (sqrt(x*x) = |x| exactly in IEEE arithmetic, so this holds for the 2-norm too) --------
+def check_stat_reduces_to_adamw(lib):
+    rng = np.random.default_rng(31)
+    n = 129
+    p0 = rng.normal(0, 0.02, n)
+    gs = [rng.normal(0, 1, n) * 10.0 ** rng.uniform(-3, 0, n) for _ in range(5)]
+    pa, ma, va = p0.copy(), np.zeros(n), np.zeros(n)
+    for t, g in enumerate(gs, start=1):
+        adamw_ref.adamw_step(pa, ma, va, g, step=t, **HP)
+    for s in STATS:
+        p, m, v = run_stat(lib, p0, gs, 1, s)
+        assert np.array_equal(p, pa) and np.array_equal(m, ma) and np.array_equal(v, va), s
+
+
+# -- |g| = c on a block: max = min = c^2, 1-norm = L c^2, 2-norm = sqrt(L) c^2, constant in t,
+#    so v_hat = k c^2 and p_T = a^T p_0 - eta sign(g) c / (sqrt(k) c + eps) (1-a^T)/(1-a) -------
+def check_stat_closed_form(lib):
+    rng = np.random.default_rng(32)
+    L, nb, T = 9, 3, 12
+    p0 = rng.normal(0, 0.02, L * nb)
+    c = np.repeat([0.5, 3e-3, 7.0], L)
+    sgn = np.sign(rng.normal(size=L * nb))
+    g = c * sgn
+    a = 1 - HP["lr"] * HP["weight_decay"]
+    for s, k in ((1, 1.0), (2, 1.0), (3, float(L)), (4, math.sqrt(L))):
+        p, m, v = run_stat(lib, p0, [g] * T, L, s)
+        assert _rel(v, k * c[::L] ** 2 * (1 - HP["beta2"] ** T)) < 1e-12, s
+        want = a ** T * p0 - HP["lr"] * sgn * c / (math.sqrt(k) * c + HP["eps"]) * (1 - a ** T) / (1 - a)
+        assert _rel(p, want) < 1e-11, s
+
+
+# -- against numpy on random data: the EMA of numpy's own max / min / sum / 2-norm --------
+def check_stat_against_numpy(lib):
+    rng = np.random.default_rng(33)
+    L, nb, T = 16, 5, 6
+    p0 = rng.normal(0, 0.02, L * nb)
+    gs = [rng.normal(0, 1, L * nb) for _ in range(T)]
+    fns = {1: lambda q: q.max(axis=1), 2: lambda q: q.min(axis=1), 3: lambda q: q.sum(axis=1),
+           4: lambda q: np.sqrt((q * q).sum(axis=1))}
+    v_mean = run(lib, p0, gs, L)[2]
+    for s in STATS:
+        p, m, v = run_stat(lib, p0, gs, L, s)
+        want = np.zeros(nb)
+        for g in gs:
+            want = (1 - HP["beta2"]) * fns[s]((g * g).reshape(nb, L)) + HP["beta2"] * want
+        assert _rel(v, want) < 1e-13, s
+        # the last step's parameter change uses eta m_hat / (sqrt(v_hat) + eps)
+        p_prev, m_prev, _ = run_stat(lib, p0, gs[:-1], L, s)
+        m_new = (1 - HP["beta1"]) * gs[-1] + HP["beta1"] * m_prev
+        denom = np.repeat(np.sqrt(want / (1 - HP["beta2"] ** T)), L) + HP["eps"]
+        expect = p_prev * (1 - HP["lr"] * HP["weight_decay"]) - HP["lr"] * (m_new / (1 - HP["beta1"] ** T)) / denom
+        assert _rel(p, expect) < 1e-12, s
+    v_max, v_min = run_stat(lib, p0, gs, L, 1)[2], run_stat(lib, p0, gs, L, 2)[2]
+    assert (v_max >= v_mean).all() and (v_mean >= v_min).all()
+    assert np.array_equal(run_stat(lib, p0, gs, L, 3)[2], L * v_mean)        # L = 16: scaling by L is exact
+
+
+def check_stat_brute_force_exact(lib):
+    rng = np.random.default_rng(34)
+    for s in STATS:
+        for n in (2, 3, 4, 6):
+            p0 = list(rng.normal(0, 0.02, n))
+            for L in [d for d in range(1, n + 1) if n % d == 0]:
+                for _ in range(8):
+                    gs = [list(rng.choice(GRAD_VALUES, n)) for _ in range(2)]
+                    p, m, v = run_stat(lib, p0, gs, L, s)
+                    blocks = [list(range(b * L, (b + 1) * L)) for b in range(n // L)]
+                    pe, me, ve = exact.adammini_exact(p0, gs, blocks, statistic=s, **HP)
+                    for got, want, floor in ((p, pe, 1e-3), (m, me, 0.0), (v, ve, 0.0)):
+                        for x, y in zip(got, want):
+                            y = float(y)
+                            assert abs(x - y) <= 4e-15 * max(abs(y), floor) + 1e-300, (s, L, gs)
+
+
+STAT_CHECKS = (check_stat_reduces_to_adamw, check_stat_closed_form, check_stat_against_numpy,
+               check_stat_brute_force_exact)

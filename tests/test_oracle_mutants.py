@@ -28,13 +28,44 @@ MUTANTS = {
 }
 
 
-@pytest.mark.parametrize("name", sorted(MUTANTS))
-def test_mutant_is_caught(tmp_path, name):
-    old, new = MUTANTS[name]
+STAT_MUTANTS = {
+    "max_is_min": ("(i == 0 || sq > acc) ? sq : acc", "(i == 0 || sq < acc) ? sq : acc"),
+    "min_is_max": ("(i == 0 || sq < acc) ? sq : acc", "(i == 0 || sq > acc) ? sq : acc"),
+    "two_norm_without_root": ("if (statistic == 4) stat = sqrt(acc);", ";"),
+    "two_norm_of_g_not_gg": ("else acc = acc + sq * sq;", "else acc = acc + sq;"),
+    "one_norm_divided": ("if (statistic == 0) stat = acc / (double)L;", "if (statistic == 0 || statistic == 3) stat = acc / (double)L;"),
+    "stat_first_element_only": ("if (statistic == 0 || statistic == 3) acc = acc + sq;", "if (statistic == 0 || statistic == 3) acc = sq;"),
+    "stat_v_not_averaged": ("v[b] = (1.0 - beta2) * stat + beta2 * v[b];", "v[b] = stat;"),
+}
+
+
+@pytest.mark.parametrize("name", sorted(STAT_MUTANTS))
+def test_statistic_mutant_is_caught(tmp_path, name):
+    old, new = STAT_MUTANTS[name]
     src = open(obuild.SOURCE).read()
     assert src.count(old) == 1, f"mutation site for {name} not unique"
     cfile = tmp_path / "mutant.c"
     cfile.write_text(src.replace(old, new))
+    so = tmp_path / f"mutant_{name}.so"
+    subprocess.run(["gcc", *obuild.CFLAGS, "-o", str(so), str(cfile), "-lm"], check=True)
+    lib = ostep.load(str(so))
+    caught = []
+    for check in pins.STAT_CHECKS:
+        try:
+            check(lib)
+        except (AssertionError, ValueError, FloatingPointError):
+            caught.append(check.__name__)
+    assert caught, f"no pin noticed the mutant '{name}'"
+
+
+@pytest.mark.parametrize("name", sorted(MUTANTS))
+def test_mutant_is_caught(tmp_path, name):
+    old, new = MUTANTS[name]
+    src = open(obuild.SOURCE).read()
+    main_end = src.index("oracle_adammini_step_stat")       # mutate Algorithm 1's routine, which comes first
+    assert src[:main_end].count(old) == 1, f"mutation site for {name} not unique"
+    cfile = tmp_path / "mutant.c"
+    cfile.write_text(src.replace(old, new, 1))
     so = tmp_path / f"mutant_{name}.so"
     subprocess.run(["gcc", *obuild.CFLAGS, "-o", str(so), str(cfile), "-lm"], check=True)
     lib = ostep.load(str(so))

@@ -20,6 +20,12 @@ def test_pin(lib, check):
     check(lib)
 
 
+@pytest.mark.parametrize("check", pins.STAT_CHECKS, ids=lambda f: f.__name__)
+def test_statistic_variant_pin(lib, check):
+    """The ablation statistics (max, min, 1-norm, 2-norm of g*g) of the paper's appendix."""
+    check(lib)
+
+
 def test_five_parameter_example_from_paper(lib):
     """Section 2.1 example: partition (1,2,3),(4,5); the per-block step size is
     eta / sqrt(mean of Adam's v over the block)."""
