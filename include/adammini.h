@@ -225,6 +225,11 @@ typedef enum {
                                  time; 1000000 = every CTA walks its own fixed, cost-balanced range.
                                  Results are bit-identical in every mode */
     , AM_OPT_CLUSTER_CHUNK = 6 /* the same for the cluster kernel, in blocks handed to a cluster at a time */
+    , AM_OPT_STATISTIC = 7     /* block statistic that feeds v: 0 = mean(g*g), Algorithm 1.  The ablation
+                                  of the paper's appendix ("Ablation Studies on the Design of Adam-mini"),
+                                  which it reports to train worse: 1 = max, 2 = min, 3 = 1-norm (sum),
+                                  4 = 2-norm of the vector g*g.  Non-zero values run on the two-pass
+                                  kernels (g read twice) */
 } am_option;
 int adammini_set_option(am_handle *h, int32_t key, int64_t value);
 

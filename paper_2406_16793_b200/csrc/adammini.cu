@@ -20,7 +20,7 @@ using namespace am;
 
 namespace {
 
-constexpr int kNumOptions = 7;
+constexpr int kNumOptions = 8;
 
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
@@ -91,7 +91,7 @@ int build_plan(am_handle *h) {
 
         int path;
         if (r.block_len <= kSmallMaxL) path = PATH_SMALL;
-        else if (h->opt[AM_OPT_PATH] == 1) path = PATH_TWOPASS;
+        else if (h->opt[AM_OPT_PATH] == 1 || h->opt[AM_OPT_STATISTIC] != 0) path = PATH_TWOPASS;
         else path = stream_classify(r.block_len, r.grad_dtype, h->n_clusters > 0);
         h->path[i] = path;
         h->elems_by_path[path] += r.numel;
@@ -286,6 +286,7 @@ int adammini_set_option(am_handle *h, int32_t key, int64_t value) {
     if ((key == AM_OPT_PATH || key == AM_OPT_PROFILE) && value > 1) return AM_ERR_INVALID_ARGUMENT;
     if ((key == AM_OPT_STREAM_CHUNK || key == AM_OPT_CLUSTER_CHUNK) && value > 4096 && value != kStaticRanges)
         return AM_ERR_INVALID_ARGUMENT;
+    if (key == AM_OPT_STATISTIC && value > 4) return AM_ERR_INVALID_ARGUMENT;
     if (key == AM_OPT_PROFILE) {
         if (value && !h->prof_ev[0])
             for (int k = 0; k < 5; ++k) AM_CUDA(h, cudaEventCreate(&h->prof_ev[k]));
@@ -380,6 +381,8 @@ int adammini_step_ex(am_handle *h, void *const *params, const void *const *grads
     sc.gscale = ex ? static_cast<float>(ex->grad_scale) : 1.f;
     sc.gscale_dev = ex ? ex->grad_scale_device : nullptr;
     sc.skip_flag = ex ? ex->skip_flag : nullptr;
+    sc.statistic = static_cast<int32_t>(h->opt[AM_OPT_STATISTIC]);
+    sc.pad = 0;
 
     const bool prof = h->opt[AM_OPT_PROFILE] != 0;
     if (prof) AM_CUDA(h, cudaEventRecord(h->prof_ev[0], stream));
@@ -396,6 +399,7 @@ int adammini_step_ex(am_handle *h, void *const *params, const void *const *grads
         ss.gscale = sc.gscale;
         ss.gscale_dev = sc.gscale_dev;
         ss.skip_flag = sc.skip_flag;
+        ss.statistic = sc.statistic;
         small_kernel<<<static_cast<unsigned>(h->small_units), kThreads, 0, stream>>>(
             h->d_tensors, h->d_small_segs, h->n_small_segs, v, ss);
         AM_CUDA(h, cudaGetLastError());
@@ -408,7 +412,7 @@ int adammini_step_ex(am_handle *h, void *const *params, const void *const *grads
     if (prof) AM_CUDA(h, cudaEventRecord(h->prof_ev[3], stream));
     if (h->piece_units) {
         twopass_partial_kernel<<<static_cast<unsigned>(h->piece_units), kThreads, 0, stream>>>(
-            h->d_tensors, h->d_piece_segs, h->n_piece_segs, h->d_partials, sc.gscale, sc.gscale_dev, sc.skip_flag);
+            h->d_tensors, h->d_piece_segs, h->n_piece_segs, h->d_partials, sc.gscale, sc.gscale_dev, sc.skip_flag, sc.statistic);
         AM_CUDA(h, cudaGetLastError());
         const unsigned fin_grid = static_cast<unsigned>(ceil_div(h->block_units, kThreads / 32));
         twopass_finalize_kernel<<<fin_grid, kThreads, 0, stream>>>(
@@ -596,6 +600,8 @@ extern "C" int adammini_step_tensor_noalloc(void *param, const void *grad, void 
     sc.gscale = 1.f;
     sc.gscale_dev = nullptr;
     sc.skip_flag = nullptr;
+    sc.statistic = 0;
+    sc.pad = 0;
 
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const int vec = block_len % 4 == 0 ? 1 : 0;

@@ -61,6 +61,8 @@ struct StepScalars {
     float gscale;           // gradients are multiplied by this on load (1 = off) ...
     const float *gscale_dev;  // ... and by this device scalar when not null
     const float *skip_flag;   // device scalar; non-zero: the step leaves everything untouched
+    int32_t statistic;        // block statistic: 0 mean, 1 max, 2 min, 3 one-norm, 4 two-norm of g*g
+    int32_t pad;
 };
 
 }  // namespace am

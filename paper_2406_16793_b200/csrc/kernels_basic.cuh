@@ -85,13 +85,45 @@ __device__ __forceinline__ void update_four(const float4 &g, float4 &m, float4 &
     update_one(g.w, m.w, p.w, beta1, omb1, lr_wd, step);
 }
 
-// Per-block scalars in double: new v_b and the step size (see update_one).
-__device__ __forceinline__ float block_step(double sum_sq, double L, float v_old,
-                                            const StepScalars &s, float *v_new) {
-    const double vn = s.omb2 * (sum_sq / L) + s.beta2 * static_cast<double>(v_old);
+// Per-block scalars in double: new v_b from the block statistic (mean of g*g in
+// Algorithm 1) and the step size (see update_one).
+__device__ __forceinline__ float block_step_from_statistic(double statistic, float v_old,
+                                                           const StepScalars &s, float *v_new) {
+    const double vn = s.omb2 * statistic + s.beta2 * static_cast<double>(v_old);
     *v_new = static_cast<float>(vn);
     const double denom = sqrt(vn * s.inv_bc2) + s.eps;
     return static_cast<float>(s.lr_over_bc1 / denom);
+}
+__device__ __forceinline__ float block_step(double sum_sq, double L, float v_old,
+                                            const StepScalars &s, float *v_new) {
+    return block_step_from_statistic(sum_sq / L, v_old, s, v_new);
+}
+
+// The ablation statistics of the paper's appendix combine like this: sums for
+// the mean, the 1-norm and the 2-norm (of g*g, resp. of (g*g)^2), max, min.
+__device__ __forceinline__ double stat_combine(double a, double b, int statistic) {
+    if (statistic == 1) return a > b ? a : b;
+    if (statistic == 2) return a < b ? a : b;
+    return a + b;
+}
+__device__ __forceinline__ double stat_identity(int statistic) {
+    if (statistic == 1) return 0.0;                    // g*g >= 0
+    if (statistic == 2) return __longlong_as_double(0x7ff0000000000000LL);   // +inf
+    return 0.0;
+}
+__device__ __forceinline__ double stat_term(float g, int statistic) {
+    const float sq = g * g;
+    return statistic == 4 ? static_cast<double>(sq) * static_cast<double>(sq) : static_cast<double>(sq);
+}
+__device__ __forceinline__ double stat_finish(double acc, double L, int statistic) {
+    if (statistic == 0) return acc / L;
+    if (statistic == 4) return sqrt(acc);
+    return acc;
+}
+__device__ __forceinline__ double warp_stat(double x, int statistic) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x = stat_combine(x, __shfl_xor_sync(0xffffffffu, x, o), statistic);
+    return x;
 }
 
 // Segment lookup: the last segment whose unit_begin is <= unit.
@@ -117,6 +149,7 @@ struct SmallScalars {
     float beta1, omb1, beta2, omb2, inv_bc2, lr_over_bc1, eps, lr_wd, gscale;
     const float *gscale_dev;
     const float *skip_flag;
+    int statistic;
 };
 
 __device__ __forceinline__ float small_block_step(float mean_sq, float v_old, const SmallScalars &s,
@@ -173,8 +206,17 @@ __device__ __forceinline__ void small_body(const DevTensor &t, const Seg &seg, i
                 sum = fmaf(gl[k], gl[k], sum);
             }
         }
+        float stat = L == 1 ? sum : __fdiv_rn(sum, Lf);
+        if (sc.statistic != 0) {
+            // ablation statistics of g*g: max, min, 1-norm, 2-norm
+            double acc = stat_identity(sc.statistic);
+#pragma unroll
+            for (int k = 0; k < kSmallMaxL; ++k)
+                if (k < L) acc = stat_combine(acc, stat_term(gl[k], sc.statistic), sc.statistic);
+            stat = static_cast<float>(stat_finish(acc, static_cast<double>(L), sc.statistic));
+        }
         float vn;
-        const float st = small_block_step(L == 1 ? sum : __fdiv_rn(sum, Lf), vt[b], sc, &vn);
+        const float st = small_block_step(stat, vt[b], sc, &vn);
         vt[b] = vn;
 #pragma unroll
         for (int k = 0; k < kSmallMaxL; ++k) {
@@ -262,21 +304,37 @@ __device__ __forceinline__ double piece_sum_sq(const PieceRef &r, float gscale) 
     return tot;
 }
 
+// Max, min or sum of (g*g)^2 over one piece (the ablation statistics): plain
+// double accumulation per thread; these variants are not performance paths.
+template <int GD>
+__device__ __forceinline__ double piece_statistic(const PieceRef &r, float gscale, int statistic) {
+    double acc = stat_identity(statistic);
+    for (int64_t i = threadIdx.x; i < r.n; i += kThreads)
+        acc = stat_combine(acc, stat_term(load_g1<GD>(r.t->g, r.start + i, gscale), statistic), statistic);
+    return acc;
+}
+
 __global__ void __launch_bounds__(kThreads)
 twopass_partial_kernel(const DevTensor *__restrict__ tensors, const Seg *__restrict__ segs, int n_segs,
                        double *__restrict__ partials, float gscale_host, const float *gscale_dev,
-                       const float *skip_flag) {
+                       const float *skip_flag, int statistic) {
     __shared__ double warp_part[kThreads / 32];
     if (step_skipped(skip_flag)) return;
     const float gscale = effective_gscale(gscale_host, gscale_dev);
     const PieceRef r = decode_piece(tensors, segs, n_segs, blockIdx.x);
-    const double w = warp_sum(r.t->gdtype == AM_BF16 ? piece_sum_sq<AM_BF16>(r, gscale) : piece_sum_sq<AM_F32>(r, gscale));
+    const bool plain_sum = statistic == 0 || statistic == 3;       // both need the sum of g*g
+    double w;
+    if (plain_sum)
+        w = warp_sum(r.t->gdtype == AM_BF16 ? piece_sum_sq<AM_BF16>(r, gscale) : piece_sum_sq<AM_F32>(r, gscale));
+    else
+        w = warp_stat(r.t->gdtype == AM_BF16 ? piece_statistic<AM_BF16>(r, gscale, statistic)
+                                             : piece_statistic<AM_F32>(r, gscale, statistic), statistic);
     if ((threadIdx.x & 31) == 0) warp_part[threadIdx.x >> 5] = w;
     __syncthreads();
     if (threadIdx.x == 0) {
-        double s = 0.0;
+        double s = warp_part[0];
 #pragma unroll
-        for (int k = 0; k < kThreads / 32; ++k) s += warp_part[k];
+        for (int k = 1; k < kThreads / 32; ++k) s = plain_sum ? s + warp_part[k] : stat_combine(s, warp_part[k], statistic);
         partials[r.t->piece_base + r.local] = s;
     }
 }
@@ -294,12 +352,14 @@ twopass_finalize_kernel(const DevTensor *__restrict__ tensors, const Seg *__rest
     const DevTensor &t = tensors[seg.tensor];
     const int64_t b = unit - seg.unit_begin;
     const double *src = partials + t.piece_base + b * t.pieces_per_block;
-    double s = 0.0;
-    for (int64_t j = lane; j < t.pieces_per_block; j += 32) s += src[j];
-    s = warp_sum(s);
+    const int statistic = sc.statistic;
+    double s = stat_identity(statistic);
+    for (int64_t j = lane; j < t.pieces_per_block; j += 32) s = stat_combine(s, src[j], statistic);
+    s = warp_stat(s, statistic);
     if (lane == 0) {
         float vn;
-        const float st = block_step(s, static_cast<double>(t.L), v[t.v_offset + b], sc, &vn);
+        const float st = block_step_from_statistic(stat_finish(s, static_cast<double>(t.L), statistic),
+                                                   v[t.v_offset + b], sc, &vn);
         v[t.v_offset + b] = vn;
         block_steps[t.block_base + b] = st;
     }

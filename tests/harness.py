@@ -66,7 +66,8 @@ def v_relative_error(got: np.ndarray, want: np.ndarray) -> float:
     fin = np.isfinite(want)
     if not np.array_equal(fin, np.isfinite(got)):
         return float("inf")
-    d = np.abs(got - want)[fin]
+    with np.errstate(invalid="ignore"):
+        d = np.abs(got - want)[fin]
     return float((d / np.maximum(np.abs(want[fin]), 1e-30)).max()) if d.size else 0.0
 
 
@@ -133,12 +134,12 @@ def make_optimizer(w: W.Workload, options: Optional[Dict[int, int]] = None, **hp
 
 
 def oracle_step_all(state: ostep.OracleState, grads_cpu: Sequence, step: int, hp: Dict[str, float],
-                    pool: Optional[cf.ThreadPoolExecutor] = None) -> None:
+                    pool: Optional[cf.ThreadPoolExecutor] = None, statistic: int = 0) -> None:
     """One oracle step over all tensors; tensors are independent, so they may
     run on several host threads (each call is the single-threaded C routine)."""
     def one(i):
         ostep.adammini_step(state.p[i], state.m[i], state.v[i], grads_cpu[i], state.block_lens[i],
-                            step=step, apply_wd=state.wd_flags[i], **hp)
+                            step=step, apply_wd=state.wd_flags[i], statistic=statistic, **hp)
     if pool is None:
         for i in range(len(grads_cpu)):
             one(i)
@@ -148,7 +149,7 @@ def oracle_step_all(state: ostep.OracleState, grads_cpu: Sequence, step: int, hp
 
 def run_parity(w: W.Workload, steps: Optional[int] = None, options: Optional[Dict[int, int]] = None,
                device="cuda", hp_override: Optional[Dict[str, float]] = None, mutate_grads=None,
-               lr_schedule=None) -> Dict[str, float]:
+               lr_schedule=None, statistic: int = 0) -> Dict[str, float]:
     """Run `steps` steps on the GPU and in the oracle; returns the worst errors.
 
     mutate_grads(step, list_of_device_grads) may edit the gradients in place
@@ -157,6 +158,8 @@ def run_parity(w: W.Workload, steps: Optional[int] = None, options: Optional[Dic
     steps = steps or w.steps
     hp = {**w.hparams, **(hp_override or {})}
     dev = DeviceState(w, device)
+    if statistic:
+        options = {**(options or {}), am.binding.OPT_STATISTIC: statistic}
     opt = make_optimizer(w, options, **(hp_override or {}))
     ora = ostep.OracleState([p.cpu() for p in dev.p], [t.block_len for t in w.tensors],
                             [bool(t.apply_weight_decay) for t in w.tensors])
@@ -172,7 +175,7 @@ def run_parity(w: W.Workload, steps: Optional[int] = None, options: Optional[Dic
                 opt.set_lr(hp_t["lr"])
             opt.step(dev.p, dev.g, dev.m, dev.v, t)
             grads_cpu = [g.cpu() for g in dev.g]
-            oracle_step_all(ora, grads_cpu, t, hp_t, pool)
+            oracle_step_all(ora, grads_cpu, t, hp_t, pool, statistic)
         opt.sync_status()
     finally:
         pool.shutdown()

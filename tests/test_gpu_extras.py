@@ -121,3 +121,17 @@ def test_skip_flag_leaves_the_state_untouched():
     ob.sync_status()
     assert all(torch.equal(x, y) for x, y in zip(before, b.p + b.m + [b.v]))
     oa.close(); ob.close()
+
+
+@pytest.mark.parametrize("statistic", [B.STAT_MAX, B.STAT_MIN, B.STAT_ONE_NORM, B.STAT_TWO_NORM],
+                         ids=["max", "min", "one-norm", "two-norm"])
+@pytest.mark.parametrize("grad_dtype", [W.F32, W.BF16], ids=["f32", "bf16"])
+def test_ablation_statistics(statistic, grad_dtype):
+    """The block statistics of the paper's ablation (max, min, 1-norm, 2-norm of
+    g*g in place of the mean) against the oracle's variant routine."""
+    H.assert_parity(H.run_parity(ragged_workload(grad_dtype), steps=4, statistic=statistic))
+
+
+def test_ablation_statistics_on_model_shapes():
+    w = W.scaled_rows(W.llama2_7b(n_layers=1, vocab=128), 128)
+    H.assert_parity(H.run_parity(w, steps=3, statistic=B.STAT_TWO_NORM))
