@@ -217,8 +217,9 @@ typedef enum {
     AM_OPT_STREAM_CTAS   = 1, /* persistent CTAs of the streaming kernel (0 = one per SM) */
     AM_OPT_CLUSTER_SIZE  = 2, /* CTAs per cluster for head-sized blocks (0 = default) */
     AM_OPT_STREAM_THREADS = 3, /* consumer threads per CTA of the streaming kernels (0 = default) */
-    AM_OPT_PROFILE       = 4, /* 1: record CUDA events around each kernel family of every step
-                                 (read them with adammini_get_profile) */
+    AM_OPT_PROFILE       = 4, /* n > 0: record CUDA events around each kernel family of every step, keeping
+                                 the latest n steps (n <= 4096); read them with adammini_get_profile.
+                                 Setting the option again restarts the record */
     AM_OPT_STREAM_CHUNK  = 5  /* how the streaming kernel's CTAs share the work: 0 = automatic (CTAs take
                                  up to 64 work items at a time from a shared counter, which evens out
                                  bandwidth differences between SMs); 1..4096 = that many items at a
@@ -254,10 +255,11 @@ typedef enum {
 } am_query;
 int adammini_query(const am_handle *h, int32_t what, int64_t *value);
 
-/* With AM_OPT_PROFILE set: waits for the last step and writes the device time in
- * milliseconds of its kernel families to ms[0..3] (host array): thread-per-block
- * kernel, streaming kernel, cluster kernel, two-pass kernels (0 where none ran). */
-int adammini_get_profile(am_handle *h, float *ms);
+/* With AM_OPT_PROFILE set: waits for the recorded steps and writes the mean device time in
+ * milliseconds per step of each kernel family to ms[0..3] (host array): thread-per-block
+ * kernel, streaming kernel, cluster kernel, two-pass kernels (0 where none ran).  *n_steps
+ * (may be NULL) receives the number of steps averaged. */
+int adammini_get_profile(am_handle *h, float *ms, int32_t *n_steps);
 
 /* The CUDA error code (cudaError_t as int) of the last AM_ERR_CUDA on this handle. */
 int adammini_last_cuda_error(const am_handle *h);

@@ -76,7 +76,7 @@ _SIGNATURES = {
     "adammini_sync_status": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p]),
     "adammini_set_option": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64]),
     "adammini_query": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.POINTER(ctypes.c_int64)]),
-    "adammini_get_profile": (ctypes.c_int, [ctypes.c_void_p, ctypes.POINTER(ctypes.c_float)]),
+    "adammini_get_profile": (ctypes.c_int, [ctypes.c_void_p, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32)]),
     "adammini_last_cuda_error": (ctypes.c_int, [ctypes.c_void_p]),
     "adammini_destroy": (ctypes.c_int, [ctypes.c_void_p]),
     "adammini_status_string": (ctypes.c_char_p, [ctypes.c_int]),
@@ -268,11 +268,13 @@ class AdamMini:
         _check(load().adammini_step_host(self._h, pa, ga, ma, vp, int(step), int(staging_bytes)), self._h)
 
     def get_profile(self):
-        """Device milliseconds of the last step's kernel families (needs
-        OPT_PROFILE): [thread-per-block, streaming, cluster, two-pass]."""
+        """Mean device milliseconds per step of each kernel family over the steps
+        recorded since OPT_PROFILE was set: ([thread-per-block, streaming, cluster,
+        two-pass], number of steps averaged)."""
         ms = (ctypes.c_float * 4)()
-        _check(load().adammini_get_profile(self._h, ms), self._h)
-        return [float(x) for x in ms]
+        n = ctypes.c_int32()
+        _check(load().adammini_get_profile(self._h, ms, ctypes.byref(n)), self._h)
+        return [float(x) for x in ms], int(n.value)
 
     def sync_status(self, stream: int = 0) -> None:
         """Wait for the stream; raises if a device-side bounded wait gave up."""

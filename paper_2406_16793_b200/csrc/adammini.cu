@@ -283,21 +283,24 @@ int adammini_set_hparams(am_handle *h, const am_hparams *hp) {
 
 int adammini_set_option(am_handle *h, int32_t key, int64_t value) {
     if (!h || key < 0 || key >= kNumOptions || value < 0) return AM_ERR_INVALID_ARGUMENT;
-    if ((key == AM_OPT_PATH || key == AM_OPT_PROFILE) && value > 1) return AM_ERR_INVALID_ARGUMENT;
+    if (key == AM_OPT_PATH && value > 1) return AM_ERR_INVALID_ARGUMENT;
     if ((key == AM_OPT_STREAM_CHUNK || key == AM_OPT_CLUSTER_CHUNK) && value > 4096 && value != kStaticRanges)
         return AM_ERR_INVALID_ARGUMENT;
     if (key == AM_OPT_STATISTIC && value > 4) return AM_ERR_INVALID_ARGUMENT;
     if (key == AM_OPT_PROFILE) {
-        if (value && !h->prof_ev[0])
-            for (int k = 0; k < 5; ++k) AM_CUDA(h, cudaEventCreate(&h->prof_ev[k]));
+        if (value > 4096) return AM_ERR_INVALID_ARGUMENT;
+        for (cudaEvent_t e : h->prof_ev) cudaEventDestroy(e);
+        h->prof_ev.clear();
+        try {
+            h->prof_ev.resize(static_cast<size_t>(value) * 5, nullptr);
+        } catch (...) {
+            return AM_ERR_ALLOC;
+        }
+        for (cudaEvent_t &e : h->prof_ev) AM_CUDA(h, cudaEventCreate(&e));
         h->opt[key] = value;
-        h->prof_recorded = false;
+        h->prof_steps = 0;
         return AM_OK;
     }
-    if (key == AM_OPT_CLUSTER_SIZE && value != 0 && value != 1 && value != 2 && value != 4 && value != 8)
-        return AM_ERR_INVALID_ARGUMENT;
-    if (key == AM_OPT_STREAM_THREADS && value != 0 && (value % 32 != 0 || value < 64 || value > 512))
-        return AM_ERR_INVALID_ARGUMENT;
     if (h->opt[key] == value) return AM_OK;
     AM_CUDA(h, cudaDeviceSynchronize());    // the old tables may still be in use
     const int64_t old = h->opt[key];
@@ -385,7 +388,8 @@ int adammini_step_ex(am_handle *h, void *const *params, const void *const *grads
     sc.pad = 0;
 
     const bool prof = h->opt[AM_OPT_PROFILE] != 0;
-    if (prof) AM_CUDA(h, cudaEventRecord(h->prof_ev[0], stream));
+    cudaEvent_t *pev = prof ? &h->prof_ev[(h->prof_steps % h->opt[AM_OPT_PROFILE]) * 5] : nullptr;
+    if (prof) AM_CUDA(h, cudaEventRecord(pev[0], stream));
     if (h->small_units) {
         SmallScalars ss;
         ss.beta1 = sc.beta1;
@@ -405,11 +409,11 @@ int adammini_step_ex(am_handle *h, void *const *params, const void *const *grads
         AM_CUDA(h, cudaGetLastError());
     }
     h->stream.bf16_copies = ex && ex->params_bf16;
-    if (prof) AM_CUDA(h, cudaEventRecord(h->prof_ev[1], stream));
+    if (prof) AM_CUDA(h, cudaEventRecord(pev[1], stream));
     AM_CUDA(h, h->stream.launch_main(h->d_tensors, v, sc, h->error_word, stream));
-    if (prof) AM_CUDA(h, cudaEventRecord(h->prof_ev[2], stream));
+    if (prof) AM_CUDA(h, cudaEventRecord(pev[2], stream));
     AM_CUDA(h, h->stream.launch_cluster(h->d_tensors, v, sc, h->error_word, stream));
-    if (prof) AM_CUDA(h, cudaEventRecord(h->prof_ev[3], stream));
+    if (prof) AM_CUDA(h, cudaEventRecord(pev[3], stream));
     if (h->piece_units) {
         twopass_partial_kernel<<<static_cast<unsigned>(h->piece_units), kThreads, 0, stream>>>(
             h->d_tensors, h->d_piece_segs, h->n_piece_segs, h->d_partials, sc.gscale, sc.gscale_dev, sc.skip_flag, sc.statistic);
@@ -424,16 +428,28 @@ int adammini_step_ex(am_handle *h, void *const *params, const void *const *grads
         AM_CUDA(h, cudaGetLastError());
     }
     if (prof) {
-        AM_CUDA(h, cudaEventRecord(h->prof_ev[4], stream));
-        h->prof_recorded = true;
+        AM_CUDA(h, cudaEventRecord(pev[4], stream));
+        ++h->prof_steps;
     }
     return AM_OK;
 }
 
-int adammini_get_profile(am_handle *h, float *ms) {
-    if (!h || !ms || !h->prof_recorded) return AM_ERR_INVALID_ARGUMENT;
-    AM_CUDA(h, cudaEventSynchronize(h->prof_ev[4]));
-    for (int k = 0; k < 4; ++k) AM_CUDA(h, cudaEventElapsedTime(&ms[k], h->prof_ev[k], h->prof_ev[k + 1]));
+int adammini_get_profile(am_handle *h, float *ms, int32_t *n_steps) {
+    if (!h || !ms || h->opt[AM_OPT_PROFILE] == 0 || h->prof_steps == 0) return AM_ERR_INVALID_ARGUMENT;
+    const int64_t ring = h->opt[AM_OPT_PROFILE];
+    const int64_t n = std::min(h->prof_steps, ring);
+    double sum[4] = {0.0, 0.0, 0.0, 0.0};
+    for (int64_t s = 0; s < n; ++s) {
+        cudaEvent_t *ev = &h->prof_ev[s * 5];
+        AM_CUDA(h, cudaEventSynchronize(ev[4]));
+        for (int k = 0; k < 4; ++k) {
+            float x = 0.f;
+            AM_CUDA(h, cudaEventElapsedTime(&x, ev[k], ev[k + 1]));
+            sum[k] += x;
+        }
+    }
+    for (int k = 0; k < 4; ++k) ms[k] = static_cast<float>(sum[k] / static_cast<double>(n));
+    if (n_steps) *n_steps = static_cast<int32_t>(n);
     return AM_OK;
 }
 
@@ -456,8 +472,8 @@ int adammini_destroy(am_handle *h) {
         if (h->pinned[k]) cudaFreeHost(h->pinned[k]);
         if (h->ev[k]) cudaEventDestroy(h->ev[k]);
     }
-    for (int k = 0; k < 5; ++k)
-        if (h->prof_ev[k]) cudaEventDestroy(h->prof_ev[k]);
+    for (cudaEvent_t e : h->prof_ev)
+        if (e) cudaEventDestroy(e);
     if (h->error_word) cudaFreeHost(h->error_word);
     delete h;
     return AM_OK;

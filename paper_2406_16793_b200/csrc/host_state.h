@@ -38,8 +38,8 @@ struct am_handle {
     int64_t elems_by_path[4] = {0, 0, 0, 0};
     int64_t algorithmic_bytes = 0;
     int64_t bytes_by_path[4] = {0, 0, 0, 0};
-    cudaEvent_t prof_ev[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
-    bool prof_recorded = false;
+    std::vector<cudaEvent_t> prof_ev;    // AM_OPT_PROFILE: 5 events per recorded step, a ring of `opt` steps
+    int64_t prof_steps = 0;              // steps recorded since profiling was switched on
 
     // pinned staging of the tensor table, double buffered
     am::DevTensor *pinned[2] = {nullptr, nullptr};

@@ -319,3 +319,21 @@ def test_sharded_ranks_tile_the_unsharded_step(world):
     assert torch.equal(v_all, ref.v)
     for r in ranks:
         r.close()
+
+
+def test_profile_ring_reports_per_family_times():
+    w = W.scaled_rows(W.llama2_7b(n_layers=1, vocab=256), 128)
+    dev = H.DeviceState(w, guarded=False)
+    opt = H.make_optimizer(w)
+    with pytest.raises(am.AdamMiniError):
+        opt.get_profile()                                   # profiling is off
+    opt.set_option(B.OPT_PROFILE, 4)
+    for t in range(1, 7):
+        dev.draw_grads(t)
+        opt.step(dev.p, dev.g, dev.m, dev.v, t)
+    ms, n = opt.get_profile()
+    assert n == 4                                           # the ring keeps the latest 4 of 6 steps
+    assert ms[0] < 0.05 and ms[3] < 0.05                    # no tiny blocks, nothing on the two-pass path
+    assert 0.0 < ms[1] < 50.0 and 0.0 < ms[2] < 50.0        # streaming kernel and cluster kernel ran
+    opt.set_option(B.OPT_PROFILE, 0)
+    opt.close()
