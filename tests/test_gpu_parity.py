@@ -337,3 +337,59 @@ def test_profile_ring_reports_per_family_times():
     assert 0.0 < ms[1] < 50.0 and 0.0 < ms[2] < 50.0        # streaming kernel and cluster kernel ran
     opt.set_option(B.OPT_PROFILE, 0)
     opt.close()
+
+
+def test_new_buffers_every_step():
+    """Callers may hand in different gradient (and state) buffers at every step:
+    the library re-reads the addresses each call."""
+    w = W.scaled_rows(W.llama2_7b(n_layers=1, vocab=256), 128)
+    ref = _run_steps(w, 1, 4)
+    dev = H.DeviceState(w, guarded=False)
+    opt = H.make_optimizer(w)
+    for t in range(1, 5):
+        dev.draw_grads(t)
+        grads = [g.clone() for g in dev.g]                 # fresh allocations
+        if t == 3:                                         # and the state moves once
+            dev.p = [x.clone() for x in dev.p]
+            dev.m = [x.clone() for x in dev.m]
+        opt.step(dev.p, grads, dev.m, dev.v, t)
+        del grads
+    opt.sync_status()
+    opt.close()
+    assert _same(ref, dev)
+
+
+@pytest.mark.parametrize("L", [1, 4096, 0], ids=["L1", "L4096", "whole"])
+def test_more_than_2_to_31_elements_in_one_tensor(L):
+    """Element offsets beyond 32 bits: one tensor of 2^31 + 2^20 elements; the
+    oracle recomputes runs at the very end (and start) of the tensor."""
+    _need_free_memory(40)
+    numel = (1 << 31) + (1 << 20)
+    if L == 0:
+        # one block: check v against a float64 sum of squares and a sampled update at the far end
+        w = W.Workload("huge-whole", 71, [W.TensorSpec("t", 1, numel, W.WHOLE, grad_dtype=W.BF16)],
+                       W.GradRecipe(-3.0, -1.0), steps=1)
+        dev = H.DeviceState(w, guarded=False)
+        opt = H.make_optimizer(w)
+        dev.draw_grads(1)
+        tail = slice(numel - 4096, numel)
+        p0 = dev.p[0][tail].double().cpu().numpy()
+        opt.step(dev.p, dev.g, dev.m, dev.v, 1)
+        opt.sync_status()
+        sum_sq = 0.0
+        for lo in range(0, numel, 1 << 28):
+            sum_sq += float(dev.g[0][lo:lo + (1 << 28)].double().square().sum())
+        hp = w.hparams
+        v_want = (1 - hp["beta2"]) * sum_sq / numel
+        assert abs(float(dev.v[0]) - v_want) <= 1e-5 * v_want
+        g = dev.g[0][tail].double().cpu().numpy()
+        m_want = (1 - hp["beta1"]) * g
+        denom = np.sqrt(v_want / (1 - hp["beta2"])) + hp["eps"]
+        p_want = p0 * (1 - hp["lr"] * hp["weight_decay"]) - hp["lr"] * (m_want / (1 - hp["beta1"])) / denom
+        assert H.block_relative_error(dev.m[0][tail].cpu().numpy(), m_want, 4096) <= H.TOL
+        assert H.block_relative_error(dev.p[0][tail].cpu().numpy(), p_want, 4096) <= H.TOL
+        opt.close()
+        return
+    w = W.Workload(f"huge-L{L}", 70, [W.TensorSpec("t", 1, numel, W.FIXED, fixed_block_len=L, grad_dtype=W.BF16)],
+                   W.GradRecipe(-3.0, -1.0), steps=2)
+    H.assert_parity(H.run_sampled_runs(w, steps=2, run_elems=4096, n_runs=12))
