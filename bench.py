@@ -205,7 +205,8 @@ def run_ours(args):
     opt = am.AdamMini(part, **w.hparams)
     for key, val in ((B.OPT_STREAM_THREADS, args.stream_threads), (B.OPT_STREAM_CTAS, args.stream_ctas),
                      (B.OPT_CLUSTER_SIZE, args.cluster_size), (B.OPT_PATH, args.path),
-                     (B.OPT_STREAM_CHUNK, args.stream_chunk), (B.OPT_CLUSTER_CHUNK, args.cluster_chunk)):
+                     (B.OPT_STREAM_CHUNK, args.stream_chunk), (B.OPT_CLUSTER_CHUNK, args.cluster_chunk),
+                     (B.OPT_STREAM_GROUPS, args.stream_groups)):
         if val:
             opt.set_option(key, val)
     launches = opt.query(B.Q_LAUNCHES_PER_STEP)
@@ -346,6 +347,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama2-7b")
     ap.add_argument("--stream-threads", type=int, default=0, help="consumer threads per CTA (0 = library default)")
+    ap.add_argument("--stream-groups", type=int, default=0, help="consumer groups per CTA (0 = library default)")
     ap.add_argument("--stream-ctas", type=int, default=0, help="persistent CTAs (0 = one per SM)")
     ap.add_argument("--cluster-size", type=int, default=0, help="CTAs per cluster for head-sized blocks (0 = default)")
     ap.add_argument("--stream-chunk", type=int, default=0, help="items per grab from the shared work counter (0 = automatic, 1000000 = static ranges)")

@@ -216,7 +216,7 @@ typedef enum {
                                  tensor with block_len > 16 (correctness anchor) */
     AM_OPT_STREAM_CTAS   = 1, /* persistent CTAs of the streaming kernel (0 = one per SM) */
     AM_OPT_CLUSTER_SIZE  = 2, /* CTAs per cluster for head-sized blocks (0 = default) */
-    AM_OPT_STREAM_THREADS = 3, /* consumer threads per CTA of the streaming kernels (0 = default) */
+    AM_OPT_STREAM_THREADS = 3, /* threads per consumer group of the streaming kernels (0 = default 256) */
     AM_OPT_PROFILE       = 4, /* n > 0: record CUDA events around each kernel family of every step, keeping
                                  the latest n steps (n <= 4096); read them with adammini_get_profile.
                                  Setting the option again restarts the record */
@@ -231,6 +231,8 @@ typedef enum {
                                   which it reports to train worse: 1 = max, 2 = min, 3 = 1-norm (sum),
                                   4 = 2-norm of the vector g*g.  Non-zero values run on the two-pass
                                   kernels (g read twice) */
+    , AM_OPT_STREAM_GROUPS = 8 /* consumer groups per CTA of the streaming kernels (0 = default 2, or 1);
+                                  groups x threads is capped at 512 */
 } am_option;
 int adammini_set_option(am_handle *h, int32_t key, int64_t value);
 

@@ -17,7 +17,7 @@ LIBRARY = os.environ.get("ADAMMINI_LIBRARY") or os.path.join(_HERE, "libadammini
 WHOLE, ROWS, HEADS, TOKENS, FIXED = 0, 1, 2, 3, 4
 F32, BF16 = 0, 1
 
-OPT_PATH, OPT_STREAM_CTAS, OPT_CLUSTER_SIZE, OPT_STREAM_THREADS, OPT_PROFILE, OPT_STREAM_CHUNK, OPT_CLUSTER_CHUNK, OPT_STATISTIC = 0, 1, 2, 3, 4, 5, 6, 7
+OPT_PATH, OPT_STREAM_CTAS, OPT_CLUSTER_SIZE, OPT_STREAM_THREADS, OPT_PROFILE, OPT_STREAM_CHUNK, OPT_CLUSTER_CHUNK, OPT_STATISTIC, OPT_STREAM_GROUPS = 0, 1, 2, 3, 4, 5, 6, 7, 8
 STAT_MEAN, STAT_MAX, STAT_MIN, STAT_ONE_NORM, STAT_TWO_NORM = 0, 1, 2, 3, 4
 (Q_LAUNCHES_PER_STEP, Q_SCRATCH_BYTES, Q_TOTAL_BLOCKS, Q_TOTAL_ELEMENTS, Q_ELEMENTS_SMALL,
  Q_ELEMENTS_STREAM, Q_ELEMENTS_CLUSTER, Q_ELEMENTS_TWOPASS, Q_ALGORITHMIC_BYTES, Q_BYTES_SMALL,

@@ -20,7 +20,7 @@ using namespace am;
 
 namespace {
 
-constexpr int kNumOptions = 8;
+constexpr int kNumOptions = 9;
 
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
@@ -73,10 +73,15 @@ int build_plan(am_handle *h) {
     sin.ctas = static_cast<int>(h->opt[AM_OPT_STREAM_CTAS]);
     sin.cluster_size = static_cast<int>(h->opt[AM_OPT_CLUSTER_SIZE]);
     sin.threads = static_cast<int>(h->opt[AM_OPT_STREAM_THREADS]);
+    sin.groups = static_cast<int>(h->opt[AM_OPT_STREAM_GROUPS]);
     sin.chunk = static_cast<int>(h->opt[AM_OPT_STREAM_CHUNK]);
     sin.cluster_chunk = static_cast<int>(h->opt[AM_OPT_CLUSTER_CHUNK]);
 
-    stream_probe_cluster(h->sm_count, sin.threads, sin.cluster_size, &h->cluster_size, &h->n_clusters);
+    {
+        int threads, groups;
+        stream_consumer_shape(sin.threads, sin.groups, &threads, &groups);
+        stream_probe_cluster(h->sm_count, threads * groups, sin.cluster_size, &h->cluster_size, &h->n_clusters);
+    }
 
     for (int i = 0; i < n; ++i) {
         const am_table_row &r = h->rows[i];
@@ -287,6 +292,7 @@ int adammini_set_option(am_handle *h, int32_t key, int64_t value) {
     if ((key == AM_OPT_STREAM_CHUNK || key == AM_OPT_CLUSTER_CHUNK) && value > 4096 && value != kStaticRanges)
         return AM_ERR_INVALID_ARGUMENT;
     if (key == AM_OPT_STATISTIC && value > 4) return AM_ERR_INVALID_ARGUMENT;
+    if (key == AM_OPT_STREAM_GROUPS && value > kMaxGroups) return AM_ERR_INVALID_ARGUMENT;
     if (key == AM_OPT_PROFILE) {
         if (value > 4096) return AM_ERR_INVALID_ARGUMENT;
         for (cudaEvent_t e : h->prof_ev) cudaEventDestroy(e);

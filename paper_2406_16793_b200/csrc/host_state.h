@@ -18,7 +18,7 @@ struct am_handle {
     int64_t total_blocks = 0;
     int64_t total_elems = 0;
     am_hparams hp{};
-    int64_t opt[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    int64_t opt[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};
 
     // launch plan
     bool planned = false;

@@ -38,7 +38,9 @@ constexpr int kWarpBlockMaxL = 1024;              // blocks up to this length ar
 constexpr int kCtrlBytes = 2048;                  // barriers, stage descriptors, reduction slots
 constexpr int kVAreaFloats = 272;                 // per stage: the old v of the stage's blocks (16-byte windows)
 constexpr int kMaxStages = 8;
-constexpr int kMaxConsumerWarps = 16;
+constexpr int kMaxConsumerWarps = 16;                // over all consumer groups
+constexpr int kMaxGroups = 2;                     // consumer groups; each owns every n-th work item
+constexpr int kExchangeSlots = 4;                 // cluster exchange slots (long blocks in flight per CTA pair of groups)
 constexpr int kMaxCluster = 8;
 constexpr int kItemSlots = 8;                     // block indices in flight from a cluster's first CTA to its peers
 constexpr int kStaticRanges = 1000000;            // AM_OPT_STREAM_CHUNK value that selects static ranges
@@ -46,6 +48,7 @@ constexpr int64_t kStreamMaxBlockBytes = 256 << 10;   // longest block one CTA h
 constexpr int64_t kClusterMaxBlockBytes = 4 << 20;    // longest block a cluster handles (bytes of g)
 constexpr unsigned long long kWaitTimeoutNs = 2000000000ull;   // 2 s
 constexpr unsigned long long kDrainTimeoutNs = 50000000ull;    // 50 ms
+constexpr unsigned long long kWaitGapCapNs = 1000000ull;       // 1 ms: the most one gap between polls adds to a wait
 
 enum StageKind : int32_t { STAGE_PACKED = 0, STAGE_SUM = 1, STAGE_APPLY = 2, STAGE_DONE = 3 };
 enum StageFlag : int32_t { SF_BF16 = 1, SF_WD = 2, SF_LAST = 4, SF_WRITE_V = 8, SF_V_STAGED = 16 };
@@ -60,7 +63,7 @@ struct StageMeta {          // written by the producer, read by the consumers
     int32_t kind;
     int32_t flags;
     int32_t v_shift;        // SF_V_STAGED: the first block's v sits at this index of the stage's v area
-    int32_t pad;
+    int32_t group;          // consumer group that processes this stage
     uint16_t *pb;           // bf16 copy of the updated parameters (nullptr: none)
 };
 static_assert(sizeof(StageMeta) == 64, "stage descriptor is 64 bytes");
@@ -82,7 +85,8 @@ struct StreamParams {
     int32_t n_stages;
     int32_t stage_bytes;
     int32_t g_region_bytes;     // m starts here inside a stage; p follows kStageElems floats later
-    int32_t consumer_threads;
+    int32_t consumer_threads;   // per consumer group
+    int32_t n_groups;
     int32_t chunk;              // > 0: items are handed out `chunk` at a time from *counter
     unsigned long long *counter;
     int64_t total_items;
@@ -92,11 +96,11 @@ struct StreamParams {
 struct Control {            // first kCtrlBytes of dynamic shared memory
     unsigned long long full[kMaxStages];
     unsigned long long empty[kMaxStages];
-    unsigned long long redbar;
-    unsigned long long xbar[2];
-    double red[2][kMaxConsumerWarps];
-    double xpart[2][kMaxCluster];
-    float redv[2];
+    unsigned long long redbar[kMaxGroups];
+    unsigned long long xbar[kExchangeSlots];
+    double red[kMaxGroups][2][kMaxConsumerWarps];
+    double xpart[kExchangeSlots][kMaxCluster];
+    float redv[kMaxGroups][2];
     int abort_flag;
     int pad;
     unsigned long long ibar[kItemSlots];   // cluster launches: "the next block index has arrived"
@@ -180,15 +184,21 @@ template <bool CLUSTER_ACQUIRE>
 __device__ __forceinline__ bool wait_phase(void *bar, uint32_t parity, Control *ctl, int *error_word,
                                            int code, unsigned long long limit_ns = kWaitTimeoutNs) {
     uint32_t spins = 0;
-    unsigned long long t0 = 0;
+    unsigned long long last = 0, waited = 0;
     for (;;) {
         const bool ok = CLUSTER_ACQUIRE ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity);
         if (ok) return true;
         if ((++spins & 255u) == 0) {
             if (*reinterpret_cast<volatile int *>(&ctl->abort_flag)) return false;
+            // Only time spent polling counts: a gap between two checks is capped, so a kernel
+            // that was switched out for a while (time slicing, a debugger) does not give up.
             const unsigned long long now = global_ns();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > limit_ns) {
+            if (last != 0) {
+                const unsigned long long gap = now - last;
+                waited += gap < kWaitGapCapNs ? gap : kWaitGapCapNs;
+            }
+            last = now;
+            if (waited > limit_ns) {
                 *reinterpret_cast<volatile int *>(&ctl->abort_flag) = 1;
                 *reinterpret_cast<volatile int *>(error_word) = code;
                 return false;
@@ -266,22 +276,23 @@ struct GroupSync {
     int buf;
 };
 
-// Sum `mine` over all consumer threads in a fixed order; also broadcasts
-// v_old read by thread 0.  Returns false on abort.
-__device__ __forceinline__ bool group_reduce(Control *ctl, GroupSync &gs, int *error_word, int ctid, int n_warps,
-                                             double mine, const float *v_ptr, double *total, float *v_old) {
+// Sum `mine` over the threads of one consumer group in a fixed order; also
+// broadcasts v_old read by the group's first thread.  Returns false on abort.
+__device__ __forceinline__ bool group_reduce(Control *ctl, GroupSync &gs, int *error_word, int group, int gtid,
+                                             int n_warps, double mine, const float *v_ptr, double *total,
+                                             float *v_old) {
     const double w = warp_sum(mine);
-    const int lane = ctid & 31;
+    const int lane = gtid & 31;
     if (lane == 0) {
-        ctl->red[gs.buf][ctid >> 5] = w;
-        if (ctid == 0) ctl->redv[gs.buf] = *v_ptr;
-        mbar_arrive(&ctl->redbar);
+        ctl->red[group][gs.buf][gtid >> 5] = w;
+        if (gtid == 0) ctl->redv[group][gs.buf] = *v_ptr;
+        mbar_arrive(&ctl->redbar[group]);
     }
-    if (!wait_phase<false>(&ctl->redbar, gs.parity, ctl, error_word, 3)) return false;
+    if (!wait_phase<false>(&ctl->redbar[group], gs.parity, ctl, error_word, 3)) return false;
     double s = 0.0;
-    for (int k = 0; k < n_warps; ++k) s += ctl->red[gs.buf][k];
+    for (int k = 0; k < n_warps; ++k) s += ctl->red[group][gs.buf][k];
     *total = s;
-    *v_old = ctl->redv[gs.buf];
+    *v_old = ctl->redv[group][gs.buf];
     gs.parity ^= 1;
     gs.buf ^= 1;
     return true;
@@ -302,7 +313,8 @@ stream_kernel(const __grid_constant__ StreamParams P) {
     unsigned char *stages = smem + kCtrlBytes;
     float *v_areas = reinterpret_cast<float *>(stages + static_cast<size_t>(P.n_stages) * P.stage_bytes);
     const int tid = threadIdx.x;
-    const int n_cwarps = P.consumer_threads >> 5;
+    const int n_gwarps = P.consumer_threads >> 5;          // warps of one consumer group
+    const int n_cwarps = n_gwarps * P.n_groups;
     const uint32_t crank = CLUSTER ? cluster_ctarank() : 0;
     const uint32_t csize = CLUSTER ? cluster_nctarank() : 1;
     const uint32_t unit = CLUSTER ? cluster_id_x() : blockIdx.x;
@@ -312,9 +324,8 @@ stream_kernel(const __grid_constant__ StreamParams P) {
             mbar_init(&ctl->full[s], 1);
             mbar_init(&ctl->empty[s], n_cwarps);
         }
-        mbar_init(&ctl->redbar, n_cwarps);
-        mbar_init(&ctl->xbar[0], csize);
-        mbar_init(&ctl->xbar[1], csize);
+        for (int k = 0; k < kMaxGroups; ++k) mbar_init(&ctl->redbar[k], n_gwarps);
+        for (int k = 0; k < kExchangeSlots; ++k) mbar_init(&ctl->xbar[k], csize);
         for (int k = 0; k < kItemSlots; ++k) mbar_init(&ctl->ibar[k], 1);
         ctl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -330,6 +341,7 @@ stream_kernel(const __grid_constant__ StreamParams P) {
             int stage = 0;
             uint32_t phase = 0;
             int64_t armed = 0;              // stages armed so far
+            int32_t item_group = 0;         // consumer group of the current item (items alternate)
             bool ok = true;
             int seg = 0;
             if (P.chunk <= 0) {
@@ -420,7 +432,7 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                     if (!(ok = acquire())) break;
                     StageMeta &mt = ctl->meta[stage];
                     mt.m = t.m + e0; mt.p = t.p + e0; mt.v = P.v + t.v_offset + b0;
-                    mt.pb = t.p_bf16 ? t.p_bf16 + e0 : nullptr;
+                    mt.pb = t.p_bf16 ? t.p_bf16 + e0 : nullptr; mt.group = item_group;
                     mt.inv_L = 1.0 / static_cast<double>(t.L);
                     mt.n = n; mt.L = static_cast<int>(t.L); mt.kind = STAGE_PACKED; mt.flags = base_flags | SF_WRITE_V;
                     const uint32_t vbytes = stage_v(mt, t.v_offset + b0, nb);
@@ -442,7 +454,7 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                         const int c = static_cast<int>(slice - off < sum_cap ? slice - off : sum_cap);
                         if (!(ok = acquire())) break;
                         StageMeta &mt = ctl->meta[stage];
-                        mt.m = nullptr; mt.p = nullptr; mt.v = P.v + t.v_offset + local; mt.pb = nullptr;
+                        mt.m = nullptr; mt.p = nullptr; mt.v = P.v + t.v_offset + local; mt.pb = nullptr; mt.group = item_group;
                         mt.inv_L = 1.0 / static_cast<double>(t.L);
                         mt.n = c; mt.L = 0; mt.kind = STAGE_SUM;
                         mt.flags = base_flags | (off + c == slice ? SF_LAST : 0) | (crank == 0 ? SF_WRITE_V : 0);
@@ -460,7 +472,7 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                         if (!(ok = acquire())) break;
                         StageMeta &mt = ctl->meta[stage];
                         mt.m = t.m + e0 + off; mt.p = t.p + e0 + off; mt.v = nullptr;
-                        mt.pb = t.p_bf16 ? t.p_bf16 + e0 + off : nullptr;
+                        mt.pb = t.p_bf16 ? t.p_bf16 + e0 + off : nullptr; mt.group = item_group;
                         mt.inv_L = 0.0;
                         mt.n = c; mt.L = 0; mt.kind = STAGE_APPLY; mt.flags = base_flags;
                         unsigned char *st = stages + static_cast<size_t>(stage) * P.stage_bytes;
@@ -471,6 +483,7 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                         advance();
                     }
                 }
+                if (++item_group == P.n_groups) item_group = 0;
             }
             if (ok && acquire()) {
                 ctl->meta[stage].kind = STAGE_DONE;
@@ -489,10 +502,18 @@ stream_kernel(const __grid_constant__ StreamParams P) {
         }
     } else {
         // ------------------------------ consumers ------------------------------
+        // The consumer warps form P.n_groups groups.  Every group follows the ring in order and
+        // reads every stage's descriptor, but only the owning group (descriptor's `group`; work
+        // items alternate between the groups) processes the stage, so the reduce / barrier /
+        // apply latencies of one item overlap with the other group's work on the next item.
+        // All warps arrive on a stage's `empty` barrier: owners after processing, the others
+        // at once (which also keeps the producer from rewriting a descriptor somebody still reads).
         const int ctid = tid - 32;
-        const int lane = ctid & 31, warp = ctid >> 5;
         const int nthr = P.consumer_threads;
-        if (ctid < nthr) {
+        const int group = ctid / nthr;
+        const int gtid = ctid - group * nthr;
+        const int lane = gtid & 31, warp = gtid >> 5;
+        if (group < P.n_groups) {
             // the gradient scale s enters as (1-beta1)*s in the first moment and as s*s on the
             // sums of squares, so the per-element work is the same with or without it
             const float gscale = effective_gscale(P.sc.gscale, P.sc.gscale_dev);
@@ -503,11 +524,19 @@ stream_kernel(const __grid_constant__ StreamParams P) {
             GroupSync gsync{0u, 0};
             float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;   // running sums of a long block
             float long_step = 0.f;
-            uint32_t long_count = 0;                         // long blocks finished (cluster exchange slot/parity)
+            uint32_t long_seen = 0;      // long blocks seen by this CTA, whoever owns them (exchange slot/parity)
             for (;;) {
                 if (!wait_phase<false>(&ctl->full[stage], phase, ctl, P.error_word, 2)) break;
                 const StageMeta mt = ctl->meta[stage];
                 if (mt.kind == STAGE_DONE) break;
+                const bool last_sum = mt.kind == STAGE_SUM && (mt.flags & SF_LAST);
+                if (mt.group != group) {
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&ctl->empty[stage]);
+                    if (last_sum) ++long_seen;
+                    if (++stage == P.n_stages) { stage = 0; phase ^= 1u; }
+                    continue;
+                }
                 const unsigned char *gs = stages + static_cast<size_t>(stage) * P.stage_bytes;
                 const float *ms = reinterpret_cast<const float *>(gs + P.g_region_bytes);
                 const float *ps = ms + kStageElems;
@@ -520,7 +549,7 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                 if (mt.kind == STAGE_PACKED) {
                     const int L = mt.L, nb = mt.n / mt.L;
                     if (L <= kWarpBlockMaxL) {
-                        for (int b = warp; b < nb; b += n_cwarps) {
+                        for (int b = warp; b < nb; b += n_gwarps) {
                             const int e = b * L;
                             float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
                             if (bf16) sum_span<AM_BF16>(gs, e, L, lane, 32, s0, s1, s2, s3);
@@ -541,41 +570,45 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                         for (int b = 0; b < nb && alive; ++b) {
                             const int e = b * L;
                             float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-                            if (bf16) sum_span<AM_BF16>(gs, e, L, ctid, nthr, s0, s1, s2, s3);
-                            else sum_span<AM_F32>(gs, e, L, ctid, nthr, s0, s1, s2, s3);
+                            if (bf16) sum_span<AM_BF16>(gs, e, L, gtid, nthr, s0, s1, s2, s3);
+                            else sum_span<AM_F32>(gs, e, L, gtid, nthr, s0, s1, s2, s3);
                             double tot;
                             float v_old;
-                            alive = group_reduce(ctl, gsync, P.error_word, ctid, n_cwarps, fold4(s0, s1, s2, s3),
+                            alive = group_reduce(ctl, gsync, P.error_word, group, gtid, n_gwarps, fold4(s0, s1, s2, s3),
                                                  v_src + b, &tot, &v_old);
                             if (!alive) break;
                             float vn;
                             const float step = stream_block_step(tot * gscale_sq, mt.inv_L, v_old, P.sc, &vn);
-                            if (ctid == 0) mt.v[b] = vn;
-                            if (bf16) apply_span<AM_BF16, COPY>(gs, ms, ps, mt.m, mt.p, mt.pb, e, L, ctid, nthr, beta1, omb1, lr_wd, step);
-                            else apply_span<AM_F32, COPY>(gs, ms, ps, mt.m, mt.p, mt.pb, e, L, ctid, nthr, beta1, omb1, lr_wd, step);
+                            if (gtid == 0) mt.v[b] = vn;
+                            if (bf16) apply_span<AM_BF16, COPY>(gs, ms, ps, mt.m, mt.p, mt.pb, e, L, gtid, nthr, beta1, omb1, lr_wd, step);
+                            else apply_span<AM_F32, COPY>(gs, ms, ps, mt.m, mt.p, mt.pb, e, L, gtid, nthr, beta1, omb1, lr_wd, step);
                         }
                     }
                     if (!alive) break;
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&ctl->empty[stage]);
                 } else if (mt.kind == STAGE_SUM) {
-                    if (bf16) sum_span<AM_BF16>(gs, 0, mt.n, ctid, nthr, a0, a1, a2, a3);
-                    else sum_span<AM_F32>(gs, 0, mt.n, ctid, nthr, a0, a1, a2, a3);
-                    if (!(mt.flags & SF_LAST)) {
+                    if (bf16) sum_span<AM_BF16>(gs, 0, mt.n, gtid, nthr, a0, a1, a2, a3);
+                    else sum_span<AM_F32>(gs, 0, mt.n, gtid, nthr, a0, a1, a2, a3);
+                    if (!last_sum) {
                         __syncwarp();
                         if (lane == 0) mbar_arrive(&ctl->empty[stage]);
                     } else {
                         double tot;
                         float v_old;
-                        if (!group_reduce(ctl, gsync, P.error_word, ctid, n_cwarps, fold4(a0, a1, a2, a3), v_src, &tot, &v_old))
+                        if (!group_reduce(ctl, gsync, P.error_word, group, gtid, n_gwarps, fold4(a0, a1, a2, a3), v_src, &tot, &v_old))
                             break;
                         __syncwarp();                       // the stage (and its v area) has been read
                         if (lane == 0) mbar_arrive(&ctl->empty[stage]);
                         a0 = a1 = a2 = a3 = 0.f;
                         if (CLUSTER) {
-                            // exchange the CTAs' sums through distributed shared memory
-                            const int slot = long_count & 1u;
-                            if (ctid == 0) {
+                            // Exchange the CTAs' sums through distributed shared memory.  Every CTA of
+                            // the cluster walks the same blocks in the same order, so block number
+                            // long_seen names the same block (and the same owning group) everywhere.
+                            // Four slots: a group reuses a slot only two of its own blocks later, after
+                            // a group barrier of every peer has ordered the earlier reads before it.
+                            const uint32_t slot = long_seen & (kExchangeSlots - 1);
+                            if (gtid == 0) {
                                 const uint32_t part = smem_addr(&ctl->xpart[slot][crank]);
                                 const uint32_t bar = smem_addr(&ctl->xbar[slot]);
                                 for (uint32_t r = 0; r < csize; ++r) {
@@ -583,18 +616,18 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                                     mbar_arrive_remote(map_to_rank(bar, r));
                                 }
                             }
-                            if (!wait_phase<true>(&ctl->xbar[slot], (long_count >> 1) & 1u, ctl, P.error_word, 4)) break;
+                            if (!wait_phase<true>(&ctl->xbar[slot], (long_seen / kExchangeSlots) & 1u, ctl, P.error_word, 4)) break;
                             tot = 0.0;
                             for (uint32_t r = 0; r < csize; ++r) tot += ctl->xpart[slot][r];
                         }
-                        ++long_count;
+                        ++long_seen;
                         float vn;
                         long_step = stream_block_step(tot * gscale_sq, mt.inv_L, v_old, P.sc, &vn);
-                        if (ctid == 0 && (mt.flags & SF_WRITE_V)) *mt.v = vn;
+                        if (gtid == 0 && (mt.flags & SF_WRITE_V)) *mt.v = vn;
                     }
                 } else {   // STAGE_APPLY
-                    if (bf16) apply_span<AM_BF16, COPY>(gs, ms, ps, mt.m, mt.p, mt.pb, 0, mt.n, ctid, nthr, beta1, omb1, lr_wd, long_step);
-                    else apply_span<AM_F32, COPY>(gs, ms, ps, mt.m, mt.p, mt.pb, 0, mt.n, ctid, nthr, beta1, omb1, lr_wd, long_step);
+                    if (bf16) apply_span<AM_BF16, COPY>(gs, ms, ps, mt.m, mt.p, mt.pb, 0, mt.n, gtid, nthr, beta1, omb1, lr_wd, long_step);
+                    else apply_span<AM_F32, COPY>(gs, ms, ps, mt.m, mt.p, mt.pb, 0, mt.n, gtid, nthr, beta1, omb1, lr_wd, long_step);
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&ctl->empty[stage]);
                 }
@@ -608,7 +641,7 @@ stream_kernel(const __grid_constant__ StreamParams P) {
 
 // ------------------------------- host-side planning -------------------------------
 struct StreamPlanInput {
-    int sm_count = 0, ctas = 0, cluster_size = 0, threads = 0, chunk = 0, cluster_chunk = 0;
+    int sm_count = 0, ctas = 0, cluster_size = 0, threads = 0, groups = 0, chunk = 0, cluster_chunk = 0;
     struct Item { int tensor; am_table_row row; };
     std::vector<Item> stream_tensors, cluster_tensors;
 };
@@ -647,7 +680,7 @@ inline StreamKernelFn stream_kernel_for(bool cluster, int gdm, bool copy) {
 struct StreamLaunch {
     std::vector<StreamSeg> segs;     // with sentinel
     std::vector<int64_t> bounds;
-    int grid = 0, cluster = 1, n_stages = 0, stage_bytes = 0, g_region_bytes = 0, threads = 0, chunk = 0;
+    int grid = 0, cluster = 1, n_stages = 0, stage_bytes = 0, g_region_bytes = 0, threads = 0, groups = 1, chunk = 0;
     int gdm = GDM_MIXED;
     unsigned long long *d_counter = nullptr;
     const StreamSeg *d_segs = nullptr;
@@ -694,6 +727,7 @@ struct StreamPlan {
         P.tensors = tensors; P.segs = L.d_segs; P.bounds = L.d_bounds; P.v = v; P.error_word = error_word;
         P.sc = sc; P.n_segs = static_cast<int>(L.segs.size()) - 1; P.n_stages = L.n_stages;
         P.stage_bytes = L.stage_bytes; P.g_region_bytes = L.g_region_bytes; P.consumer_threads = L.threads;
+        P.n_groups = L.groups;
         P.v_len = v_len;
         P.chunk = L.chunk; P.counter = L.d_counter; P.total_items = L.bounds.empty() ? 0 : L.bounds.back();
         if (P.chunk > 0) {
@@ -702,7 +736,7 @@ struct StreamPlan {
         }
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(L.grid);
-        cfg.blockDim = dim3(32 + L.threads);
+        cfg.blockDim = dim3(32 + L.threads * L.groups);
         cfg.dynamicSmemBytes = L.smem_bytes();
         cfg.stream = stream;
         cudaLaunchAttribute attr[1];
@@ -796,10 +830,10 @@ inline void stream_build_launch(const std::vector<StreamPlanInput::Item> &tensor
 
 // Largest cluster size (<= wanted) the device can keep resident with this
 // kernel's shared memory, and how many such clusters fit at once.
-inline void stream_probe_cluster(int sm_count, int threads, int wanted, int *cluster_size, int *n_clusters) {
+inline void stream_probe_cluster(int sm_count, int consumer_threads, int wanted, int *cluster_size, int *n_clusters) {
     *cluster_size = 0;
     *n_clusters = 0;
-    if (threads <= 0) threads = 256;
+    const int threads = consumer_threads > 0 ? consumer_threads : 512;
     const size_t smem = kCtrlBytes + 5 * (kStageElems * 10 + kVAreaFloats * 4);   // the larger of the two stage layouts
     for (int cs = wanted > 0 ? wanted : kMaxCluster; cs >= 1; cs >>= 1) {
         cudaLaunchConfig_t cfg = {};
@@ -823,11 +857,20 @@ inline void stream_probe_cluster(int sm_count, int threads, int wanted, int *clu
     }
 }
 
+// Consumer groups and threads per group of a launch (0 = defaults: two groups of 256).
+inline void stream_consumer_shape(int threads_opt, int groups_opt, int *threads, int *groups) {
+    *groups = groups_opt > 0 ? std::min(groups_opt, kMaxGroups) : kMaxGroups;
+    *threads = threads_opt > 0 ? threads_opt : 256;
+    while (*threads * *groups > kMaxConsumerWarps * 32) *threads -= 32;
+}
+
 inline void stream_finish_plan(const StreamPlanInput &in, int cluster_size, int n_clusters, StreamPlan *plan) {
-    const int threads = in.threads > 0 ? in.threads : 256;
+    int threads, groups;
+    stream_consumer_shape(in.threads, in.groups, &threads, &groups);
     const int ctas = in.ctas > 0 ? in.ctas : in.sm_count;
     stream_build_launch(in.stream_tensors, false, ctas, &plan->main);
     plan->main.threads = threads;
+    plan->main.groups = groups;
     plan->main.cluster = 1;
     // work distribution: ranges of `chunk` items from a shared counter unless static ranges were asked for
     if (in.chunk == kStaticRanges) plan->main.chunk = 0;
@@ -848,7 +891,7 @@ inline void stream_finish_plan(const StreamPlanInput &in, int cluster_size, int 
         int chunk = in.cluster_chunk;
         if (in.cluster_size == 0 && small_blocks && cluster_size > 4) {
             int cs4 = 0, n4 = 0;
-            stream_probe_cluster(in.sm_count, threads, 4, &cs4, &n4);
+            stream_probe_cluster(in.sm_count, threads * groups, 4, &cs4, &n4);
             if (cs4 == 4 && n4 > 0) { cluster_size = 4; n_clusters = n4; }
         }
         if (chunk == 0) chunk = (in.cluster_size == 0 && !small_blocks) ? kStaticRanges : 1;
@@ -856,6 +899,7 @@ inline void stream_finish_plan(const StreamPlanInput &in, int cluster_size, int 
         plan->clus.grid *= cluster_size;          // bounds are per cluster
         plan->clus.cluster = cluster_size;
         plan->clus.threads = threads;
+        plan->clus.groups = in.groups > 0 ? groups : 1;     // measured: a second group does not help the head kernel
         plan->clus.chunk = chunk == kStaticRanges ? 0 : chunk;
     }
 }

@@ -85,10 +85,23 @@ def test_ragged_shapes(grad_dtype, options):
     H.assert_parity(H.run_parity(ragged_workload(grad_dtype), options=options))
 
 
-@pytest.mark.parametrize("threads", [128, 512])
-def test_other_consumer_thread_counts(threads):
+@pytest.mark.parametrize("threads,groups", [(128, 1), (512, 1), (128, 2), (256, 1)])
+def test_other_consumer_shapes(threads, groups):
     w = W.scaled_rows(W.llama2_7b(n_layers=1), 128)
-    H.assert_parity(H.run_parity(w, steps=3, options={B.OPT_STREAM_THREADS: threads}))
+    H.assert_parity(H.run_parity(w, steps=3, options={B.OPT_STREAM_THREADS: threads, B.OPT_STREAM_GROUPS: groups}))
+
+
+def test_consumer_groups_give_identical_bits():
+    w = W.scaled_rows(W.llama2_7b(n_layers=2, vocab=1024), 512)
+    a = _run_steps(w, 1, 3)
+    dev = H.DeviceState(w, guarded=False)
+    opt = H.make_optimizer(w, {B.OPT_STREAM_GROUPS: 1})
+    for t in (1, 2, 3):
+        dev.draw_grads(t)
+        opt.step(dev.p, dev.g, dev.m, dev.v, t)
+    opt.sync_status()
+    opt.close()
+    assert _same(a, dev)
 
 
 @pytest.mark.parametrize("cluster", [1, 2, 4])
@@ -225,6 +238,7 @@ def test_full_size_llama2_7b_sampled_blocks():
     benchmark steps them; the oracle recomputes sampled blocks of every kind
     (token rows, heads, output-neuron rows of 4096 and 11008, norms) from the
     first, a middle and the last layer."""
+    torch.cuda.empty_cache()
     free, _ = torch.cuda.mem_get_info()
     if free < 75 * (1 << 30):
         pytest.skip("needs about 70 GB of free device memory")
@@ -258,6 +272,7 @@ def test_gpt2_small_full_model_hundred_steps():
 
 
 def _need_free_memory(gib):
+    torch.cuda.empty_cache()                # memory cached by earlier tests counts as free
     free, _ = torch.cuda.mem_get_info()
     if free < gib * (1 << 30):
         pytest.skip(f"needs about {gib} GiB of free device memory")
