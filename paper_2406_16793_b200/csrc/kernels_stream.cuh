@@ -1,11 +1,13 @@
 // The single-read streaming kernels.
 //
-// One persistent CTA per SM.  A producer thread walks the CTA's share of the
-// work and moves gradients, first moments and parameters from HBM into a ring
-// of shared-memory stages with bulk asynchronous copies (cp.async.bulk,
-// completion counted on an mbarrier).  The consumer warps wait for a stage,
-// reduce g*g over each block (Algorithm 1: v = (1-beta2) mean(g*g) + beta2 v),
-// turn the block's new v into a step size and apply the elementwise update,
+// One persistent CTA per SM.  A producer thread takes work items (from a
+// global counter, a range at a time, or from a fixed range of its own) and
+// moves gradients, first moments, parameters and the blocks' old v from HBM
+// into a ring of shared-memory stages with bulk asynchronous copies
+// (cp.async.bulk, completion counted on an mbarrier).  The consumer warps,
+// in one or two groups that own alternate work items, wait for a stage, reduce
+// g*g over each block (Algorithm 1: v = (1-beta2) mean(g*g) + beta2 v), turn
+// the block's new v into a step size and apply the elementwise update,
 // writing m and p back with 16-byte stores.
 //
 // Three kinds of stage:
@@ -17,6 +19,10 @@
 //           block is split over a cluster).
 //   APPLY   g, m, p of one chunk of that block: g is fetched a second time, a
 //           few microseconds after the first, and is served by L2.
+//
+// A block is always reduced in one fixed order (per thread, per warp, per
+// group, per cluster rank), whichever CTA or group gets it, so results do not
+// depend on the launch shape or on how the work was handed out.
 //
 // Every wait is bounded: a wait that gives up sets the abort flag and the
 // handle's error word, and all roles leave through the common exit.
@@ -38,9 +44,9 @@ constexpr int kWarpBlockMaxL = 1024;              // blocks up to this length ar
 constexpr int kCtrlBytes = 2048;                  // barriers, stage descriptors, reduction slots
 constexpr int kVAreaFloats = 272;                 // per stage: the old v of the stage's blocks (16-byte windows)
 constexpr int kMaxStages = 8;
-constexpr int kMaxConsumerWarps = 16;                // over all consumer groups
+constexpr int kMaxConsumerWarps = 16;              // over all consumer groups
 constexpr int kMaxGroups = 2;                     // consumer groups; each owns every n-th work item
-constexpr int kExchangeSlots = 4;                 // cluster exchange slots (long blocks in flight per CTA pair of groups)
+constexpr int kExchangeSlots = 4;                 // slots of the cluster exchange, used in turn by consecutive long blocks
 constexpr int kMaxCluster = 8;
 constexpr int kItemSlots = 8;                     // block indices in flight from a cluster's first CTA to its peers
 constexpr int kStaticRanges = 1000000;            // AM_OPT_STREAM_CHUNK value that selects static ranges
@@ -94,16 +100,16 @@ struct StreamParams {
 };
 
 struct Control {            // first kCtrlBytes of dynamic shared memory
-    unsigned long long full[kMaxStages];
-    unsigned long long empty[kMaxStages];
-    unsigned long long redbar[kMaxGroups];
-    unsigned long long xbar[kExchangeSlots];
-    double red[kMaxGroups][2][kMaxConsumerWarps];
-    double xpart[kExchangeSlots][kMaxCluster];
-    float redv[kMaxGroups][2];
-    int abort_flag;
+    unsigned long long full[kMaxStages];     // producer -> consumers: the stage's copies have landed
+    unsigned long long empty[kMaxStages];    // consumers -> producer: every consumer warp is done with the stage
+    unsigned long long redbar[kMaxGroups];   // barrier of one consumer group (an mbarrier, so that waits are bounded)
+    unsigned long long xbar[kExchangeSlots]; // cluster exchange: all CTAs' partial sums of a block have arrived
+    double red[kMaxGroups][2][kMaxConsumerWarps];   // per-warp partial sums of a group, double buffered
+    double xpart[kExchangeSlots][kMaxCluster];      // partial sums of the cluster's CTAs, by rank
+    float redv[kMaxGroups][2];               // old v of the block being reduced, broadcast to the group
+    int abort_flag;                          // raised by a wait that gave up; every wait polls it
     int pad;
-    unsigned long long ibar[kItemSlots];   // cluster launches: "the next block index has arrived"
+    unsigned long long ibar[kItemSlots];     // cluster launches: "the next block index has arrived"
     long long next_item[kItemSlots];
     StageMeta meta[kMaxStages];
 };
