@@ -45,7 +45,11 @@ typedef enum {
     AM_ROWS   = 1,  /* value, attn.proj, mlp: one block per output neuron (row)    */
     AM_HEADS  = 2,  /* query, key: one block per head = rows/n_heads rows          */
     AM_TOKENS = 3,  /* embed, output: one block per token row                      */
-    AM_FIXED  = 4   /* explicit block length (any divisor of numel)                */
+    AM_FIXED  = 4,  /* explicit block length (any divisor of numel)                */
+    AM_PART   = 5   /* a contiguous PART of one block whose other parts are held elsewhere (a flat
+                       shard that cuts a block between data-parallel ranks): rows = 1, cols = the
+                       local length, fixed_block_len = the length of the whole block.  The sum of
+                       g*g over the whole block is supplied to the step (see am_step_extras)      */
 } am_kind;
 
 typedef enum { AM_F32 = 0, AM_BF16 = 1 } am_dtype;
@@ -66,7 +70,8 @@ typedef struct am_tensor_desc {
     int64_t rows, cols;
     int32_t kind;               /* am_kind */
     int32_t n_heads;            /* AM_HEADS only; rows % n_heads == 0 */
-    int64_t fixed_block_len;    /* AM_FIXED only; (rows*cols) % fixed_block_len == 0 */
+    int64_t fixed_block_len;    /* AM_FIXED: block length, (rows*cols) % fixed_block_len == 0;
+                                   AM_PART: length of the whole block, >= rows*cols */
     int32_t grad_dtype;         /* am_dtype of this tensor's gradient */
     int32_t apply_weight_decay; /* 0: skip the decay line for this tensor */
 } am_tensor_desc;
@@ -77,6 +82,7 @@ typedef struct am_tensor_desc {
 typedef struct am_table_row {
     int64_t numel, block_len, n_blocks, v_offset;
     int32_t kind, grad_dtype, wd, pad;
+    int64_t mean_len;           /* divisor of the block mean: block_len, except for AM_PART (whole block's length) */
 } am_table_row;
 
 /* eta, beta1, beta2, eps, lambda of Algorithm 1.  Doubles, so the caller's
@@ -123,7 +129,8 @@ int adammini_set_hparams(am_handle *h, const am_hparams *hp);
  *   params, grads, m : host arrays of n_tensors DEVICE pointers, in table order;
  *                      tensor i holds rows*cols contiguous elements
  *                      (params/m float32, grads of the tensor's grad_dtype).
- *                      All must be 16-byte aligned.  grads are only read.
+ *                      All must be 16-byte aligned (AM_PART tensors: aligned to their element
+ *                      size, since a shard may cut a block anywhere).  grads are only read.
  *   v                : DEVICE pointer, float32[total_blocks], 16-byte aligned.
  *   step             : t, 1-based.
  *   cuda_stream      : a cudaStream_t (NULL = the legacy default stream).
@@ -151,11 +158,22 @@ typedef struct am_step_extras {
     double grad_scale;
     const float *grad_scale_device;
     const float *skip_flag;
+    const double *part_sums;   /* required when the table has AM_PART tensors: DEVICE array with one entry
+                                  per AM_PART tensor, in table order: the sum of g*g (unscaled gradients)
+                                  over the WHOLE block, i.e. the parts' sums from adammini_part_sums added
+                                  up over all holders (an all-reduce between data-parallel ranks) */
 } am_step_extras;
 
 /* adammini_step with extras (`ex` may be NULL, which is adammini_step). */
 int adammini_step_ex(am_handle *h, void *const *params, const void *const *grads, void *const *m,
                      float *v, int64_t step, void *cuda_stream, const am_step_extras *ex);
+
+/* Sums of g*g of the table's AM_PART tensors (this holder's parts only), written to
+ * `out` (DEVICE array, one double per AM_PART tensor in table order), asynchronously on
+ * the stream.  grads: as for adammini_step (only the AM_PART entries are read).  The
+ * caller adds the parts of every block over all its holders and passes the totals to
+ * adammini_step_ex as am_step_extras.part_sums. */
+int adammini_part_sums(am_handle *h, const void *const *grads, double *out, void *cuda_stream);
 
 /* The same step for callers whose state lives in HOST memory (offloaded
  * optimizer state): params, grads, m are host arrays of HOST pointers, v is a
@@ -253,7 +271,8 @@ typedef enum {
     AM_Q_BYTES_TWOPASS     = 12,
     AM_Q_STREAM_CTAS       = 13, /* launch shape of the streaming kernel */
     AM_Q_CLUSTER_SIZE      = 14,
-    AM_Q_CLUSTER_COUNT     = 15
+    AM_Q_CLUSTER_COUNT     = 15,
+    AM_Q_PART_TENSORS      = 16  /* number of AM_PART tensors in the table */
 } am_query;
 int adammini_query(const am_handle *h, int32_t what, int64_t *value);
 

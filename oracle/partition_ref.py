@@ -15,7 +15,7 @@ from __future__ import annotations
 from dataclasses import dataclass
 from typing import Iterable, List, Sequence
 
-WHOLE, ROWS, HEADS, TOKENS, FIXED = 0, 1, 2, 3, 4
+WHOLE, ROWS, HEADS, TOKENS, FIXED, PART = 0, 1, 2, 3, 4, 5
 F32, BF16 = 0, 1
 
 
@@ -39,6 +39,7 @@ class TableRow:
     kind: int
     grad_dtype: int
     wd: int
+    mean_len: int = 0       # divisor of the block mean; differs from block_len only for PART
 
 
 def block_len_of(d: TensorDesc) -> int:
@@ -56,6 +57,10 @@ def block_len_of(d: TensorDesc) -> int:
         if d.fixed_block_len <= 0 or numel % d.fixed_block_len:
             raise ValueError("fixed block length must divide numel")
         return d.fixed_block_len
+    if d.kind == PART:                       # a part of one block held elsewhere too: one local block
+        if d.rows != 1 or d.fixed_block_len < numel:
+            raise ValueError("a part cannot be longer than its block")
+        return numel
     raise ValueError(f"unknown kind {d.kind}")
 
 
@@ -70,7 +75,8 @@ def build_table(descs: Sequence[TensorDesc]) -> tuple[List[TableRow], int]:
         L = block_len_of(d)
         nb = numel // L
         rows.append(TableRow(numel, L, nb, v_offset, d.kind, d.grad_dtype,
-                             1 if d.apply_weight_decay else 0))
+                             1 if d.apply_weight_decay else 0,
+                             d.fixed_block_len if d.kind == PART else L))
         v_offset += nb
     return rows, v_offset
 

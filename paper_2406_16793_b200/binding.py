@@ -14,14 +14,15 @@ from typing import Iterable, List, Optional, Sequence
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIBRARY = os.environ.get("ADAMMINI_LIBRARY") or os.path.join(_HERE, "libadammini.so")
 
-WHOLE, ROWS, HEADS, TOKENS, FIXED = 0, 1, 2, 3, 4
+WHOLE, ROWS, HEADS, TOKENS, FIXED, PART = 0, 1, 2, 3, 4, 5
 F32, BF16 = 0, 1
 
 OPT_PATH, OPT_STREAM_CTAS, OPT_CLUSTER_SIZE, OPT_STREAM_THREADS, OPT_PROFILE, OPT_STREAM_CHUNK, OPT_CLUSTER_CHUNK, OPT_STATISTIC, OPT_STREAM_GROUPS = 0, 1, 2, 3, 4, 5, 6, 7, 8
 STAT_MEAN, STAT_MAX, STAT_MIN, STAT_ONE_NORM, STAT_TWO_NORM = 0, 1, 2, 3, 4
 (Q_LAUNCHES_PER_STEP, Q_SCRATCH_BYTES, Q_TOTAL_BLOCKS, Q_TOTAL_ELEMENTS, Q_ELEMENTS_SMALL,
  Q_ELEMENTS_STREAM, Q_ELEMENTS_CLUSTER, Q_ELEMENTS_TWOPASS, Q_ALGORITHMIC_BYTES, Q_BYTES_SMALL,
- Q_BYTES_STREAM, Q_BYTES_CLUSTER, Q_BYTES_TWOPASS, Q_STREAM_CTAS, Q_CLUSTER_SIZE, Q_CLUSTER_COUNT) = range(16)
+ Q_BYTES_STREAM, Q_BYTES_CLUSTER, Q_BYTES_TWOPASS, Q_STREAM_CTAS, Q_CLUSTER_SIZE, Q_CLUSTER_COUNT,
+ Q_PART_TENSORS) = range(17)
 
 
 class TensorDesc(ctypes.Structure):
@@ -33,7 +34,7 @@ class TensorDesc(ctypes.Structure):
 class TableRow(ctypes.Structure):
     _fields_ = [("numel", ctypes.c_int64), ("block_len", ctypes.c_int64), ("n_blocks", ctypes.c_int64),
                 ("v_offset", ctypes.c_int64), ("kind", ctypes.c_int32), ("grad_dtype", ctypes.c_int32),
-                ("wd", ctypes.c_int32), ("pad", ctypes.c_int32)]
+                ("wd", ctypes.c_int32), ("pad", ctypes.c_int32), ("mean_len", ctypes.c_int64)]
 
 
 class HParams(ctypes.Structure):
@@ -43,7 +44,8 @@ class HParams(ctypes.Structure):
 
 class StepExtras(ctypes.Structure):
     _fields_ = [("params_bf16", ctypes.POINTER(ctypes.c_void_p)), ("grad_scale", ctypes.c_double),
-                ("grad_scale_device", ctypes.c_void_p), ("skip_flag", ctypes.c_void_p)]
+                ("grad_scale_device", ctypes.c_void_p), ("skip_flag", ctypes.c_void_p),
+                ("part_sums", ctypes.c_void_p)]
 
 
 class AdamMiniError(RuntimeError):
@@ -68,6 +70,7 @@ _SIGNATURES = {
     "adammini_step_ex": (ctypes.c_int, [ctypes.c_void_p, ctypes.POINTER(ctypes.c_void_p), ctypes.POINTER(ctypes.c_void_p),
                                         ctypes.POINTER(ctypes.c_void_p), ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p,
                                         ctypes.POINTER(StepExtras)]),
+    "adammini_part_sums": (ctypes.c_int, [ctypes.c_void_p, ctypes.POINTER(ctypes.c_void_p), ctypes.c_void_p, ctypes.c_void_p]),
     "adammini_step_host": (ctypes.c_int, [ctypes.c_void_p, ctypes.POINTER(ctypes.c_void_p), ctypes.POINTER(ctypes.c_void_p),
                                           ctypes.POINTER(ctypes.c_void_p), ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64]),
     "adammini_step_tensor_noalloc": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
@@ -242,7 +245,7 @@ class AdamMini:
 
     def step_ex(self, params: Sequence, grads: Sequence, m: Sequence, v, step: int, stream: int = 0, *,
                 params_bf16: Optional[Sequence] = None, grad_scale: float = 1.0, grad_scale_device=None,
-                skip_flag=None) -> None:
+                skip_flag=None, part_sums=None) -> None:
         """A step with the optional extras of adammini_step_ex: bf16 copies of the
         updated parameters, a gradient scale (host value and/or device scalar)
         and a device flag that turns the step into a no-op."""
@@ -257,7 +260,14 @@ class AdamMini:
         ex.grad_scale = float(grad_scale)
         ex.grad_scale_device = int(grad_scale_device.data_ptr()) if grad_scale_device is not None else None
         ex.skip_flag = int(skip_flag.data_ptr()) if skip_flag is not None else None
+        ex.part_sums = int(part_sums.data_ptr()) if part_sums is not None else None
         _check(load().adammini_step_ex(self._h, pa, ga, ma, vp, int(step), stream or None, ctypes.byref(ex)), self._h)
+
+    def part_sums(self, grads: Sequence, out, stream: int = 0) -> None:
+        """Sums of g*g of this holder's parts of cut blocks (the table's PART
+        tensors, in table order) into `out`, a device float64 tensor."""
+        ga = _ptr_array(_data_ptrs(grads))
+        _check(load().adammini_part_sums(self._h, ga, int(out.data_ptr()), stream or None), self._h)
 
     def step_host(self, params: Sequence, grads: Sequence, m: Sequence, v, step: int,
                   staging_bytes: int = 0) -> None:

@@ -63,7 +63,9 @@ int build_plan(am_handle *h) {
     const int n = static_cast<int>(h->rows.size());
     h->path.assign(n, PATH_TWOPASS);
     h->host_tensors.assign(n, DevTensor{});
-    std::vector<Seg> small_segs, piece_segs, block_segs;
+    std::vector<Seg> small_segs, piece_segs, block_segs, part_segs;
+    std::vector<int32_t> part_tensors;
+    int64_t part_units = 0;
     int64_t small_units = 0, piece_units = 0, block_units = 0;
     for (int k = 0; k < 4; ++k) h->elems_by_path[k] = h->bytes_by_path[k] = 0;
     h->algorithmic_bytes = 0;
@@ -92,10 +94,13 @@ int build_plan(am_handle *h) {
         t.v_offset = r.v_offset;
         t.gdtype = r.grad_dtype;
         t.wd = r.wd;
+        t.mean_len = r.mean_len;
+        t.part_index = -1;
         const int64_t gsz = r.grad_dtype == AM_BF16 ? 2 : 4;
 
         int path;
-        if (r.block_len <= kSmallMaxL) path = PATH_SMALL;
+        if (r.kind == AM_PART) path = PATH_TWOPASS;          // its sum of squares comes from outside
+        else if (r.block_len <= kSmallMaxL) path = PATH_SMALL;
         else if (h->opt[AM_OPT_PATH] == 1 || h->opt[AM_OPT_STATISTIC] != 0) path = PATH_TWOPASS;
         else path = stream_classify(r.block_len, r.grad_dtype, h->n_clusters > 0);
         h->path[i] = path;
@@ -129,8 +134,16 @@ int build_plan(am_handle *h) {
             Seg s;
             s.unit_begin = piece_units;
             s.tensor = i;
-            s.aux = (r.block_len % 4 == 0) ? 1 : 0;
+            s.aux = (r.block_len % 4 == 0 && r.kind != AM_PART) ? 1 : 0;   // parts may start at any element
             piece_segs.push_back(s);
+            if (r.kind == AM_PART) {
+                t.part_index = static_cast<int32_t>(part_tensors.size());
+                part_tensors.push_back(i);
+                Seg ps = s;
+                ps.unit_begin = part_units;
+                part_segs.push_back(ps);
+                part_units += r.n_blocks * ppb;
+            }
             Seg b;
             b.unit_begin = block_units;
             b.tensor = i;
@@ -142,6 +155,7 @@ int build_plan(am_handle *h) {
             stream_add_tensor(sin, i, r, path);
         }
     }
+    if (part_units > 0x7fffffffLL) return AM_ERR_TOO_LARGE;
     if (small_units > 0x7fffffffLL || piece_units > 0x7fffffffLL || ceil_div(block_units, kThreads / 32) > 0x7fffffffLL)
         return AM_ERR_TOO_LARGE;
 
@@ -159,6 +173,8 @@ int build_plan(am_handle *h) {
     const size_t o_partials = take(sizeof(double) * std::max<int64_t>(piece_units, 1));
     const size_t o_steps = take(sizeof(float) * std::max<int64_t>(block_units, 1));
     const size_t o_stream = take(std::max<size_t>(sp.table_bytes(), 16));
+    const size_t o_part_segs = take(sizeof(Seg) * std::max<size_t>(part_segs.size(), 1));
+    const size_t o_part_list = take(sizeof(int32_t) * std::max<size_t>(part_tensors.size(), 1));
     h->arena_bytes = off;
     AM_CUDA(h, cudaMalloc(&h->arena, h->arena_bytes));
     char *base = static_cast<char *>(h->arena);
@@ -171,6 +187,14 @@ int build_plan(am_handle *h) {
     h->n_small_segs = static_cast<int>(small_segs.size());
     h->n_piece_segs = static_cast<int>(piece_segs.size());
     h->n_block_segs = static_cast<int>(block_segs.size());
+    h->d_part_segs = reinterpret_cast<Seg *>(base + o_part_segs);
+    h->d_part_tensors = reinterpret_cast<int32_t *>(base + o_part_list);
+    h->n_parts = static_cast<int>(part_tensors.size());
+    h->part_units = part_units;
+    if (!part_segs.empty()) {
+        AM_CUDA(h, cudaMemcpy(h->d_part_segs, part_segs.data(), sizeof(Seg) * part_segs.size(), cudaMemcpyHostToDevice));
+        AM_CUDA(h, cudaMemcpy(h->d_part_tensors, part_tensors.data(), sizeof(int32_t) * part_tensors.size(), cudaMemcpyHostToDevice));
+    }
     h->small_units = small_units;
     h->piece_units = piece_units;
     h->block_units = block_units;
@@ -337,6 +361,7 @@ int adammini_query(const am_handle *h, int32_t what, int64_t *value) {
     case AM_Q_BYTES_TWOPASS: *value = h->bytes_by_path[PATH_TWOPASS]; break;
     case AM_Q_STREAM_CTAS: *value = h->stream.main.grid; break;
     case AM_Q_CLUSTER_SIZE: *value = h->stream.clus.active() ? h->stream.clus.cluster : 0; break;
+    case AM_Q_PART_TENSORS: *value = h->n_parts; break;
     case AM_Q_CLUSTER_COUNT: *value = h->stream.clus.active() ? h->stream.clus.grid / h->stream.clus.cluster : 0; break;
     default: return AM_ERR_INVALID_ARGUMENT;
     }
@@ -359,9 +384,17 @@ int adammini_step_ex(am_handle *h, void *const *params, const void *const *grads
     if (!params || !grads || !m || !v) return AM_ERR_INVALID_ARGUMENT;
     for (int i = 0; i < n; ++i) {
         if (!params[i] || !grads[i] || !m[i]) return AM_ERR_INVALID_ARGUMENT;
-        if (!aligned16(params[i]) || !aligned16(grads[i]) || !aligned16(m[i])) return AM_ERR_MISALIGNED;
+        if (h->rows[i].kind == AM_PART) {      // a part of a block may start at any element
+            const uintptr_t gmask = h->rows[i].grad_dtype == AM_BF16 ? 1u : 3u;
+            if ((reinterpret_cast<uintptr_t>(params[i]) & 3u) || (reinterpret_cast<uintptr_t>(m[i]) & 3u) ||
+                (reinterpret_cast<uintptr_t>(grads[i]) & gmask))
+                return AM_ERR_MISALIGNED;
+        } else if (!aligned16(params[i]) || !aligned16(grads[i]) || !aligned16(m[i])) {
+            return AM_ERR_MISALIGNED;
+        }
     }
     if (!aligned16(v)) return AM_ERR_MISALIGNED;
+    if (h->n_parts > 0 && (!ex || !ex->part_sums || h->opt[AM_OPT_STATISTIC] != 0)) return AM_ERR_INVALID_ARGUMENT;
     if (ex && ex->params_bf16)
         for (int i = 0; i < n; ++i)
             if (!aligned16(ex->params_bf16[i])) return AM_ERR_MISALIGNED;
@@ -392,6 +425,7 @@ int adammini_step_ex(am_handle *h, void *const *params, const void *const *grads
     sc.skip_flag = ex ? ex->skip_flag : nullptr;
     sc.statistic = static_cast<int32_t>(h->opt[AM_OPT_STATISTIC]);
     sc.pad = 0;
+    sc.part_sums = ex ? ex->part_sums : nullptr;
 
     const bool prof = h->opt[AM_OPT_PROFILE] != 0;
     cudaEvent_t *pev = prof ? &h->prof_ev[(h->prof_steps % h->opt[AM_OPT_PROFILE]) * 5] : nullptr;
@@ -456,6 +490,49 @@ int adammini_get_profile(am_handle *h, float *ms, int32_t *n_steps) {
     }
     for (int k = 0; k < 4; ++k) ms[k] = static_cast<float>(sum[k] / static_cast<double>(n));
     if (n_steps) *n_steps = static_cast<int32_t>(n);
+    return AM_OK;
+}
+
+int adammini_part_sums(am_handle *h, const void *const *grads, double *out, void *cuda_stream) {
+    if (!h || !h->planned || !grads) return AM_ERR_INVALID_ARGUMENT;
+    if (h->n_parts == 0) return AM_OK;
+    if (!out) return AM_ERR_INVALID_ARGUMENT;
+    const int n = static_cast<int>(h->rows.size());
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    int dev = -1;
+    AM_CUDA(h, cudaGetDevice(&dev));
+    if (dev != h->device) return AM_ERR_INVALID_ARGUMENT;
+    // the kernels read the gradient addresses from the device tensor table: refresh those
+    bool changed = !h->ptrs_valid;
+    for (int i = 0; i < n; ++i) {
+        if (h->rows[i].kind != AM_PART) continue;
+        if (!grads[i]) return AM_ERR_INVALID_ARGUMENT;
+        if (reinterpret_cast<uintptr_t>(grads[i]) & (h->rows[i].grad_dtype == AM_BF16 ? 1u : 3u)) return AM_ERR_MISALIGNED;
+        if (h->host_tensors[i].g != grads[i]) {
+            h->host_tensors[i].g = grads[i];
+            changed = true;
+        }
+    }
+    if (changed) {
+        const int k = h->next_pinned;
+        h->next_pinned ^= 1;
+        if (h->ev_pending[k]) {
+            AM_CUDA(h, cudaEventSynchronize(h->ev[k]));
+            h->ev_pending[k] = false;
+        }
+        std::memcpy(h->pinned[k], h->host_tensors.data(), sizeof(DevTensor) * n);
+        AM_CUDA(h, cudaMemcpyAsync(h->d_tensors, h->pinned[k], sizeof(DevTensor) * n, cudaMemcpyHostToDevice, stream));
+        AM_CUDA(h, cudaEventRecord(h->ev[k], stream));
+        h->ev_pending[k] = true;
+        // the other addresses of the table may be stale: the next step uploads it again
+        h->ptrs_valid = false;
+    }
+    twopass_partial_kernel<<<static_cast<unsigned>(h->part_units), kThreads, 0, stream>>>(
+        h->d_tensors, h->d_part_segs, h->n_parts, h->d_partials, 1.f, nullptr, nullptr, 0);
+    AM_CUDA(h, cudaGetLastError());
+    part_sums_kernel<<<static_cast<unsigned>(ceil_div(h->n_parts, kThreads / 32)), kThreads, 0, stream>>>(
+        h->d_tensors, h->d_part_tensors, h->n_parts, h->d_partials, out);
+    AM_CUDA(h, cudaGetLastError());
     return AM_OK;
 }
 
@@ -590,6 +667,8 @@ extern "C" int adammini_step_tensor_noalloc(void *param, const void *grad, void 
     }
     t.piece_base = 0;
     t.block_base = 0;      // block_steps is indexed by block inside the array
+    t.mean_len = block_len;
+    t.part_index = -1;
     if (t.n_blocks > AM_NOALLOC_MAX_BLOCKS) return AM_ERR_TOO_LARGE;
     const int64_t pieces = t.n_blocks * t.pieces_per_block;
     if (pieces > AM_NOALLOC_MAX_PIECES) return AM_ERR_TOO_LARGE;
@@ -624,6 +703,7 @@ extern "C" int adammini_step_tensor_noalloc(void *param, const void *grad, void 
     sc.skip_flag = nullptr;
     sc.statistic = 0;
     sc.pad = 0;
+    sc.part_sums = nullptr;
 
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const int vec = block_len % 4 == 0 ? 1 : 0;

@@ -40,6 +40,9 @@ struct DevTensor {
     int64_t pieces_per_block;
     int64_t piece_base;       // first partial of this tensor in the scratch array
     int64_t block_base;       // first per-block step size of this tensor in the scratch array
+    int64_t mean_len;         // divisor of the block mean (the whole block's length for a part of a block)
+    int32_t part_index;       // >= 0: this tensor is a part of a block; index of its externally supplied sum
+    int32_t pad2;
 };
 
 // A run of work units that belong to one tensor; units are numbered
@@ -63,6 +66,7 @@ struct StepScalars {
     const float *skip_flag;   // device scalar; non-zero: the step leaves everything untouched
     int32_t statistic;        // block statistic: 0 mean, 1 max, 2 min, 3 one-norm, 4 two-norm of g*g
     int32_t pad;
+    const double *part_sums;  // whole-block sums of g*g for tensors that are parts of blocks
 };
 
 }  // namespace am

@@ -357,12 +357,34 @@ twopass_finalize_kernel(const DevTensor *__restrict__ tensors, const Seg *__rest
     for (int64_t j = lane; j < t.pieces_per_block; j += 32) s = stat_combine(s, src[j], statistic);
     s = warp_stat(s, statistic);
     if (lane == 0) {
+        if (t.part_index >= 0) {
+            // a part of a block: the whole block's sum of g*g comes from outside (unscaled gradients)
+            const double gs = static_cast<double>(effective_gscale(sc.gscale, sc.gscale_dev));
+            s = sc.part_sums[t.part_index] * gs * gs;
+        }
         float vn;
-        const float st = block_step_from_statistic(stat_finish(s, static_cast<double>(t.L), statistic),
+        const float st = block_step_from_statistic(stat_finish(s, static_cast<double>(t.mean_len), statistic),
                                                    v[t.v_offset + b], sc, &vn);
         v[t.v_offset + b] = vn;
         block_steps[t.block_base + b] = st;
     }
+}
+
+// Local sums of g*g of the tensors that are parts of blocks: one warp per such
+// tensor adds the tensor's partial sums (written by twopass_partial_kernel with
+// a gradient scale of 1) in a fixed order.
+__global__ void __launch_bounds__(kThreads)
+part_sums_kernel(const DevTensor *__restrict__ tensors, const int32_t *__restrict__ part_tensors, int n_parts,
+                 const double *__restrict__ partials, double *__restrict__ out) {
+    const int unit = blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
+    if (unit >= n_parts) return;
+    const int lane = threadIdx.x & 31;
+    const DevTensor &t = tensors[part_tensors[unit]];
+    const double *src = partials + t.piece_base;
+    double s = 0.0;
+    for (int64_t j = lane; j < t.pieces_per_block; j += 32) s += src[j];
+    s = warp_sum(s);
+    if (lane == 0) out[unit] = s;
 }
 
 template <int GD>

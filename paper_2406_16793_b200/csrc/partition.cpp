@@ -28,6 +28,9 @@ int64_t block_length(const am_tensor_desc &d, int64_t numel) {
     case AM_FIXED:
         if (d.fixed_block_len <= 0 || numel % d.fixed_block_len != 0) return 0;
         return d.fixed_block_len;
+    case AM_PART:               // the local part of one longer block is this tensor's single "block"
+        if (d.rows != 1 || d.fixed_block_len < numel) return 0;
+        return numel;
     default:
         return 0;
     }
@@ -54,7 +57,7 @@ int adammini_partition_build(const am_tensor_desc *descs, int32_t n_tensors, am_
                 delete part;
                 return AM_ERR_SHAPE;
             }
-            if ((d.grad_dtype != AM_F32 && d.grad_dtype != AM_BF16) || d.kind < AM_WHOLE || d.kind > AM_FIXED) {
+            if ((d.grad_dtype != AM_F32 && d.grad_dtype != AM_BF16) || d.kind < AM_WHOLE || d.kind > AM_PART) {
                 delete part;
                 return AM_ERR_INVALID_ARGUMENT;
             }
@@ -73,6 +76,7 @@ int adammini_partition_build(const am_tensor_desc *descs, int32_t n_tensors, am_
             r.grad_dtype = d.grad_dtype;
             r.wd = d.apply_weight_decay ? 1 : 0;
             r.pad = 0;
+            r.mean_len = d.kind == AM_PART ? d.fixed_block_len : L;
             part->rows.push_back(r);
             v_offset += r.n_blocks;
         }

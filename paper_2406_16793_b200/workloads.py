@@ -24,7 +24,7 @@ from typing import Dict, List, Optional
 import torch
 
 # Partition kinds and dtype codes (values of the library's C enums).
-WHOLE, ROWS, HEADS, TOKENS, FIXED = 0, 1, 2, 3, 4
+WHOLE, ROWS, HEADS, TOKENS, FIXED, PART = 0, 1, 2, 3, 4, 5
 F32, BF16 = 0, 1
 
 BASE_SEED = 20240616
@@ -50,7 +50,7 @@ class TensorSpec:
 
     @property
     def block_len(self) -> int:
-        if self.kind == WHOLE:
+        if self.kind in (WHOLE, PART):      # PART: the local part of a longer block is the tensor's one block
             return self.numel
         if self.kind in (ROWS, TOKENS):
             return self.cols

@@ -408,3 +408,73 @@ def test_more_than_2_to_31_elements_in_one_tensor(L):
     w = W.Workload(f"huge-L{L}", 70, [W.TensorSpec("t", 1, numel, W.FIXED, fixed_block_len=L, grad_dtype=W.BF16)],
                    W.GradRecipe(-3.0, -1.0), steps=2)
     H.assert_parity(H.run_sampled_runs(w, steps=2, run_elems=4096, n_runs=12))
+
+
+def _flat_model():
+    T = W.TensorSpec
+    bf = dict(grad_dtype=W.BF16)
+    tensors = [
+        T("embed", 300, 4096, W.TOKENS, **bf),
+        T("query", 256, 4096, W.HEADS, n_heads=2, **bf),
+        T("down", 40, 11008, W.ROWS, **bf),
+        T("odd", 9, 1001, W.ROWS, **bf),
+        T("short", 500, 36, W.ROWS, grad_dtype=W.F32),
+        T("norm", 1, 4096, W.WHOLE, **bf),
+        T("whole", 1, 3 << 20, W.WHOLE, **bf),
+    ]
+    return W.Workload("flat-shards", 62, tensors, W.GradRecipe(-4.0, -1.0), steps=3)
+
+
+@pytest.mark.parametrize("world", [2, 3, 5])
+def test_flat_shards_that_cut_blocks(world):
+    """FSDP-style flat shards: every rank owns an equal contiguous range of the
+    flat parameter space, blocks cut by a range boundary get their sum of g*g
+    through one exchange of partial sums.  The ranks' shares are stepped one
+    after the other on the one GPU (phase 1 of all, the exchange, phase 2 of
+    all) and must match the oracle's unsharded run; blocks that no boundary
+    cuts must equal the unsharded GPU run bit for bit."""
+    from paper_2406_16793_b200 import sharding
+    w = _flat_model()
+    ref = _run_steps(w, 1, w.steps)
+    dev = H.DeviceState(w, guarded=True)
+    ora = ostep_state(w, dev)
+    ranks = [sharding.ShardedFlatStep(w.tensors, world, r, **w.hparams) for r in range(world)]
+    assert sum(r.n_parts for r in ranks) >= 2                      # some block is cut
+    v_local = [torch.zeros(max(r.local_blocks, 1), device="cuda") for r in ranks]
+    for t in range(1, w.steps + 1):
+        dev.draw_grads(t)
+        gathered = torch.stack([r.local_sums(dev.g).clone() for r in ranks])      # stands in for the all-gather
+        for r, v in zip(ranks, v_local):
+            r.combine(gathered)
+            r.apply(dev.p, dev.g, dev.m, v, t)
+        H.oracle_step_all(ora, [g.cpu() for g in dev.g], t, w.hparams)
+    torch.cuda.synchronize()
+    assert dev.guards_intact()
+    cut = set()
+    for r in ranks:
+        cut |= set(r.plan.part_keys)
+    for i, spec in enumerate(w.tensors):
+        L = spec.block_len
+        assert H.block_relative_error(dev.p[i].cpu().numpy(), ora.p[i], L) <= H.TOL
+        assert H.block_relative_error(dev.m[i].cpu().numpy(), ora.m[i], L) <= H.TOL
+        same = (dev.p[i] == ref.p[i]).view(-1, L).all(dim=1).cpu()
+        for b in range(spec.n_blocks):
+            if (i, b) not in cut:
+                assert bool(same[b]), (i, b)
+    # every holder of a cut block keeps the same second moment, and it matches the oracle
+    v_off = np.cumsum([0] + [t.n_blocks for t in w.tensors])
+    for r, v in zip(ranks, v_local):
+        k = 0
+        for p in r.pieces:
+            got = v[k:k + p.n_blocks].cpu().numpy()
+            want = ora.v[p.tensor][p.block:p.block + p.n_blocks]
+            assert H.v_relative_error(got, want) <= H.TOL
+            k += p.n_blocks
+    for r in ranks:
+        r.close()
+
+
+def ostep_state(w, dev):
+    from oracle import step as ostep
+    return ostep.OracleState([p.cpu() for p in dev.p], [t.block_len for t in w.tensors],
+                             [bool(t.apply_weight_decay) for t in w.tensors])

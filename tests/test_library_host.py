@@ -34,8 +34,16 @@ def test_library_exports_every_declared_entry_point():
     assert set(binding.exported_names()) == set(names)
 
 
+def parts_workload():
+    T = W.TensorSpec
+    return W.Workload("parts", 80, [T("tail", 1, 1000, W.PART, fixed_block_len=4096, grad_dtype=W.BF16),
+                                    T("rows", 6, 4096, W.ROWS, grad_dtype=W.BF16),
+                                    T("head", 1, 3001, W.PART, fixed_block_len=11008, grad_dtype=W.BF16)],
+                      W.GradRecipe(-4.0, -1.0), steps=2)
+
+
 def workloads():
-    return [W.tiny_gpt2(), W.gpt2_small(), W.llama2_7b(), W.llama3_8b()] + \
+    return [W.tiny_gpt2(), W.gpt2_small(), W.llama2_7b(), W.llama3_8b(), parts_workload()] + \
            [W.flat_sweep(L) for L in (1, 128, 4096, 524288, 1 << 30)]
 
 
@@ -48,8 +56,8 @@ def test_partition_table_is_bit_exact(w):
         for t in w.tensors])
     assert total == want_total and len(rows) == len(want)
     for got, ref in zip(rows, want):
-        assert (got.numel, got.block_len, got.n_blocks, got.v_offset, got.kind, got.grad_dtype, got.wd) == \
-               (ref.numel, ref.block_len, ref.n_blocks, ref.v_offset, ref.kind, ref.grad_dtype, ref.wd)
+        assert (got.numel, got.block_len, got.n_blocks, got.v_offset, got.kind, got.grad_dtype, got.wd, got.mean_len) == \
+               (ref.numel, ref.block_len, ref.n_blocks, ref.v_offset, ref.kind, ref.grad_dtype, ref.wd, ref.mean_len)
     part.close()
 
 

@@ -92,3 +92,75 @@ def test_two_ranks_equal_the_unsharded_step(tmp_path):
             assert np.array_equal(v, v_all[v0:v0 + v.size])
             seen += p.size
     assert seen == w.numel
+
+
+# ----------------------------------------------------------------------------
+# flat shards that cut blocks: tiling, and the one exchange of partial sums
+# ----------------------------------------------------------------------------
+def odd_model():
+    T = W.TensorSpec
+    tensors = W.llama_like(1, 64, 4, 2, 176, 96, grad_dtype=W.BF16) + [
+        T("odd.rows", 9, 1001, W.ROWS, grad_dtype=W.BF16), T("odd.short", 50, 36, W.ROWS, grad_dtype=W.F32),
+        T("odd.whole", 1, 7777, W.WHOLE, grad_dtype=W.F32)]
+    return W.Workload("odd", 32, tensors, W.GradRecipe(-4.0, -1.0), steps=2)
+
+
+@pytest.mark.parametrize("world", [1, 2, 3, 7, 16])
+def test_flat_pieces_tile_and_parts_stay_inside_one_block(world):
+    for w in (small_model(), odd_model(), W.llama2_7b(n_layers=2), W.flat_sweep(1 << 30)):
+        shards = sharding.shard_flat(w.tensors, world)
+        cursor = {}
+        for r in shards:
+            for p in r:
+                t = w.tensors[p.tensor]
+                assert p.elem_begin == cursor.get(p.tensor, 0) and p.elem_end > p.elem_begin
+                cursor[p.tensor] = p.elem_end
+                assert p.block_len == t.block_len
+                if p.part:
+                    assert p.elem_begin // t.block_len == (p.elem_end - 1) // t.block_len == p.block
+                else:
+                    assert p.elem_begin % t.block_len == 0 and p.elem_end % t.block_len == 0
+                    item = 2 if t.grad_dtype == W.BF16 else 4
+                    assert (p.elem_begin * item) % 16 == 0                     # whole-block runs stay 16-byte aligned
+        assert cursor == {i: t.numel for i, t in enumerate(w.tensors)}
+        loads = [sum(p.numel for p in r) for r in shards]
+        assert max(loads) - min(loads) <= 16
+
+
+def _flat_rank_main(rank, world, port, result_dir):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    w = odd_model()
+    plan = sharding.FlatExchangePlan(w.tensors, world, rank)
+    grads = [ostep.widen(W.gen_grad(w, i, 1)) for i in range(len(w.tensors))]
+    local = torch.zeros(plan.max_parts, dtype=torch.float64)
+    k = 0
+    for p in plan.pieces:
+        if p.part:
+            g = grads[p.tensor][p.elem_begin:p.elem_end]
+            local[k] = float((g * g).sum())
+            k += 1
+    gathered = [torch.zeros_like(local) for _ in range(world)]
+    dist.all_gather(gathered, local)                                    # the step's one exchange
+    totals = plan.combine(torch.stack(gathered))
+    torch.save((plan.part_keys, totals[:plan.n_parts]), os.path.join(result_dir, f"rank{rank}.pt"))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+@pytest.mark.parametrize("world", [2, 3])
+def test_exchange_gives_every_holder_the_whole_block_sum(tmp_path, world):
+    mp.spawn(_flat_rank_main, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True)
+    w = odd_model()
+    grads = [ostep.widen(W.gen_grad(w, i, 1)) for i in range(len(w.tensors))]
+    seen = {}
+    for rank in range(world):
+        keys, totals = torch.load(os.path.join(tmp_path, f"rank{rank}.pt"), weights_only=False)
+        for (tensor, block), tot in zip(keys, totals.tolist()):
+            L = w.tensors[tensor].block_len
+            g = grads[tensor][block * L:(block + 1) * L]
+            want = float((g * g).sum())
+            assert abs(tot - want) <= 1e-12 * want
+            assert seen.setdefault((tensor, block), tot) == tot             # every holder has the same bits
+    assert seen, "no block was cut"
