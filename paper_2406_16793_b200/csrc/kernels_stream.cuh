@@ -882,8 +882,11 @@ inline void stream_finish_plan(const StreamPlanInput &in, int cluster_size, int 
     if (in.chunk == kStaticRanges) plan->main.chunk = 0;
     else if (in.chunk > 0) plan->main.chunk = in.chunk;
     else {
+        // a workload of a couple of items per CTA gains nothing from the counter (and saves its memset)
         const int64_t items = plan->main.bounds.empty() ? 0 : plan->main.bounds.back();
-        plan->main.chunk = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(64, items / (int64_t(32) * std::max(ctas, 1)))));
+        plan->main.chunk = items <= 2 * static_cast<int64_t>(ctas)
+                               ? 0
+                               : static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(64, items / (int64_t(32) * std::max(ctas, 1)))));
     }
     plan->clus = StreamLaunch();
     if (!in.cluster_tensors.empty() && n_clusters > 0) {
