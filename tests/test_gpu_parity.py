@@ -246,7 +246,7 @@ def test_full_size_llama2_7b_sampled_blocks():
     picks = [0, len(w.tensors) - 1, len(w.tensors) - 2]
     for layer in (0, 17, 31):
         picks += list(range(1 + 9 * layer, 1 + 9 * (layer + 1)))
-    worst = H.run_sampled_parity(w, steps=4, tensor_indices=picks, blocks_per_tensor=3)
+    worst = H.run_sampled_parity(w, steps=w.steps, tensor_indices=picks, blocks_per_tensor=3)     # 20 steps
     assert worst["blocks"] >= 60
     H.assert_parity(worst)
 
@@ -287,7 +287,7 @@ def test_full_size_llama3_8b_sampled_blocks():
     picks = [0, len(w.tensors) - 1, len(w.tensors) - 2]
     for layer in (0, 31):
         picks += list(range(1 + 9 * layer, 1 + 9 * (layer + 1)))
-    worst = H.run_sampled_parity(w, steps=3, tensor_indices=picks, blocks_per_tensor=3)
+    worst = H.run_sampled_parity(w, steps=w.steps, tensor_indices=picks, blocks_per_tensor=3)     # 20 steps
     assert worst["blocks"] >= 40
     H.assert_parity(worst)
 
@@ -300,9 +300,9 @@ def test_full_size_flat_sweep_sampled_blocks(L):
     w = W.flat_sweep(L)
     if L < 4096:
         # sample runs of 4096/L consecutive blocks by viewing them as one tensor of short blocks
-        worst = H.run_sampled_runs(w, steps=3, run_elems=4096, n_runs=24)
+        worst = H.run_sampled_runs(w, steps=w.steps, run_elems=4096, n_runs=24)                   # 10 steps
     else:
-        worst = H.run_sampled_parity(w, steps=3, tensor_indices=[0], blocks_per_tensor=6)
+        worst = H.run_sampled_parity(w, steps=w.steps, tensor_indices=[0], blocks_per_tensor=6)
     H.assert_parity(worst)
 
 
