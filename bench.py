@@ -73,8 +73,9 @@ def pick_workload(name: str):
     }
     if name in table:
         return table[name]()
-    if name.startswith("flat-L"):
-        return W.flat_sweep(int(name[6:]))
+    if name.startswith("flat-L"):                      # flat-L<block length>[-n<log2 of the element count>]
+        parts = name[6:].split("-n")
+        return W.flat_sweep(int(parts[0]), numel=1 << (int(parts[1]) if len(parts) > 1 else 30))
     if name.startswith("llama2-7b-layers"):
         return W.llama2_7b(n_layers=int(name[len("llama2-7b-layers"):]))
     raise SystemExit(f"unknown workload {name}")

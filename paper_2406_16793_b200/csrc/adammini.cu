@@ -63,7 +63,8 @@ int build_plan(am_handle *h) {
     const int n = static_cast<int>(h->rows.size());
     h->path.assign(n, PATH_TWOPASS);
     h->host_tensors.assign(n, DevTensor{});
-    std::vector<Seg> small_segs, piece_segs, block_segs, part_segs;
+    std::vector<Seg> small_segs, piece_segs, block_segs, part_segs, wide_segs;
+    int64_t wide_units = 0;
     std::vector<int32_t> part_tensors;
     int64_t part_units = 0;
     int64_t small_units = 0, piece_units = 0, block_units = 0;
@@ -149,13 +150,19 @@ int build_plan(am_handle *h) {
             b.tensor = i;
             b.aux = 0;
             block_segs.push_back(b);
+            if (ppb >= kWideBlockPieces) {          // finalized by a CTA per block
+                Seg ws = b;
+                ws.unit_begin = wide_units;
+                wide_segs.push_back(ws);
+                wide_units += r.n_blocks;
+            }
             piece_units += r.n_blocks * ppb;
             block_units += r.n_blocks;
         } else {
             stream_add_tensor(sin, i, r, path);
         }
     }
-    if (part_units > 0x7fffffffLL) return AM_ERR_TOO_LARGE;
+    if (part_units > 0x7fffffffLL || wide_units > 0x7fffffffLL) return AM_ERR_TOO_LARGE;
     if (small_units > 0x7fffffffLL || piece_units > 0x7fffffffLL || ceil_div(block_units, kThreads / 32) > 0x7fffffffLL)
         return AM_ERR_TOO_LARGE;
 
@@ -173,6 +180,7 @@ int build_plan(am_handle *h) {
     const size_t o_partials = take(sizeof(double) * std::max<int64_t>(piece_units, 1));
     const size_t o_steps = take(sizeof(float) * std::max<int64_t>(block_units, 1));
     const size_t o_stream = take(std::max<size_t>(sp.table_bytes(), 16));
+    const size_t o_wide_segs = take(sizeof(Seg) * std::max<size_t>(wide_segs.size(), 1));
     const size_t o_part_segs = take(sizeof(Seg) * std::max<size_t>(part_segs.size(), 1));
     const size_t o_part_list = take(sizeof(int32_t) * std::max<size_t>(part_tensors.size(), 1));
     h->arena_bytes = off;
@@ -187,6 +195,11 @@ int build_plan(am_handle *h) {
     h->n_small_segs = static_cast<int>(small_segs.size());
     h->n_piece_segs = static_cast<int>(piece_segs.size());
     h->n_block_segs = static_cast<int>(block_segs.size());
+    h->d_wide_segs = reinterpret_cast<Seg *>(base + o_wide_segs);
+    h->n_wide_segs = static_cast<int>(wide_segs.size());
+    h->wide_units = wide_units;
+    if (!wide_segs.empty())
+        AM_CUDA(h, cudaMemcpy(h->d_wide_segs, wide_segs.data(), sizeof(Seg) * wide_segs.size(), cudaMemcpyHostToDevice));
     h->d_part_segs = reinterpret_cast<Seg *>(base + o_part_segs);
     h->d_part_tensors = reinterpret_cast<int32_t *>(base + o_part_list);
     h->n_parts = static_cast<int>(part_tensors.size());
@@ -209,7 +222,7 @@ int build_plan(am_handle *h) {
         if (e != cudaSuccess) return cuda_fail(h, e);
     }
 
-    h->launches = (small_units ? 1 : 0) + (piece_units ? 3 : 0) + sp.launches();
+    h->launches = (small_units ? 1 : 0) + (piece_units ? 3 : 0) + (wide_units ? 1 : 0) + sp.launches();
     h->planned = true;
     return AM_OK;
 }
@@ -463,6 +476,11 @@ int adammini_step_ex(am_handle *h, void *const *params, const void *const *grads
             h->d_tensors, h->d_block_segs, h->n_block_segs, h->block_units, h->d_partials,
             h->d_block_steps, v, sc);
         AM_CUDA(h, cudaGetLastError());
+        if (h->wide_units) {
+            twopass_finalize_wide_kernel<<<static_cast<unsigned>(h->wide_units), kThreads, 0, stream>>>(
+                h->d_tensors, h->d_wide_segs, h->n_wide_segs, h->d_partials, h->d_block_steps, v, sc);
+            AM_CUDA(h, cudaGetLastError());
+        }
         twopass_update_kernel<<<static_cast<unsigned>(h->piece_units), kThreads, 0, stream>>>(
             h->d_tensors, h->d_piece_segs, h->n_piece_segs, h->d_block_steps, sc);
         AM_CUDA(h, cudaGetLastError());

@@ -17,6 +17,7 @@ constexpr int kSmallUnitBlocks = 1024;   // blocks per CTA unit (general L)
 constexpr int kSmallUnitVec = 4096;      // elements per CTA unit (L == 1, float4 path)
 constexpr int64_t kPieceMax = 32768;     // elements per partial sum, two-pass path
 constexpr int64_t kMaxPiecesPerBlock = 16384;
+constexpr int64_t kWideBlockPieces = 256;   // blocks with at least this many partial sums are finalized by a whole CTA
 
 // ---------------------------------------------------------------------------
 // small helpers
@@ -350,6 +351,7 @@ twopass_finalize_kernel(const DevTensor *__restrict__ tensors, const Seg *__rest
     const int lane = threadIdx.x & 31;
     const Seg seg = segs[find_seg(segs, n_segs, unit)];
     const DevTensor &t = tensors[seg.tensor];
+    if (t.pieces_per_block >= kWideBlockPieces) return;      // twopass_finalize_wide_kernel's
     const int64_t b = unit - seg.unit_begin;
     const double *src = partials + t.piece_base + b * t.pieces_per_block;
     const int statistic = sc.statistic;
@@ -385,6 +387,41 @@ part_sums_kernel(const DevTensor *__restrict__ tensors, const int32_t *__restric
     for (int64_t j = lane; j < t.pieces_per_block; j += 32) s += src[j];
     s = warp_sum(s);
     if (lane == 0) out[unit] = s;
+}
+
+// One CTA per block, for blocks with many partial sums (a whole large tensor as
+// one block): every thread adds a strided share, then a fixed-order tree.
+__global__ void __launch_bounds__(kThreads)
+twopass_finalize_wide_kernel(const DevTensor *__restrict__ tensors, const Seg *__restrict__ segs, int n_segs,
+                             const double *__restrict__ partials, float *__restrict__ block_steps,
+                             float *__restrict__ v, StepScalars sc) {
+    __shared__ double warp_part[kThreads / 32];
+    if (step_skipped(sc.skip_flag)) return;
+    const int64_t unit = blockIdx.x;
+    const Seg seg = segs[find_seg(segs, n_segs, unit)];
+    const DevTensor &t = tensors[seg.tensor];
+    const int64_t b = unit - seg.unit_begin;
+    const double *src = partials + t.piece_base + b * t.pieces_per_block;
+    const int statistic = sc.statistic;
+    double s = stat_identity(statistic);
+    for (int64_t j = threadIdx.x; j < t.pieces_per_block; j += kThreads) s = stat_combine(s, src[j], statistic);
+    s = warp_stat(s, statistic);
+    if ((threadIdx.x & 31) == 0) warp_part[threadIdx.x >> 5] = s;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        s = warp_part[0];
+#pragma unroll
+        for (int k = 1; k < kThreads / 32; ++k) s = stat_combine(s, warp_part[k], statistic);
+        if (t.part_index >= 0) {
+            const double gs = static_cast<double>(effective_gscale(sc.gscale, sc.gscale_dev));
+            s = sc.part_sums[t.part_index] * gs * gs;
+        }
+        float vn;
+        const float st = block_step_from_statistic(stat_finish(s, static_cast<double>(t.mean_len), statistic),
+                                                   v[t.v_offset + b], sc, &vn);
+        v[t.v_offset + b] = vn;
+        block_steps[t.block_base + b] = st;
+    }
 }
 
 template <int GD>
