@@ -230,27 +230,28 @@ int adammini_sync_status(am_handle *h, void *cuda_stream);
 
 /* Options and queries (keys below).  Unknown keys: AM_ERR_INVALID_ARGUMENT. */
 typedef enum {
-    AM_OPT_PATH          = 0, /* 0 = automatic; 1 = force the three-launch two-pass path for every
-                                 tensor with block_len > 16 (correctness anchor) */
-    AM_OPT_STREAM_CTAS   = 1, /* persistent CTAs of the streaming kernel (0 = one per SM) */
-    AM_OPT_CLUSTER_SIZE  = 2, /* CTAs per cluster for head-sized blocks (0 = default) */
-    AM_OPT_STREAM_THREADS = 3, /* threads per consumer group of the streaming kernels (0 = default 256) */
-    AM_OPT_PROFILE       = 4, /* n > 0: record CUDA events around each kernel family of every step, keeping
-                                 the latest n steps (n <= 4096); read them with adammini_get_profile.
-                                 Setting the option again restarts the record */
-    AM_OPT_STREAM_CHUNK  = 5  /* how the streaming kernel's CTAs share the work: 0 = automatic (CTAs take
-                                 up to 64 work items at a time from a shared counter, which evens out
-                                 bandwidth differences between SMs); 1..4096 = that many items at a
-                                 time; 1000000 = every CTA walks its own fixed, cost-balanced range.
-                                 Results are bit-identical in every mode */
-    , AM_OPT_CLUSTER_CHUNK = 6 /* the same for the cluster kernel, in blocks handed to a cluster at a time */
-    , AM_OPT_STATISTIC = 7     /* block statistic that feeds v: 0 = mean(g*g), Algorithm 1.  The ablation
+    AM_OPT_PATH           = 0, /* 0 = automatic; 1 = force the two-pass path for every tensor with
+                                  block_len > 16 (correctness anchor) */
+    AM_OPT_STREAM_CTAS    = 1, /* persistent CTAs of the streaming kernel (0 = one per SM) */
+    AM_OPT_CLUSTER_SIZE   = 2, /* CTAs per cluster for head-sized blocks: 1, 2, 4, 8 (0 = chosen by block size) */
+    AM_OPT_STREAM_THREADS = 3, /* threads per consumer group of the streaming kernels, a multiple of 32
+                                  from 64 to 512 (0 = default 256); groups x threads is capped at 512 */
+    AM_OPT_PROFILE        = 4, /* n > 0: record CUDA events around each kernel family of every step, keeping
+                                  the latest n steps (n <= 4096); read them with adammini_get_profile.
+                                  Setting the option again restarts the record */
+    AM_OPT_STREAM_CHUNK   = 5, /* how the streaming kernel's CTAs share the work: 0 = automatic (CTAs take
+                                  up to 64 work items at a time from a shared counter, which evens out
+                                  bandwidth differences between SMs; fixed ranges for tiny workloads);
+                                  1..4096 = that many items at a time; 1000000 = every CTA walks its own
+                                  fixed, cost-balanced range.  Results are bit-identical in every mode */
+    AM_OPT_CLUSTER_CHUNK  = 6, /* the same for the cluster kernel, in blocks handed to a cluster at a time */
+    AM_OPT_STATISTIC      = 7, /* block statistic that feeds v: 0 = mean(g*g), Algorithm 1.  The ablation
                                   of the paper's appendix ("Ablation Studies on the Design of Adam-mini"),
                                   which it reports to train worse: 1 = max, 2 = min, 3 = 1-norm (sum),
                                   4 = 2-norm of the vector g*g.  Non-zero values run on the two-pass
                                   kernels (g read twice) */
-    , AM_OPT_STREAM_GROUPS = 8 /* consumer groups per CTA of the streaming kernels (0 = default 2, or 1);
-                                  groups x threads is capped at 512 */
+    AM_OPT_STREAM_GROUPS  = 8  /* consumer groups per CTA of the streaming kernel, which own alternate
+                                  work items: 1 or 2 (0 = default: 2; the cluster kernel runs one) */
 } am_option;
 int adammini_set_option(am_handle *h, int32_t key, int64_t value);
 
