@@ -321,12 +321,16 @@ def run_e2e(args, opt, w, world, dev, p, g, m, v):
     for line in open("/proc/meminfo"):
         if line.startswith("MemAvailable"):
             avail = int(line.split()[1]) * 1024
-    if avail < 2.2 * need * max(1, min(world, torch.cuda.device_count())):
+    if avail < 1.5 * need * max(1, min(world, torch.cuda.device_count())):
         return {"value": None, "unit": UNIT, "skipped": f"host memory: need {need} B pinned per rank, {avail} B available"}
-    hp = [x.to("cpu", non_blocking=False).pin_memory() for x in p]
-    hm = [x.to("cpu").pin_memory() for x in m]
-    hg = [x.to("cpu").pin_memory() for x in g]
-    hv = v.to("cpu").pin_memory()
+    def pinned_copy(x):                     # straight into pinned memory: no pageable intermediate
+        out = torch.empty(x.shape, dtype=x.dtype, pin_memory=True)
+        out.copy_(x)
+        return out
+    hp = [pinned_copy(x) for x in p]
+    hm = [pinned_copy(x) for x in m]
+    hg = [pinned_copy(x) for x in g]
+    hv = pinned_copy(v)
     h2d = sum(x.numel() * x.element_size() for x in hp + hm + hg) + hv.numel() * 4
     d2h = sum(x.numel() * x.element_size() for x in hp + hm) + hv.numel() * 4
     steps = max(1, min(args.e2e_steps, args.steps))
