@@ -153,6 +153,19 @@ __device__ __forceinline__ void bulk_load(void *dst_smem, const void *src_gmem, 
         "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
         ::"r"(smem_addr(dst_smem)), "l"(src_gmem), "r"(bytes), "r"(smem_addr(bar)) : "memory");
 }
+// The same with an L2 eviction-priority hint (a policy from createpolicy).
+__device__ __forceinline__ void bulk_load_hint(void *dst_smem, const void *src_gmem, uint32_t bytes, void *bar,
+                                               unsigned long long policy) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+        ::"r"(smem_addr(dst_smem)), "l"(src_gmem), "r"(bytes), "r"(smem_addr(bar)), "l"(policy) : "memory");
+}
+__device__ __forceinline__ unsigned long long l2_policy_evict_last() {
+    unsigned long long p; asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p)); return p;
+}
+__device__ __forceinline__ unsigned long long l2_policy_evict_first() {
+    unsigned long long p; asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p)); return p;
+}
 __device__ __forceinline__ uint32_t cluster_ctarank() {
     uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r;
 }
@@ -355,6 +368,7 @@ stream_kernel(const __grid_constant__ StreamParams P) {
             uint32_t phase = 0;
             int64_t armed = 0;              // stages armed so far
             int32_t item_group = 0;         // consumer group of the current item (items alternate)
+            const unsigned long long keep_in_l2 = l2_policy_evict_last(), drop_from_l2 = l2_policy_evict_first();
             bool ok = true;
             int seg = 0;
             if (P.chunk <= 0) {
@@ -477,7 +491,9 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                         if (vbytes)
                             bulk_load(v_areas + stage * kVAreaFloats, P.v + ((t.v_offset + local) & ~int64_t(3)), vbytes,
                                       &ctl->full[stage]);
-                        bulk_load(st, gbase + (e0 + off) * gsz, c * gsz, &ctl->full[stage]);
+                        // a head's gradients are fetched twice: keep the first copy in L2 ...
+                        if (CLUSTER) bulk_load_hint(st, gbase + (e0 + off) * gsz, c * gsz, &ctl->full[stage], keep_in_l2);
+                        else bulk_load(st, gbase + (e0 + off) * gsz, c * gsz, &ctl->full[stage]);
                         advance();
                     }
                     for (int64_t off = 0; off < slice && ok; off += kStageElems) {
@@ -490,7 +506,9 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                         mt.n = c; mt.L = 0; mt.kind = STAGE_APPLY; mt.flags = base_flags;
                         unsigned char *st = stages + static_cast<size_t>(stage) * P.stage_bytes;
                         mbar_arrive_expect_tx(&ctl->full[stage], static_cast<uint32_t>(c) * (gsz + 8));
-                        bulk_load(st, gbase + (e0 + off) * gsz, c * gsz, &ctl->full[stage]);
+                        // ... and let go of it at the second fetch (measured: head kernel 3.00 ms against 3.10 ms)
+                        if (CLUSTER) bulk_load_hint(st, gbase + (e0 + off) * gsz, c * gsz, &ctl->full[stage], drop_from_l2);
+                        else bulk_load(st, gbase + (e0 + off) * gsz, c * gsz, &ctl->full[stage]);
                         bulk_load(st + P.g_region_bytes, t.m + e0 + off, c * 4, &ctl->full[stage]);
                         bulk_load(st + P.g_region_bytes + kStageElems * 4, t.p + e0 + off, c * 4, &ctl->full[stage]);
                         advance();
