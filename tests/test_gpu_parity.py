@@ -478,3 +478,31 @@ def ostep_state(w, dev):
     from oracle import step as ostep
     return ostep.OracleState([p.cpu() for p in dev.p], [t.block_len for t in w.tensors],
                              [bool(t.apply_weight_decay) for t in w.tensors])
+
+
+def test_many_small_tensors_of_mixed_kinds():
+    """Hundreds of small tensors of seeded random shapes, kinds and gradient
+    dtypes in one table: segment walking, ragged last stages, the end of v."""
+    rng = np.random.default_rng(20240616)
+    cols_choices = [1, 3, 8, 24, 40, 128, 768, 1000, 1001, 3072, 4096, 5000, 11008]
+    tensors = []
+    for i in range(400):
+        cols = int(rng.choice(cols_choices))
+        rows = int(rng.integers(1, 40))
+        gd = int(rng.integers(0, 2))
+        kind = int(rng.choice([W.WHOLE, W.ROWS, W.TOKENS, W.HEADS, W.FIXED]))
+        kw = {}
+        if kind == W.HEADS:
+            divs = [d for d in range(1, rows + 1) if rows % d == 0]
+            kw["n_heads"] = int(rng.choice(divs))
+        if kind == W.FIXED:
+            n = rows * cols
+            divs = [d for d in (1, 2, 4, 8, 16, cols, n) if n % d == 0]
+            kw["fixed_block_len"] = int(rng.choice(divs))
+        if kind == W.WHOLE:
+            rows, cols = 1, rows * cols
+        tensors.append(W.TensorSpec(f"t{i}", rows, cols, kind, grad_dtype=gd,
+                                    apply_weight_decay=int(rng.integers(0, 2)), **kw))
+    w = W.Workload("many-small", 63, tensors, W.GradRecipe(-4.0, -1.0), steps=3)
+    H.assert_parity(H.run_parity(w))
+    H.assert_parity(H.run_parity(w, steps=2, options={B.OPT_STREAM_CHUNK: 3}))
