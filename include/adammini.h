@@ -181,7 +181,9 @@ int adammini_part_sums(am_handle *h, const void *const *grads, double *out, void
  * buffers (host->device copies, the kernels above, device->host copies) on
  * internal streams and returns after everything has landed back in host
  * memory.  Pinned host memory gives full copy bandwidth; pageable works.
- * `staging_bytes` bounds the device memory used for staging (0 = default). */
+ * `staging_bytes` bounds the device memory used for staging (0 = default: 3 GiB, or three times
+ * the largest tensor's p + m + g if that is more).  Tables with AM_PART tensors are not supported
+ * here (AM_ERR_INVALID_ARGUMENT): their step needs the exchange of part sums in between. */
 int adammini_step_host(am_handle *h, void *const *params, const void *const *grads, void *const *m,
                        float *v, int64_t step, int64_t staging_bytes);
 

@@ -115,6 +115,7 @@ extern "C" int adammini_step_host(am_handle *h, void *const *params, const void 
     if (!h || !h->planned || step < 1 || staging_bytes < 0) return AM_ERR_INVALID_ARGUMENT;
     const int n = static_cast<int>(h->rows.size());
     if (n == 0) return AM_OK;
+    if (h->n_parts > 0) return AM_ERR_INVALID_ARGUMENT;     // parts of blocks need the exchange of their sums
     if (!params || !grads || !m || !v) return AM_ERR_INVALID_ARGUMENT;
     for (int i = 0; i < n; ++i)
         if (!params[i] || !grads[i] || !m[i]) return AM_ERR_INVALID_ARGUMENT;
