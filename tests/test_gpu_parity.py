@@ -113,7 +113,7 @@ def test_other_cluster_sizes(cluster):
 
 def test_zero_gradient_rows_and_an_infinity():
     """Rows with all-zero gradients keep v = 0 and take no Adam step; an
-    infinite gradient propagates exactly as in the oracle."""
+    infinite and a NaN gradient propagate exactly as in the oracle (no skip, no clip)."""
     w = W.scaled_rows(W.llama2_7b(n_layers=1, vocab=512), 64)
 
     def mutate(step, grads):
@@ -121,6 +121,8 @@ def test_zero_gradient_rows_and_an_infinity():
         grads[4].view(-1, 4096)[5].zero_()
         if step == 2:
             grads[5].view(-1)[12345] = float("inf")
+        if step == 3:
+            grads[7].view(-1)[4096 * 3 + 17] = float("nan")      # poisons exactly one block (row 3)
 
     H.assert_parity(H.run_parity(w, steps=4, mutate_grads=mutate))
 
