@@ -74,10 +74,16 @@ struct StageMeta {          // written by the producer, read by the consumers
 };
 static_assert(sizeof(StageMeta) == 64, "stage descriptor is 64 bytes");
 
-struct StreamSeg {          // a run of items of one tensor
-    int64_t item_begin;
+// A run of work items of one tensor.  Items are addressed in "slots": an item
+// takes as many consecutive slots as it has stages, so that a range of slots is
+// about the same amount of work whatever kind of item it holds; the item whose
+// first slot lies in a CTA's range belongs to that CTA.
+struct StreamSeg {
+    int64_t item_begin;     // first slot of the segment
     int32_t tensor;
     int32_t bpi;            // blocks per item (PACKED); 0: one long block per item
+    int32_t slots;          // slots per item (1 for PACKED items and for cluster launches)
+    int32_t pad;
 };
 
 struct StreamParams {
@@ -446,7 +452,15 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                 while (seg + 1 < P.n_segs && P.segs[seg + 1].item_begin <= it) ++seg;
                 const StreamSeg sg = P.segs[seg];
                 const DevTensor &t = P.tensors[sg.tensor];
-                const int64_t local = it - sg.item_begin;
+                int64_t local = it - sg.item_begin;
+                if (sg.slots > 1) {
+                    const int64_t rem = local % sg.slots;
+                    if (rem != 0) {             // inside an item that began in somebody else's range
+                        it += sg.slots - rem - 1;
+                        continue;
+                    }
+                    local /= sg.slots;
+                }
                 const int gsz = t.gdtype == AM_BF16 ? 2 : 4;
                 const int base_flags = (t.gdtype == AM_BF16 ? SF_BF16 : 0) | (t.wd ? SF_WD : 0);
                 const unsigned char *gbase = static_cast<const unsigned char *>(t.g);
@@ -515,6 +529,7 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                     }
                 }
                 if (++item_group == P.n_groups) item_group = 0;
+                it += sg.slots - 1;             // the loop's increment then lands on the next item
             }
             if (ok && acquire()) {
                 ctl->meta[stage].kind = STAGE_DONE;
@@ -810,50 +825,64 @@ inline void stream_build_launch(const std::vector<StreamPlanInput::Item> &tensor
     out->n_stages = std::min<int>(kMaxStages, static_cast<int>((kSmemBudget - kCtrlBytes) / (out->stage_bytes + kVAreaFloats * 4)));
 
     std::vector<double> item_cost;      // per segment
-    int64_t items = 0;
+    int64_t slots = 0, n_items = 0;
     for (const auto &it : tensors) {
         const am_table_row &r = it.row;
-        const double gsz = r.grad_dtype == AM_BF16 ? 2 : 4;
+        const int gsz = r.grad_dtype == AM_BF16 ? 2 : 4;
         StreamSeg s;
-        s.item_begin = items;
+        s.item_begin = slots;
         s.tensor = it.tensor;
+        s.pad = 0;
+        int64_t seg_items;
         if (!cluster && r.block_len <= kStageElems) {
             s.bpi = static_cast<int32_t>(kStageElems / r.block_len);
-            items += (r.n_blocks + s.bpi - 1) / s.bpi;
+            s.slots = 1;
+            seg_items = (r.n_blocks + s.bpi - 1) / s.bpi;
             item_cost.push_back(static_cast<double>(s.bpi) * r.block_len * (gsz + 16));
         } else {
             s.bpi = 0;
-            items += r.n_blocks;
+            const int64_t sum_cap = out->stage_bytes / gsz;
+            s.slots = cluster ? 1 : static_cast<int32_t>((r.block_len + sum_cap - 1) / sum_cap +
+                                                         (r.block_len + kStageElems - 1) / kStageElems);
+            seg_items = r.n_blocks;
             item_cost.push_back(static_cast<double>(r.block_len) * (2 * gsz + 16));
         }
+        slots += seg_items * s.slots;
+        n_items += seg_items;
         out->segs.push_back(s);
     }
     StreamSeg sentinel;
-    sentinel.item_begin = items;
+    sentinel.item_begin = slots;
     sentinel.tensor = -1;
     sentinel.bpi = 0;
+    sentinel.slots = 1;
+    sentinel.pad = 0;
     out->segs.push_back(sentinel);
 
-    // contiguous item ranges of (nearly) equal cost
+    // contiguous ranges of (nearly) equal cost, cut at item starts
     double total = 0.0;
-    for (size_t k = 0; k + 1 < out->segs.size(); ++k)
-        total += item_cost[k] * static_cast<double>(out->segs[k + 1].item_begin - out->segs[k].item_begin);
-    workers = static_cast<int>(std::min<int64_t>(workers, items));
+    auto seg_items_of = [&](size_t k) {
+        return (out->segs[k + 1].item_begin - out->segs[k].item_begin) / out->segs[k].slots;
+    };
+    for (size_t k = 0; k + 1 < out->segs.size(); ++k) total += item_cost[k] * static_cast<double>(seg_items_of(k));
+    workers = static_cast<int>(std::min<int64_t>(workers, n_items));
     out->bounds.assign(workers + 1, 0);
-    out->bounds[workers] = items;
+    out->bounds[workers] = slots;
     size_t k = 0;
     double before = 0.0;                // cost of the segments before k
     for (int w = 1; w < workers; ++w) {
         const double target = total * w / workers;
         for (;;) {
-            const double seg_cost = item_cost[k] * static_cast<double>(out->segs[k + 1].item_begin - out->segs[k].item_begin);
+            const double seg_cost = item_cost[k] * static_cast<double>(seg_items_of(k));
             if (before + seg_cost >= target || k + 2 >= out->segs.size()) break;
             before += seg_cost;
             ++k;
         }
-        int64_t idx = out->segs[k].item_begin + static_cast<int64_t>((target - before) / item_cost[k] + 0.5);
+        int64_t item = static_cast<int64_t>((target - before) / item_cost[k] + 0.5);
+        item = std::min(item, seg_items_of(k));
+        int64_t idx = out->segs[k].item_begin + item * out->segs[k].slots;
         idx = std::max(idx, out->bounds[w - 1]);
-        idx = std::min(idx, items);
+        idx = std::min(idx, slots);
         out->bounds[w] = idx;
     }
     out->grid = workers;
@@ -908,7 +937,7 @@ inline void stream_finish_plan(const StreamPlanInput &in, int cluster_size, int 
     else if (in.chunk > 0) plan->main.chunk = in.chunk;
     else {
         // a workload of a couple of items per CTA gains nothing from the counter (and saves its memset)
-        const int64_t items = plan->main.bounds.empty() ? 0 : plan->main.bounds.back();
+        const int64_t items = plan->main.bounds.empty() ? 0 : plan->main.bounds.back();     // in slots
         plan->main.chunk = items <= 2 * static_cast<int64_t>(ctas)
                                ? 0
                                : static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(64, items / (int64_t(32) * std::max(ctas, 1)))));
