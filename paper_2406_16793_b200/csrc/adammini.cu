@@ -353,6 +353,7 @@ int adammini_set_option(am_handle *h, int32_t key, int64_t value) {
         h->opt[key] = old;
         build_plan(h);
     }
+    host_step_release(h);                   // its per-group handles were planned with the old options
     return rc;
 }
 

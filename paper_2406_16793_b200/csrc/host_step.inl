@@ -31,6 +31,7 @@ inline size_t tensor_staging_bytes(const am_table_row &r) {
 
 struct HostStepState {
     size_t slot_bytes = 0;
+    bool ready = false;          // every group has its handle
     void *slots[kHostSlots] = {nullptr, nullptr, nullptr};
     cudaStream_t streams[kHostSlots] = {nullptr, nullptr, nullptr};
     std::vector<HostGroup> groups;
@@ -57,7 +58,7 @@ int host_step_prepare(am_handle *h, int64_t staging_bytes) {
     for (const am_table_row &r : h->rows) largest = std::max(largest, tensor_staging_bytes(r));
     const size_t budget = staging_bytes > 0 ? static_cast<size_t>(staging_bytes) : kHostDefaultStaging;
     const size_t slot_bytes = std::max(budget / kHostSlots, largest);
-    if (h->host_step && h->host_step->slot_bytes == slot_bytes) return AM_OK;
+    if (h->host_step && h->host_step->ready && h->host_step->slot_bytes == slot_bytes) return AM_OK;
     host_step_release(h);
 
     HostStepState *s = new (std::nothrow) HostStepState();

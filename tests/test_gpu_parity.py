@@ -229,6 +229,8 @@ def test_host_buffer_step_matches_device_step(staging):
         hg = [x.cpu() for x in dev.g]                       # pageable on purpose
         opt.step(dev.p, dev.g, dev.m, dev.v, t)
         opt.step_host(hp, hg, hm, hv, t, staging_bytes=staging)
+        if t == 2:                                          # the staged handles follow an option change
+            opt.set_option(B.OPT_STREAM_CHUNK, 3)
     opt.sync_status()
     for a, b in zip(dev.p + dev.m + [dev.v], hp + hm + [hv]):
         assert torch.equal(a.cpu(), b)
