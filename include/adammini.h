@@ -181,6 +181,8 @@ int adammini_part_sums(am_handle *h, const void *const *grads, double *out, void
  * buffers (host->device copies, the kernels above, device->host copies) on
  * internal streams and returns after everything has landed back in host
  * memory.  Pinned host memory gives full copy bandwidth; pageable works.
+ * Every group runs with the launch shape this handle resolved, so the result
+ * equals adammini_step's on the same handle bit for bit.
  * `staging_bytes` bounds the device memory used for staging (0 = default: 3 GiB, or three times
  * the largest tensor's p + m + g if that is more).  Tables with AM_PART tensors are not supported
  * here (AM_ERR_INVALID_ARGUMENT): their step needs the exchange of part sums in between. */

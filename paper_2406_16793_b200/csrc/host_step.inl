@@ -105,7 +105,15 @@ int host_step_prepare(am_handle *h, int64_t staging_bytes) {
         if (rc != AM_OK) return rc;
         for (int key = 0; key < kNumOptions; ++key)
             if (key != AM_OPT_PROFILE && h->opt[key]) adammini_set_option(g.sub, key, h->opt[key]);
+        // The order in which a long block's partial sums are added depends on the cluster size, and
+        // the automatic choice looks at all tensors of a table: give the group the size this handle
+        // resolved, so that the staged step returns the bits adammini_step returns.
+        if (h->stream.clus.active() && h->opt[AM_OPT_CLUSTER_SIZE] == 0) {
+            const int rc2 = adammini_set_option(g.sub, AM_OPT_CLUSTER_SIZE, h->stream.clus.cluster);
+            if (rc2 != AM_OK) return rc2;
+        }
     }
+    s->ready = true;
     return AM_OK;
 }
 

@@ -22,7 +22,9 @@
 //
 // A block is always reduced in one fixed order (per thread, per warp, per
 // group, per cluster rank), whichever CTA or group gets it, so results do not
-// depend on the launch shape or on how the work was handed out.
+// depend on the number of CTAs or groups or on how the work was handed out; the
+// threads per group and the cluster size fix that order and so can change the
+// last bit of a sum.
 //
 // Every wait is bounded: a wait that gives up sets the abort flag and the
 // handle's error word, and all roles leave through the common exit.

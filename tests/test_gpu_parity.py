@@ -214,11 +214,7 @@ def test_empty_partition_and_queries():
     opt.close()
 
 
-@pytest.mark.parametrize("staging", [0, 3 * (24 << 20)], ids=["default-staging", "many-groups"])
-def test_host_buffer_step_matches_device_step(staging):
-    """adammini_step_host (state in host memory, streamed through staging slots)
-    gives the same bits as adammini_step on device-resident state."""
-    w = W.scaled_rows(W.llama2_7b(n_layers=1, vocab=512), 128)
+def _host_step_equals_device_step(w, staging):
     dev = H.DeviceState(w, guarded=False)
     opt = H.make_optimizer(w)
     hp = [x.cpu().pin_memory() for x in dev.p]
@@ -235,6 +231,26 @@ def test_host_buffer_step_matches_device_step(staging):
     for a, b in zip(dev.p + dev.m + [dev.v], hp + hm + [hv]):
         assert torch.equal(a.cpu(), b)
     opt.close()
+
+
+@pytest.mark.parametrize("staging", [0, 3 * (24 << 20)], ids=["default-staging", "many-groups"])
+def test_host_buffer_step_matches_device_step(staging):
+    """adammini_step_host (state in host memory, streamed through staging slots)
+    gives the same bits as adammini_step on device-resident state."""
+    _host_step_equals_device_step(W.scaled_rows(W.llama2_7b(n_layers=1, vocab=512), 128), staging)
+
+
+def test_host_buffer_step_keeps_the_cluster_size_of_the_whole_table():
+    """Heads of 0.35 MB and of 1.3 MB land in different staging groups; on its own
+    the first would run on smaller clusters than the table as a whole does, and its
+    sums would round differently."""
+    T = W.TensorSpec
+    bf = dict(grad_dtype=W.BF16)
+    tensors = [T("rows", 300, 768, W.ROWS, **bf), T("head_a", 4, 179456, W.ROWS, **bf),
+               T("whole", 1, 2319092, W.WHOLE, **bf), T("head_b", 4, 640128, W.ROWS, **bf),
+               T("tail", 150, 1424, W.ROWS, **bf)]
+    w = W.Workload("two-head-sizes", 77, tensors, W.GradRecipe(-4.0, -1.0), steps=3)
+    _host_step_equals_device_step(w, 3 * (40 << 20))
 
 
 def test_full_size_llama2_7b_sampled_blocks():
@@ -510,3 +526,60 @@ def test_many_small_tensors_of_mixed_kinds():
     w = W.Workload("many-small", 63, tensors, W.GradRecipe(-4.0, -1.0), steps=3)
     H.assert_parity(H.run_parity(w))
     H.assert_parity(H.run_parity(w, steps=2, options={B.OPT_STREAM_CHUNK: 3}))
+
+
+def _random_table(rng):
+    """A seeded random table that mixes every path: thread-per-block, packed rows,
+    block lengths that are not a multiple of 16 bytes, long single-CTA rows,
+    cluster-sized blocks, whole tensors beyond the cluster limit, heads."""
+    T = W.TensorSpec
+    tensors, budget = [], 12_000_000
+    for i in range(int(rng.integers(2, 14))):
+        gd = int(rng.integers(0, 2))
+        gsz = 2 if gd == W.BF16 else 4
+        kw = dict(grad_dtype=gd, apply_weight_decay=int(rng.integers(0, 2)))
+        cls = rng.choice(["small", "packed", "odd", "long", "cluster", "whole", "heads"])
+        if cls == "small":
+            t = T(f"t{i}", int(rng.integers(1, 3000)), int(rng.integers(1, 17)), W.ROWS, **kw)
+        elif cls == "packed":
+            L = int(rng.integers(3, 513)) * 8
+            t = T(f"t{i}", int(rng.integers(1, max(2, 400000 // L))), L, W.ROWS, **kw)
+        elif cls == "odd":
+            L = int(rng.integers(17, 9000))
+            t = T(f"t{i}", int(rng.integers(1, max(2, 200000 // L))), L, W.ROWS, **kw)
+        elif cls == "long":
+            L = int(rng.integers(513, (256 * 1024 // gsz) // 8 + 1)) * 8
+            t = T(f"t{i}", int(rng.integers(1, 9)), L, W.ROWS, **kw)
+        elif cls == "cluster":
+            lo = (256 * 1024 // gsz) // 64 + 1
+            L = int(rng.integers(lo, lo + 8001)) * 64
+            t = T(f"t{i}", int(rng.integers(1, 5)), L, W.ROWS, **kw)
+        elif cls == "heads":
+            nh, rph, cols = int(rng.integers(1, 9)), int(rng.integers(1, 65)), int(rng.integers(1, 65)) * 8
+            t = T(f"t{i}", nh * rph, cols, W.HEADS, n_heads=nh, **kw)
+        else:
+            t = T(f"t{i}", 1, int(rng.integers(1, 3_000_000)), W.WHOLE, **kw)
+        if t.numel <= budget:
+            budget -= t.numel
+            tensors.append(t)
+    return tensors or [T("t", 4, 64, W.ROWS)]
+
+
+def _random_options(rng):
+    o = {}
+    for key, values in ((B.OPT_STREAM_THREADS, [128, 256, 512]), (B.OPT_STREAM_GROUPS, [1, 2]),
+                        (B.OPT_CLUSTER_SIZE, [1, 2, 4, 8]), (B.OPT_STREAM_CHUNK, [1, 2, 5, 64, 1000000]),
+                        (B.OPT_CLUSTER_CHUNK, [1, 2, 3, 1000000]), (B.OPT_STREAM_CTAS, [1, 3, 7, 37, 148])):
+        if rng.random() < 0.5:
+            o[key] = int(rng.choice(values))
+    return o
+
+
+def test_random_tables_and_launch_options():
+    """Forty seeded random tables, each under random launch options, two steps."""
+    for seed in range(40):
+        rng = np.random.default_rng(7000 + seed)
+        w = W.Workload(f"random{seed}", 800 + seed, _random_table(rng), W.GradRecipe(-4.0, -1.0), steps=2)
+        options = _random_options(rng)
+        worst = H.run_parity(w, options=options)
+        assert max(worst.values()) <= H.TOL, (seed, options, worst)
