@@ -89,3 +89,27 @@ def test_status_strings():
     seen = {lib.adammini_status_string(s).decode() for s in range(-7, 1)}
     assert len(seen) == 8 and "unknown status" not in seen
     assert lib.adammini_status_string(-99).decode() == "unknown status"
+
+
+def test_missing_library_fails_loudly(tmp_path):
+    """Without the shared object the binding raises at once: there is no other path."""
+    import subprocess
+    import sys
+    code = ("import paper_2406_16793_b200 as am\n"
+            "from paper_2406_16793_b200 import workloads as W\n"
+            "try:\n"
+            "    am.Partition(W.tiny_gpt2().tensors)\n"
+            "except RuntimeError as e:\n"
+            "    assert 'missing' in str(e) and 'no CPU fallback' in str(e), e\n"
+            "    print('raised')\n")
+    env = dict(os.environ, ADAMMINI_LIBRARY=str(tmp_path / "libadammini.so"), PYTHONPATH=ROOT)
+    out = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, timeout=120)
+    assert out.returncode == 0 and out.stdout.strip() == "raised", out.stderr
+
+
+@pytest.mark.skipif(__import__("torch").cuda.is_available(), reason="checks the behaviour without a device")
+def test_creating_a_handle_without_a_device_reports_a_cuda_error():
+    part = am.Partition(W.tiny_gpt2().tensors)
+    with pytest.raises(am.AdamMiniError) as e:
+        am.AdamMini(part, lr=1e-3, beta1=0.9, beta2=0.95, eps=1e-8, weight_decay=0.1)
+    assert e.value.status == -4
