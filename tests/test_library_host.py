@@ -113,3 +113,53 @@ def test_creating_a_handle_without_a_device_reports_a_cuda_error():
     with pytest.raises(am.AdamMiniError) as e:
         am.AdamMini(part, lr=1e-3, beta1=0.9, beta2=0.95, eps=1e-8, weight_decay=0.1)
     assert e.value.status == -4
+
+
+def test_random_descriptors_agree_with_the_reference_partitioner():
+    """2000 seeded random descriptors, valid and invalid: the library accepts
+    exactly what the Python rules accept and exports the same row."""
+    import numpy as np
+    rng = np.random.default_rng(424242)
+    accepted = rejected = 0
+    batch = []
+    for _ in range(2000):
+        kind = int(rng.choice([W.WHOLE, W.ROWS, W.HEADS, W.TOKENS, W.FIXED, W.PART]))
+        rows = int(rng.choice([0, 1, 1, 2, 3, 7, 12, 64, 300]))
+        cols = int(rng.choice([0, 1, 5, 8, 24, 768, 4096, 100003]))
+        n_heads = int(rng.choice([0, 1, 2, 3, 4, 12]))
+        fixed = int(rng.choice([0, 1, 2, 4, 5, 8, 24, 4096, 1 << 20, 1 << 33]))
+        d = pr.TensorDesc(rows, cols, kind, n_heads, fixed, int(rng.integers(0, 2)), int(rng.integers(0, 2)))
+        try:
+            want, _ = pr.build_table([d])
+        except ValueError:
+            want = None
+        spec = W.TensorSpec("t", rows, cols, kind, n_heads=n_heads, fixed_block_len=fixed,
+                            grad_dtype=d.grad_dtype, apply_weight_decay=d.apply_weight_decay)
+        if want is None:
+            with pytest.raises(am.AdamMiniError) as e:
+                am.Partition([spec])
+            assert e.value.status == -2, d
+            rejected += 1
+            continue
+        batch.append((spec, d))
+        accepted += 1
+    assert accepted > 300 and rejected > 300
+    # all accepted descriptors as one table: offsets accumulate the same way
+    part = am.Partition([s for s, _ in batch])
+    rows_got, total = part.export()
+    want, want_total = pr.build_table([d for _, d in batch])
+    assert total == want_total
+    for got, ref in zip(rows_got, want):
+        assert (got.numel, got.block_len, got.n_blocks, got.v_offset, got.kind, got.grad_dtype, got.wd, got.mean_len) == \
+               (ref.numel, ref.block_len, ref.n_blocks, ref.v_offset, ref.kind, ref.grad_dtype, ref.wd, ref.mean_len)
+    part.close()
+
+
+def test_random_names_agree_with_the_reference_name_rule():
+    import numpy as np
+    rng = np.random.default_rng(7)
+    words = ["embed", "output", "query", "key", "value", "attn.proj", "mlp", "attn", "proj", "norm", "weight", "bias",
+             "layers", "wq", "lm_head", "tok", "fc", "0", "11", "."]
+    for _ in range(500):
+        name = "".join(rng.choice(words, size=int(rng.integers(1, 6))))
+        assert binding.kind_from_name(name) == pr.kind_from_name(name), name
