@@ -97,7 +97,9 @@ typedef struct am_handle am_handle;
 /* ---- partitioner (host only; Algorithm 2 / Algorithm 3) ------------------------
  * Builds the flat block table from `n_tensors` descriptors (host array, read
  * during the call only).  On success *out owns the table; free it with
- * adammini_partition_free.  AM_ERR_SHAPE if a descriptor does not divide. */
+ * adammini_partition_free.  AM_ERR_SHAPE if a descriptor does not divide (or its
+ * rows * cols overflows int64), AM_ERR_TOO_LARGE if the element count of the whole
+ * table does, AM_ERR_INVALID_ARGUMENT for an unknown kind or dtype. */
 int adammini_partition_build(const am_tensor_desc *descs, int32_t n_tensors, am_partition **out);
 
 /* Number of tensors in the table. */

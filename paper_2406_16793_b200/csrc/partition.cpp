@@ -50,7 +50,7 @@ int adammini_partition_build(const am_tensor_desc *descs, int32_t n_tensors, am_
     if (!part) return AM_ERR_ALLOC;
     try {
         part->rows.reserve(n_tensors);
-        int64_t v_offset = 0;
+        int64_t v_offset = 0, total_elems = 0;
         for (int32_t i = 0; i < n_tensors; ++i) {
             const am_tensor_desc &d = descs[i];
             if (d.rows <= 0 || d.cols <= 0 || d.rows > std::numeric_limits<int64_t>::max() / d.cols) {
@@ -67,6 +67,11 @@ int adammini_partition_build(const am_tensor_desc *descs, int32_t n_tensors, am_
                 delete part;
                 return AM_ERR_SHAPE;
             }
+            if (numel > std::numeric_limits<int64_t>::max() - total_elems) {     // the table's totals stay in int64
+                delete part;
+                return AM_ERR_TOO_LARGE;
+            }
+            total_elems += numel;               // bounds the block count too: n_blocks <= numel
             am_table_row r;
             r.numel = numel;
             r.block_len = L;

@@ -82,6 +82,13 @@ def test_partition_rejects_bad_descriptors():
     with pytest.raises(am.AdamMiniError) as e:
         am.Partition([W.TensorSpec("dtype", 2, 2, W.ROWS, grad_dtype=7)])
     assert e.value.status == -1
+    # sizes that overflow int64: one tensor (rows * cols), and the sum over tensors
+    with pytest.raises(am.AdamMiniError) as e:
+        am.Partition([W.TensorSpec("huge", 1 << 40, 1 << 40, W.ROWS)])
+    assert e.value.status == -2
+    with pytest.raises(am.AdamMiniError) as e:
+        am.Partition([W.TensorSpec(f"t{i}", 1 << 62, 1, W.ROWS) for i in range(3)])
+    assert e.value.status == -7
 
 
 def test_status_strings():
