@@ -289,7 +289,8 @@ int adammini_query(const am_handle *h, int32_t what, int64_t *value);
  * (may be NULL) receives the number of steps averaged. */
 int adammini_get_profile(am_handle *h, float *ms, int32_t *n_steps);
 
-/* The CUDA error code (cudaError_t as int) of the last AM_ERR_CUDA on this handle. */
+/* The CUDA error code (cudaError_t as int) of the last AM_ERR_CUDA on this handle; with
+ * h == NULL, of the calling thread's last adammini_create that failed with AM_ERR_CUDA. */
 int adammini_last_cuda_error(const am_handle *h);
 
 int adammini_destroy(am_handle *h);

@@ -117,7 +117,7 @@ def _check(status: int, handle=None) -> None:
     if status != 0:
         lib = load()
         msg = lib.adammini_status_string(status).decode()
-        if status == -4 and handle is not None:
+        if status == -4:          # no handle: the error of the creation that just failed
             msg += f" (cudaError {lib.adammini_last_cuda_error(handle)})"
         raise AdamMiniError(status, msg)
 

@@ -262,6 +262,9 @@ int refresh_pointers(am_handle *h, void *const *params, const void *const *grads
 
 extern "C" {
 
+// CUDA error of the last adammini_create that failed in this thread (there is no handle to ask then)
+static thread_local int g_create_cuda_error = 0;
+
 int adammini_create(const am_partition *part, const am_hparams *hp, am_handle **out) {
     if (!out) return AM_ERR_INVALID_ARGUMENT;
     *out = nullptr;
@@ -295,13 +298,13 @@ int adammini_create(const am_partition *part, const am_hparams *hp, am_handle **
     if (e == cudaSuccess) *h->error_word = 0;
     if (e == cudaSuccess) e = stream_configure_kernels();
     if (e != cudaSuccess) {
-        const int code = static_cast<int>(e);
+        g_create_cuda_error = static_cast<int>(e);
         adammini_destroy(h);
-        (void)code;
         return AM_ERR_CUDA;
     }
     rc = build_plan(h);
     if (rc != AM_OK) {
+        if (rc == AM_ERR_CUDA) g_create_cuda_error = h->last_cuda_error;
         adammini_destroy(h);
         return rc;
     }
@@ -382,7 +385,7 @@ int adammini_query(const am_handle *h, int32_t what, int64_t *value) {
     return AM_OK;
 }
 
-int adammini_last_cuda_error(const am_handle *h) { return h ? h->last_cuda_error : 0; }
+int adammini_last_cuda_error(const am_handle *h) { return h ? h->last_cuda_error : g_create_cuda_error; }
 
 int adammini_step(am_handle *h, void *const *params, const void *const *grads, void *const *m,
                   float *v, int64_t step, void *cuda_stream) {

@@ -120,6 +120,8 @@ def test_creating_a_handle_without_a_device_reports_a_cuda_error():
     with pytest.raises(am.AdamMiniError) as e:
         am.AdamMini(part, lr=1e-3, beta1=0.9, beta2=0.95, eps=1e-8, weight_decay=0.1)
     assert e.value.status == -4
+    assert binding.load().adammini_last_cuda_error(None) != 0          # which CUDA error it was
+    assert "cudaError" in str(e.value)
 
 
 def test_random_descriptors_agree_with_the_reference_partitioner():
