@@ -237,6 +237,26 @@ def check_widening(lib):
     p2 = np.zeros(2); m2 = np.zeros(2); v2 = np.zeros(1)
     ostep.adammini_step(p2, m2, v2, g32, 2, step=1, lib=lib, **HP)
     assert np.array_equal(p, p2) and np.array_equal(m, m2) and np.array_equal(v, v2)
+    # float32 gradients keep all 24 significant bits: values bfloat16 cannot hold, a denormal,
+    # the largest finite float; numpy's own conversion to float64 is the reference
+    g32 = np.array([1.0 + 2.0 ** -23, np.pi, -1.0 / 3.0, 1e-30, 1.4e-45, 3.4028235e38, -7.0e-5, 123456.789],
+                   dtype=np.float32)
+    pa = np.linspace(-1.0, 1.0, 8); ma = np.zeros(8); va = np.zeros(2)
+    pb = pa.copy(); mb = np.zeros(8); vb = np.zeros(2)
+    for t in (1, 2):
+        ostep.adammini_step(pa, ma, va, g32, 4, step=t, lib=lib, **HP)
+        ostep.adammini_step(pb, mb, vb, g32.astype(np.float64), 4, step=t, lib=lib, **HP)
+    assert np.array_equal(pa, pb) and np.array_equal(ma, mb) and np.array_equal(va, vb)
+    assert ma[0] - 0.19 > 1e-8                                  # m = 0.19 * (1 + 2^-23): the last bit of g is there
+    rng = np.random.default_rng(5)
+    bits32 = rng.integers(0, 1 << 32, 4096, dtype=np.uint64).astype(np.uint32)
+    src = bits32.view(np.float32)
+    out32 = np.empty(4096, dtype=np.float64)
+    lib.oracle_widen_f32(src.ctypes.data, out32.ctypes.data, 4096)
+    with np.errstate(invalid="ignore"):
+        want32 = src.astype(np.float64)
+    ok = ~np.isnan(want32)
+    assert np.array_equal(out32[ok], want32[ok]) and np.isnan(out32[~ok]).all()
     del ctypes
 
 

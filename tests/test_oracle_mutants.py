@@ -25,6 +25,30 @@ MUTANTS = {
     "update_sign": ("p[k] = p[k] - lr * m_hat / denom;", "p[k] = p[k] + lr * m_hat / denom;"),
     "bf16_shift": ("((uint32_t)h) << 16", "((uint32_t)h) << 15"),
     "mean_over_tensor": ("sum_sq / (double)L", "sum_sq / (double)numel"),
+    # second wave
+    "decay_flag_ignored": ("if (apply_wd)", "if (1)"),
+    # (p - lr*u) * (1 - lr*wd) instead of p * (1 - lr*wd) - lr*u
+    "decay_after_the_adam_term": ("p[k] = p[k] - lr * m_hat / denom;",
+                                  "p[k] = p[k] - lr * m_hat / denom * (apply_wd ? 1.0 - lr * wd : 1.0);"),
+    "bias_corrections_swapped": ("const double bc1 = 1.0 - pow(beta1, (double)t);",
+                                 "const double bc1 = 1.0 - pow(beta2, (double)t);"),
+    "beta2_bias_uses_beta1": ("const double bc2 = 1.0 - pow(beta2, (double)t);",
+                              "const double bc2 = 1.0 - pow(beta1, (double)t);"),
+    "v_not_stored": ("v[b] = (1.0 - beta2) * mean_sq + beta2 * v[b];\n        const double v_hat = v[b] / bc2;",
+                     "const double v_new = (1.0 - beta2) * mean_sq + beta2 * v[b];\n        const double v_hat = v_new / bc2;"),
+    "v_hat_from_old_v": ("v[b] = (1.0 - beta2) * mean_sq + beta2 * v[b];\n        const double v_hat = v[b] / bc2;",
+                         "const double v_hat = v[b] / bc2;\n        v[b] = (1.0 - beta2) * mean_sq + beta2 * v[b];"),
+    "root_dropped": ("sqrt(v_hat) + eps", "v_hat + eps"),
+    "eps_dropped": ("sqrt(v_hat) + eps", "sqrt(v_hat)"),
+    "m_updated_after_use": ("const double m_hat = m[k] / bc1;", "const double m_hat = (m[k] - (1.0 - beta1) * gi) / (beta1 > 0 ? beta1 : 1.0) / bc1;"),
+    "last_block_skipped": ("for (int64_t b = 0; b < n_blocks; ++b) {", "for (int64_t b = 0; b + 1 < n_blocks || b == 0; ++b) {"),
+    "last_element_of_block_not_summed": ("for (int64_t i = 0; i < L; ++i) {\n            const double gi = grad_at(g, g_dtype, lo + i);\n            sum_sq",
+                                         "for (int64_t i = 0; i + 1 < L || i == 0; ++i) {\n            const double gi = grad_at(g, g_dtype, lo + i);\n            sum_sq"),
+    "gradient_index_shifted": ("const double gi = grad_at(g, g_dtype, k);", "const double gi = grad_at(g, g_dtype, k > 0 ? k - 1 : k);"),
+    "f32_read_as_bf16_pairs": ("case ORACLE_G_F32:  return (double)((const float *)g)[i];",
+                               "case ORACLE_G_F32:  return widen_bf16(((const uint16_t *)g)[2 * i + 1]);"),
+    "lr_applied_twice": ("p[k] = p[k] - lr * m_hat / denom;", "p[k] = p[k] - lr * lr * m_hat / denom;"),
+    "wd_not_scaled_by_lr": ("p[k] = p[k] - lr * wd * p[k];", "p[k] = p[k] - wd * p[k];"),
 }
 
 
