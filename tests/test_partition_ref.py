@@ -80,3 +80,17 @@ def test_rejects_indivisible_shapes():
         pr.build_table([pr.TensorDesc(10, 4, pr.HEADS, n_heads=3)])
     with pytest.raises(ValueError):
         pr.build_table([pr.TensorDesc(1, 10, pr.FIXED, fixed_block_len=4)])
+
+
+def test_name_rule_precedence():
+    """Algorithm 3 tests the names in a fixed order: embed/output first, then
+    query/key, then value/attn.proj/mlp; anything else is one block."""
+    assert pr.kind_from_name("output_embed_query") == pr.TOKENS
+    assert pr.kind_from_name("embed.key") == pr.TOKENS
+    assert pr.kind_from_name("mlp.query") == pr.HEADS
+    assert pr.kind_from_name("attn.value.key") == pr.HEADS
+    assert pr.kind_from_name("h.0.attn.value") == pr.ROWS
+    assert pr.kind_from_name("h.0.attn.proj") == pr.ROWS
+    assert pr.kind_from_name("h.0.mlp.fc") == pr.ROWS
+    assert pr.kind_from_name("lm_output") == pr.TOKENS
+    assert pr.kind_from_name("ln_f") == pr.WHOLE and pr.kind_from_name("attn.c_proj") == pr.WHOLE
