@@ -49,7 +49,7 @@ def kernel_digest() -> str:
     for name in ("kernels_basic.cuh", "kernels_stream.cuh"):
         text = open(os.path.join(csrc, name)).read()
         if name == "kernels_basic.cuh":
-            text = text[:text.index("// L <= 16: one thread per block")]
+            text = text[:text.index("// Short blocks (L <= 64)")]
         else:
             text = text[:text.index("host-side planning")]          # device code only
         text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)

@@ -63,7 +63,8 @@ int build_plan(am_handle *h) {
     const int n = static_cast<int>(h->rows.size());
     h->path.assign(n, PATH_TWOPASS);
     h->host_tensors.assign(n, DevTensor{});
-    std::vector<Seg> small_segs, piece_segs, block_segs, part_segs, wide_segs;
+    std::vector<Seg> small_segs, tile_segs, piece_segs, block_segs, part_segs, wide_segs;
+    int64_t tile_units = 0;
     int64_t wide_units = 0;
     std::vector<int32_t> part_tensors;
     int64_t part_units = 0;
@@ -101,7 +102,7 @@ int build_plan(am_handle *h) {
 
         int path;
         if (r.kind == AM_PART) path = PATH_TWOPASS;          // its sum of squares comes from outside
-        else if (r.block_len <= kSmallMaxL) path = PATH_SMALL;
+        else if (r.block_len <= kSmallMaxL && !(h->opt[AM_OPT_PATH] == 1 && r.block_len > 16)) path = PATH_SMALL;
         else if (h->opt[AM_OPT_PATH] == 1 || h->opt[AM_OPT_STATISTIC] != 0) path = PATH_TWOPASS;
         else path = stream_classify(r.block_len, r.grad_dtype, h->n_clusters > 0);
         h->path[i] = path;
@@ -116,11 +117,17 @@ int build_plan(am_handle *h) {
 
         if (path == PATH_SMALL) {
             Seg s;
-            s.unit_begin = small_units;
             s.tensor = i;
             s.aux = (r.block_len == 1 && r.v_offset % 4 == 0 && r.numel % 4 == 0) ? 1 : 0;
-            small_units += s.aux ? ceil_div(r.numel, kSmallUnitVec) : ceil_div(r.n_blocks, kSmallUnitBlocks);
-            small_segs.push_back(s);
+            if (s.aux) {                // the AdamW case: four one-element blocks per thread
+                s.unit_begin = small_units;
+                small_units += ceil_div(r.numel, kSmallUnitVec);
+                small_segs.push_back(s);
+            } else {                    // tiles of whole blocks staged in shared memory
+                s.unit_begin = tile_units;
+                tile_units += ceil_div(r.n_blocks, tile_blocks(r.block_len));
+                tile_segs.push_back(s);
+            }
         } else if (path == PATH_TWOPASS) {
             int64_t piece_len = r.block_len, ppb = 1;
             if (r.block_len > kPieceMax) {
@@ -163,7 +170,7 @@ int build_plan(am_handle *h) {
         }
     }
     if (part_units > 0x7fffffffLL || wide_units > 0x7fffffffLL) return AM_ERR_TOO_LARGE;
-    if (small_units > 0x7fffffffLL || piece_units > 0x7fffffffLL || ceil_div(block_units, kThreads / 32) > 0x7fffffffLL)
+    if (small_units > 0x7fffffffLL || tile_units > 0x7fffffffLL || piece_units > 0x7fffffffLL || ceil_div(block_units, kThreads / 32) > 0x7fffffffLL)
         return AM_ERR_TOO_LARGE;
 
     StreamPlan &sp = h->stream;
@@ -175,6 +182,7 @@ int build_plan(am_handle *h) {
     auto take = [&](size_t bytes) { size_t o = off; off = round_up(off + bytes, 256); return o; };
     const size_t o_tensors = take(sizeof(DevTensor) * std::max(n, 1));
     const size_t o_small = take(sizeof(Seg) * std::max<size_t>(small_segs.size(), 1));
+    const size_t o_tile = take(sizeof(Seg) * std::max<size_t>(tile_segs.size(), 1));
     const size_t o_piece = take(sizeof(Seg) * std::max<size_t>(piece_segs.size(), 1));
     const size_t o_block = take(sizeof(Seg) * std::max<size_t>(block_segs.size(), 1));
     const size_t o_partials = take(sizeof(double) * std::max<int64_t>(piece_units, 1));
@@ -188,6 +196,9 @@ int build_plan(am_handle *h) {
     char *base = static_cast<char *>(h->arena);
     h->d_tensors = reinterpret_cast<DevTensor *>(base + o_tensors);
     h->d_small_segs = reinterpret_cast<Seg *>(base + o_small);
+    h->d_tile_segs = reinterpret_cast<Seg *>(base + o_tile);
+    h->n_tile_segs = static_cast<int>(tile_segs.size());
+    h->tile_units = tile_units;
     h->d_piece_segs = reinterpret_cast<Seg *>(base + o_piece);
     h->d_block_segs = reinterpret_cast<Seg *>(base + o_block);
     h->d_partials = reinterpret_cast<double *>(base + o_partials);
@@ -213,6 +224,8 @@ int build_plan(am_handle *h) {
     h->block_units = block_units;
     if (!small_segs.empty())
         AM_CUDA(h, cudaMemcpy(h->d_small_segs, small_segs.data(), sizeof(Seg) * small_segs.size(), cudaMemcpyHostToDevice));
+    if (!tile_segs.empty())
+        AM_CUDA(h, cudaMemcpy(h->d_tile_segs, tile_segs.data(), sizeof(Seg) * tile_segs.size(), cudaMemcpyHostToDevice));
     if (!piece_segs.empty())
         AM_CUDA(h, cudaMemcpy(h->d_piece_segs, piece_segs.data(), sizeof(Seg) * piece_segs.size(), cudaMemcpyHostToDevice));
     if (!block_segs.empty())
@@ -222,7 +235,7 @@ int build_plan(am_handle *h) {
         if (e != cudaSuccess) return cuda_fail(h, e);
     }
 
-    h->launches = (small_units ? 1 : 0) + (piece_units ? 3 : 0) + (wide_units ? 1 : 0) + sp.launches();
+    h->launches = (small_units ? 1 : 0) + (tile_units ? 1 : 0) + (piece_units ? 3 : 0) + (wide_units ? 1 : 0) + sp.launches();
     h->planned = true;
     return AM_OK;
 }
@@ -447,7 +460,7 @@ int adammini_step_ex(am_handle *h, void *const *params, const void *const *grads
     const bool prof = h->opt[AM_OPT_PROFILE] != 0;
     cudaEvent_t *pev = prof ? &h->prof_ev[(h->prof_steps % h->opt[AM_OPT_PROFILE]) * 5] : nullptr;
     if (prof) AM_CUDA(h, cudaEventRecord(pev[0], stream));
-    if (h->small_units) {
+    if (h->small_units || h->tile_units) {
         SmallScalars ss;
         ss.beta1 = sc.beta1;
         ss.omb1 = sc.omb1;
@@ -461,9 +474,16 @@ int adammini_step_ex(am_handle *h, void *const *params, const void *const *grads
         ss.gscale_dev = sc.gscale_dev;
         ss.skip_flag = sc.skip_flag;
         ss.statistic = sc.statistic;
-        small_kernel<<<static_cast<unsigned>(h->small_units), kThreads, 0, stream>>>(
-            h->d_tensors, h->d_small_segs, h->n_small_segs, v, ss);
-        AM_CUDA(h, cudaGetLastError());
+        if (h->small_units) {
+            small_kernel<<<static_cast<unsigned>(h->small_units), kThreads, 0, stream>>>(
+                h->d_tensors, h->d_small_segs, h->n_small_segs, v, ss);
+            AM_CUDA(h, cudaGetLastError());
+        }
+        if (h->tile_units) {
+            tile_kernel<<<static_cast<unsigned>(h->tile_units), kThreads, 0, stream>>>(
+                h->d_tensors, h->d_tile_segs, h->n_tile_segs, v, ss);
+            AM_CUDA(h, cudaGetLastError());
+        }
     }
     h->stream.bf16_copies = ex && ex->params_bf16;
     if (prof) AM_CUDA(h, cudaEventRecord(pev[1], stream));
