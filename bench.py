@@ -261,7 +261,7 @@ def run_ours(args):
     fam_ms, prof_steps = opt.get_profile()
     opt.set_option(B.OPT_PROFILE, 0)
     fam_bytes = [opt.query(q) for q in (B.Q_BYTES_SMALL, B.Q_BYTES_STREAM, B.Q_BYTES_CLUSTER, B.Q_BYTES_TWOPASS)]
-    fam_names = ["small_kernel", "stream_kernel<false>", "stream_kernel<true>", "twopass_kernels"]
+    fam_names = ["short_block_kernels", "stream_kernel<false>", "stream_kernel<true>", "twopass_kernels"]
     peak, peak_kind = measured_peak_gbs()
     kernels = {}
     for nme, ms_k, by in zip(fam_names, fam_ms, fam_bytes):

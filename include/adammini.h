@@ -237,7 +237,8 @@ int adammini_sync_status(am_handle *h, void *cuda_stream);
 /* Options and queries (keys below).  Unknown keys: AM_ERR_INVALID_ARGUMENT. */
 typedef enum {
     AM_OPT_PATH           = 0, /* 0 = automatic; 1 = force the two-pass path for every tensor with
-                                  block_len > 16 (correctness anchor) */
+                                  block_len > 16 (correctness anchor: a second implementation of every
+                                  other kernel family's work) */
     AM_OPT_STREAM_CTAS    = 1, /* persistent CTAs of the streaming kernel (0 = one per SM) */
     AM_OPT_CLUSTER_SIZE   = 2, /* CTAs per cluster for head-sized blocks: 1, 2, 4, 8 (0 = chosen by block size) */
     AM_OPT_STREAM_THREADS = 3, /* threads per consumer group of the streaming kernels, a multiple of 32
@@ -266,7 +267,7 @@ typedef enum {
     AM_Q_SCRATCH_BYTES     = 1, /* device scratch owned by the handle */
     AM_Q_TOTAL_BLOCKS      = 2,
     AM_Q_TOTAL_ELEMENTS    = 3,
-    AM_Q_ELEMENTS_SMALL    = 4, /* elements routed to the thread-per-block kernel (block_len <= 16) */
+    AM_Q_ELEMENTS_SMALL    = 4, /* elements routed to the short-block kernels (block_len <= 64) */
     AM_Q_ELEMENTS_STREAM   = 5, /* ... to the single-launch streaming kernel */
     AM_Q_ELEMENTS_CLUSTER  = 6, /* ... to the cluster kernel (head-sized blocks) */
     AM_Q_ELEMENTS_TWOPASS  = 7, /* ... to the two-pass path (blocks beyond on-chip/L2 reach, or unaligned) */
@@ -284,8 +285,8 @@ typedef enum {
 int adammini_query(const am_handle *h, int32_t what, int64_t *value);
 
 /* With AM_OPT_PROFILE set: waits for the recorded steps and writes the mean device time in
- * milliseconds per step of each kernel family to ms[0..3] (host array): thread-per-block
- * kernel, streaming kernel, cluster kernel, two-pass kernels (0 where none ran).  *n_steps
+ * milliseconds per step of each kernel family to ms[0..3] (host array): short-block
+ * kernels, streaming kernel, cluster kernel, two-pass kernels (0 where none ran).  *n_steps
  * (may be NULL) receives the number of steps averaged. */
 int adammini_get_profile(am_handle *h, float *ms, int32_t *n_steps);
 

@@ -279,7 +279,7 @@ class AdamMini:
 
     def get_profile(self):
         """Mean device milliseconds per step of each kernel family over the steps
-        recorded since OPT_PROFILE was set: ([thread-per-block, streaming, cluster,
+        recorded since OPT_PROFILE was set: ([short-block, streaming, cluster,
         two-pass], number of steps averaged)."""
         ms = (ctypes.c_float * 4)()
         n = ctypes.c_int32()

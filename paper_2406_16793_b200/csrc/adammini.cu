@@ -14,6 +14,7 @@
 #include "adammini_internal.h"
 #include "kernels_basic.cuh"
 #include "kernels_stream.cuh"
+#include "kernels_tile.cuh"
 #include "host_state.h"
 
 using namespace am;
@@ -310,6 +311,7 @@ int adammini_create(const am_partition *part, const am_hparams *hp, am_handle **
     if (e == cudaSuccess) e = cudaMallocHost(&h->error_word, sizeof(int));
     if (e == cudaSuccess) *h->error_word = 0;
     if (e == cudaSuccess) e = stream_configure_kernels();
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(tile_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileSmemBytes);
     if (e != cudaSuccess) {
         g_create_cuda_error = static_cast<int>(e);
         adammini_destroy(h);
@@ -480,8 +482,8 @@ int adammini_step_ex(am_handle *h, void *const *params, const void *const *grads
             AM_CUDA(h, cudaGetLastError());
         }
         if (h->tile_units) {
-            tile_kernel<<<static_cast<unsigned>(h->tile_units), kThreads, 0, stream>>>(
-                h->d_tensors, h->d_tile_segs, h->n_tile_segs, v, ss);
+            tile_kernel<<<static_cast<unsigned>(h->tile_units), kThreads, kTileSmemBytes, stream>>>(
+                h->d_tensors, h->d_tile_segs, h->n_tile_segs, v, ss, h->error_word);
             AM_CUDA(h, cudaGetLastError());
         }
     }

@@ -1,6 +1,6 @@
-// Device helpers, the kernels for short blocks (L <= 64) and the two-pass
-// kernels (partial sums -> finalize -> update) that handle any block length and
-// any alignment.  Update rule: Algorithm 1 of the paper.
+// Device helpers, the kernel for one-element blocks and the two-pass kernels
+// (partial sums -> finalize -> update) that handle any block length and any
+// alignment.  Update rule: Algorithm 1 of the paper.
 #ifndef ADAMMINI_KERNELS_BASIC_CUH_
 #define ADAMMINI_KERNELS_BASIC_CUH_
 
@@ -14,9 +14,6 @@ namespace am {
 constexpr int kThreads = 256;            // CTA size of the kernels in this file
 constexpr int kSmallMaxL = 64;           // blocks up to this length go to the short-block kernels
 constexpr int kSmallUnitVec = 4096;      // elements per CTA unit (L == 1, float4 path)
-constexpr int kTileElems = 8192;         // elements per CTA unit of the tile kernel ...
-constexpr int kTileMaxBlocks = 1024;     // ... and at most this many blocks
-constexpr int kTileWords = 9216;         // >= blocks * (L | 1) for every L <= kSmallMaxL
 constexpr int64_t kPieceMax = 32768;     // elements per partial sum, two-pass path
 constexpr int64_t kMaxPiecesPerBlock = 16384;
 constexpr int64_t kWideBlockPieces = 256;   // blocks with at least this many partial sums are finalized by a whole CTA
@@ -146,14 +143,9 @@ __device__ __forceinline__ double warp_sum(double x) {
 }
 
 // ---------------------------------------------------------------------------
-// Short blocks (L <= 64): float32 scalars throughout.
-//  - L == 1 with everything 16-byte aligned: one thread per four blocks (this
-//    is AdamW).
-//  - otherwise the tile kernel: a CTA stages the gradients of a tile of whole
-//    blocks in shared memory with coalesced loads, one thread per block adds up
-//    its block from there (rows padded to an odd stride: no bank conflicts),
-//    then all threads update the tile's elements with coalesced loads and
-//    stores of m and p.  Any block length and alignment; g is read once.
+// Short blocks (L <= 64): float32 scalars throughout.  L == 1 with everything
+// 16-byte aligned runs here, one thread per four blocks (this is AdamW); every
+// other case runs on the tile kernel (kernels_tile.cuh).
 // ---------------------------------------------------------------------------
 struct SmallScalars {
     float beta1, omb1, beta2, omb2, inv_bc2, lr_over_bc1, eps, lr_wd, gscale;
@@ -209,107 +201,6 @@ small_kernel(const DevTensor *__restrict__ tensors, const Seg *__restrict__ segs
     const int64_t local = unit - seg.unit_begin;
     if (t.gdtype == AM_BF16) small_body<AM_BF16>(t, local, v, sc);
     else small_body<AM_F32>(t, local, v, sc);
-}
-
-// Blocks per tile: a multiple of four, so that every tile starts on a 16-byte boundary.
-__host__ __device__ inline int tile_blocks(int64_t L) {
-    int64_t nb = kTileElems / L;
-    if (nb > kTileMaxBlocks) nb = kTileMaxBlocks;
-    return static_cast<int>(nb & ~int64_t(3));
-}
-
-template <int GD>
-__device__ __forceinline__ void tile_body(const DevTensor &t, int64_t tile, float *__restrict__ v,
-                                          const SmallScalars &sc, float *sg, float *sstep) {
-    const int L = static_cast<int>(t.L), Ls = L | 1;
-    const int per_tile = tile_blocks(L);
-    const int64_t b0 = tile * per_tile;
-    const int64_t left = t.n_blocks - b0;
-    const int nb = static_cast<int>(left < per_tile ? left : per_tile);
-    const int64_t e0 = b0 * L;                   // a multiple of four elements
-    const int n = nb * L, nvec = n & ~3;         // a ragged last tile ends with up to three single elements
-    const float lr_wd = t.wd ? sc.lr_wd : 0.f;
-    const float gscale = effective_gscale(sc.gscale, sc.gscale_dev);
-
-    // gradients -> shared memory, block b of the tile at sg[b * Ls ...]
-    for (int i = threadIdx.x * 4; i < nvec; i += kThreads * 4) {
-        const float4 g = load_g4<GD>(t.g, e0 + i, gscale);
-        const float x[4] = {g.x, g.y, g.z, g.w};
-        int b = i / L, k = i - b * L;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            sg[b * Ls + k] = x[j];
-            if (++k == L) { k = 0; ++b; }
-        }
-    }
-    for (int i = nvec + threadIdx.x; i < n; i += kThreads) {
-        const int b = i / L;
-        sg[b * Ls + (i - b * L)] = load_g1<GD>(t.g, e0 + i, gscale);
-    }
-    __syncthreads();
-
-    // one thread per block: statistic, v and the block's step size
-    float *vt = v + t.v_offset + b0;
-    for (int b = threadIdx.x; b < nb; b += kThreads) {
-        const float *row = sg + b * Ls;
-        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-        int k = 0;
-        for (; k + 3 < L; k += 4) {
-            s0 = fmaf(row[k], row[k], s0); s1 = fmaf(row[k + 1], row[k + 1], s1);
-            s2 = fmaf(row[k + 2], row[k + 2], s2); s3 = fmaf(row[k + 3], row[k + 3], s3);
-        }
-        for (; k < L; ++k) s0 = fmaf(row[k], row[k], s0);
-        const float sum = (s0 + s1) + (s2 + s3);
-        float stat = L == 1 ? sum : __fdiv_rn(sum, static_cast<float>(L));
-        if (sc.statistic != 0) {
-            // ablation statistics of g*g: max, min, 1-norm, 2-norm
-            double acc = stat_identity(sc.statistic);
-            for (k = 0; k < L; ++k) acc = stat_combine(acc, stat_term(row[k], sc.statistic), sc.statistic);
-            stat = static_cast<float>(stat_finish(acc, static_cast<double>(L), sc.statistic));
-        }
-        float vn;
-        sstep[b] = small_block_step(stat, vt[b], sc, &vn);
-        vt[b] = vn;
-    }
-    __syncthreads();
-
-    // elementwise update, coalesced
-    float *mg = t.m + e0, *pg = t.p + e0;
-    for (int i = threadIdx.x * 4; i < nvec; i += kThreads * 4) {
-        float4 m = *reinterpret_cast<const float4 *>(mg + i);
-        float4 p = *reinterpret_cast<const float4 *>(pg + i);
-        float *mm[4] = {&m.x, &m.y, &m.z, &m.w}, *pp[4] = {&p.x, &p.y, &p.z, &p.w};
-        int b = i / L, k = i - b * L;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            update_one(sg[b * Ls + k], *mm[j], *pp[j], sc.beta1, sc.omb1, lr_wd, sstep[b]);
-            if (++k == L) { k = 0; ++b; }
-        }
-        *reinterpret_cast<float4 *>(mg + i) = m;
-        *reinterpret_cast<float4 *>(pg + i) = p;
-        if (t.p_bf16) store_bf16x4(t.p_bf16 + e0 + i, p);
-    }
-    for (int i = nvec + threadIdx.x; i < n; i += kThreads) {
-        const int b = i / L;
-        float m = mg[i], p = pg[i];
-        update_one(sg[b * Ls + (i - b * L)], m, p, sc.beta1, sc.omb1, lr_wd, sstep[b]);
-        mg[i] = m;
-        pg[i] = p;
-        if (t.p_bf16) store_bf16(t.p_bf16 + e0 + i, p);
-    }
-}
-
-__global__ void __launch_bounds__(kThreads)
-tile_kernel(const DevTensor *__restrict__ tensors, const Seg *__restrict__ segs, int n_segs,
-            float *__restrict__ v, SmallScalars sc) {
-    __shared__ float sg[kTileWords];
-    __shared__ float sstep[kTileMaxBlocks];
-    if (step_skipped(sc.skip_flag)) return;
-    const int64_t unit = blockIdx.x;
-    const Seg seg = segs[find_seg(segs, n_segs, unit)];
-    const DevTensor &t = tensors[seg.tensor];
-    if (t.gdtype == AM_BF16) tile_body<AM_BF16>(t, unit - seg.unit_begin, v, sc, sg, sstep);
-    else tile_body<AM_F32>(t, unit - seg.unit_begin, v, sc, sg, sstep);
 }
 
 // ---------------------------------------------------------------------------

@@ -586,3 +586,30 @@ def test_random_tables_and_launch_options():
         options = _random_options(rng)
         worst = H.run_parity(w, options=options)
         assert max(worst.values()) <= H.TOL, (seed, options, worst)
+
+
+@pytest.mark.parametrize("grad_dtype", [W.F32, W.BF16], ids=["f32", "bf16"])
+def test_every_short_block_length(grad_dtype):
+    """Block lengths 1..64, each over a few tiles of the short-block kernel plus a
+    ragged last tile (whole blocks that end off any 16-byte boundary), with and
+    without weight decay, against the oracle; then the same with a gradient scale,
+    a bf16 copy and an ablation statistic, which take the same kernel."""
+    tensors = [W.TensorSpec(f"l{L}", 3 * (4096 // L) + 5, L, W.ROWS, grad_dtype=grad_dtype, apply_weight_decay=L % 2)
+               for L in range(1, 65)]
+    w = W.Workload("short-blocks", 91 + grad_dtype, tensors, W.GradRecipe(-4.0, -1.0), steps=3)
+    H.assert_parity(H.run_parity(w))
+    H.assert_parity(H.run_parity(w, steps=2, statistic=B.STAT_TWO_NORM))
+    # a bf16 copy does not change the float32 result and is its rounding
+    a, b = H.DeviceState(w, guarded=False), H.DeviceState(w, guarded=True)
+    copies = [H.Guarded(t.numel, torch.bfloat16, "cuda") for t in w.tensors]
+    oa, ob = H.make_optimizer(w), H.make_optimizer(w)
+    a.draw_grads(1)
+    for x, y in zip(a.g, b.g):
+        y.copy_(x)
+    oa.step(a.p, a.g, a.m, a.v, 1)
+    ob.step_ex(b.p, b.g, b.m, b.v, 1, params_bf16=[c.view for c in copies])
+    oa.sync_status(); ob.sync_status()
+    assert _same(a, b) and b.guards_intact()
+    for c, p in zip(copies, b.p):
+        assert torch.equal(c.view, p.to(torch.bfloat16)) and c.intact()
+    oa.close(); ob.close()
