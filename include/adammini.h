@@ -255,8 +255,8 @@ typedef enum {
     AM_OPT_STATISTIC      = 7, /* block statistic that feeds v: 0 = mean(g*g), Algorithm 1.  The ablation
                                   of the paper's appendix ("Ablation Studies on the Design of Adam-mini"),
                                   which it reports to train worse: 1 = max, 2 = min, 3 = 1-norm (sum),
-                                  4 = 2-norm of the vector g*g.  Non-zero values run on the two-pass
-                                  kernels (g read twice) */
+                                  4 = 2-norm of the vector g*g.  Non-zero values run on the short-block
+                                  kernels (block_len <= 64) and the two-pass kernels (g read twice) */
     AM_OPT_STREAM_GROUPS  = 8  /* consumer groups per CTA of the streaming kernel, which own alternate
                                   work items: 1 or 2 (0 = default: 2; the cluster kernel runs one) */
 } am_option;
@@ -267,10 +267,12 @@ typedef enum {
     AM_Q_SCRATCH_BYTES     = 1, /* device scratch owned by the handle */
     AM_Q_TOTAL_BLOCKS      = 2,
     AM_Q_TOTAL_ELEMENTS    = 3,
-    AM_Q_ELEMENTS_SMALL    = 4, /* elements routed to the short-block kernels (block_len <= 64) */
+    AM_Q_ELEMENTS_SMALL    = 4, /* elements routed to the short-block kernels (block_len <= 64, and blocks of
+                                   up to 4096 elements whose starts are not 16-byte aligned) */
     AM_Q_ELEMENTS_STREAM   = 5, /* ... to the single-launch streaming kernel */
     AM_Q_ELEMENTS_CLUSTER  = 6, /* ... to the cluster kernel (head-sized blocks) */
-    AM_Q_ELEMENTS_TWOPASS  = 7, /* ... to the two-pass path (blocks beyond on-chip/L2 reach, or unaligned) */
+    AM_Q_ELEMENTS_TWOPASS  = 7, /* ... to the two-pass path (blocks beyond on-chip/L2 reach, or longer than 4096
+                                   elements with unaligned starts) */
     AM_Q_ALGORITHMIC_BYTES = 8, /* bytes one step must move: per tensor g once (twice for blocks beyond
                                    on-chip/L2 reach), m and p read+written, v read+written */
     AM_Q_BYTES_SMALL       = 9, /* the same, split by the kernel family that handles the tensor */

@@ -105,7 +105,11 @@ int build_plan(am_handle *h) {
         if (r.kind == AM_PART) path = PATH_TWOPASS;          // its sum of squares comes from outside
         else if (r.block_len <= kSmallMaxL && !(h->opt[AM_OPT_PATH] == 1 && r.block_len > 16)) path = PATH_SMALL;
         else if (h->opt[AM_OPT_PATH] == 1 || h->opt[AM_OPT_STATISTIC] != 0) path = PATH_TWOPASS;
-        else path = stream_classify(r.block_len, r.grad_dtype, h->n_clusters > 0);
+        else {
+            path = stream_classify(r.block_len, r.grad_dtype, h->n_clusters > 0);
+            // block starts off the 16-byte grid: the tile kernel copes, up to its tile size
+            if (path == PATH_TWOPASS && r.block_len <= kTileMaxL) path = PATH_SMALL;
+        }
         h->path[i] = path;
         h->elems_by_path[path] += r.numel;
 

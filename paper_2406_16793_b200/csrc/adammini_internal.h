@@ -16,7 +16,7 @@ namespace am {
 
 // Which kernel family updates a tensor.
 enum Path : int32_t {
-    PATH_SMALL = 0,    // block_len <= 64: the short-block kernels
+    PATH_SMALL = 0,    // block_len <= 64, or <= 4096 with unaligned block starts: small_kernel / tile_kernel
     PATH_STREAM = 1,   // blocks that fit a shared-memory stage, and rows re-read from L2
     PATH_CLUSTER = 2,  // head-sized blocks: one thread-block cluster per block
     PATH_TWOPASS = 3   // everything else: partial sums, finalize, update (g read twice)

@@ -1,14 +1,23 @@
-// Short blocks (block length <= 64, any alignment), float32 scalars throughout.
+// Blocks that the streaming kernels do not take: short ones (block length
+// <= 64) and those of up to 4096 elements whose length breaks the 16-byte
+// alignment of block starts.  float32 scalars throughout.
 //
-// A CTA handles one tile of whole blocks (up to 4096 elements).  One thread
-// starts three bulk asynchronous copies (g, m and p of the tile, completion
-// counted on an mbarrier), so that about 50 KB per CTA are in flight without
-// holding a register.  When they have landed, the gradients are widened and
-// re-laid into rows padded to an odd stride, one thread per block adds up its
-// row (Algorithm 1: v = (1-beta2) mean(g*g) + beta2 v; no bank conflicts thanks
-// to the odd stride) and leaves the block's step size in shared memory, and all
-// threads update the tile's elements from shared memory and write m and p back
-// with coalesced 16-byte stores.  g is read from HBM once.
+// A CTA handles one tile: a run of whole blocks of one tensor, up to 4096
+// elements, starting wherever the first block starts.  One thread starts three
+// bulk asynchronous copies (the 32-byte aligned middle of the tile's g, m and p;
+// completion counted on an mbarrier), so that about 50 KB per CTA are in flight
+// without holding a register; the up to seven elements before and after the
+// aligned middle come by plain loads, and every thread fetches the old v of its
+// blocks meanwhile.  When the copies have landed, the gradients are widened and
+// scaled into float rows in shared memory.  Then the block sums
+// (Algorithm 1: v = (1-beta2) mean(g*g) + beta2 v):
+//   L <= 64: one thread per block, rows padded to an odd stride (no bank conflicts);
+//   L  > 64: eight lanes per block (up to 256 elements) or a warp per block,
+//            striding over the row.
+// The block's step size stays in shared memory, and all threads update the
+// tile's elements from shared memory and write m and p back with coalesced
+// 16-byte stores (single elements up to the first 16-byte boundary and after the
+// last).  g is read from HBM once.
 //
 // The wait on the mbarrier is bounded like those of the streaming kernels.
 #ifndef ADAMMINI_KERNELS_TILE_CUH_
@@ -24,17 +33,27 @@ namespace am {
 
 constexpr int kTileElems = 4096;         // elements per tile ...
 constexpr int kTileMaxBlocks = 1024;     // ... and at most this many blocks
-constexpr int kTileWords = 5120;         // >= blocks * (L | 1) for every L <= kSmallMaxL
-// shared memory: m, p, the raw gradients, the padded gradient rows, the step sizes, the mbarrier
-constexpr int kTileSmemBytes = (3 * kTileElems + kTileWords + kTileMaxBlocks) * 4 + 16;
+constexpr int kTileMaxL = 4096;          // longest block the kernel takes
+constexpr int kTileLinear = kTileElems + 8;   // a tile in shared memory, shifted by up to 7 elements
+constexpr int kTileWords = 5120;         // >= blocks * (L | 1) for every L <= kSmallMaxL, and >= kTileLinear
+// shared memory: m, p, the raw gradients, the gradient rows, the step sizes, the mbarrier
+constexpr int kTileSmemBytes = (3 * kTileLinear + kTileWords + kTileMaxBlocks) * 4 + 16;
 constexpr int kTileTimeoutCode = 7;
+static_assert(kTileWords >= kTileLinear, "long rows are stored unpadded");
 
-// Blocks per tile: a multiple of eight, so that every tile starts on a 16-byte
-// boundary whatever the block length and the gradient type.
+// Blocks per tile.  Short blocks: a multiple of eight, so that every tile starts
+// on a 32-byte boundary; longer ones: as many as fit.
 __host__ __device__ inline int tile_blocks(int64_t L) {
     int64_t nb = kTileElems / L;
+    if (L > kSmallMaxL) return static_cast<int>(nb < 1 ? 1 : nb);
     if (nb > kTileMaxBlocks) nb = kTileMaxBlocks;
     return static_cast<int>(nb & ~int64_t(7));
+}
+
+template <int GD>
+__device__ __forceinline__ float tile_raw_at(const unsigned char *sraw, int j) {
+    if (GD == AM_BF16) return __uint_as_float(static_cast<uint32_t>(reinterpret_cast<const uint16_t *>(sraw)[j]) << 16);
+    return reinterpret_cast<const float *>(sraw)[j];
 }
 
 template <int GD>
@@ -42,45 +61,64 @@ __device__ __forceinline__ void tile_body(const DevTensor &t, int64_t tile, floa
                                           const SmallScalars &sc, int *error_word, float *sm, float *sp,
                                           unsigned char *sraw, float *sg, float *sstep, unsigned long long *bar) {
     constexpr int gsz = GD == AM_BF16 ? 2 : 4;
-    const int L = static_cast<int>(t.L), Ls = L | 1;
+    const int L = static_cast<int>(t.L);
+    const bool short_rows = L <= kSmallMaxL;
+    const int Ls = short_rows ? (L | 1) : L;     // row stride of the widened gradients
     const int per_tile = tile_blocks(L);
     const int64_t b0 = tile * per_tile;
     const int64_t left = t.n_blocks - b0;
     const int nb = static_cast<int>(left < per_tile ? left : per_tile);
-    const int64_t e0 = b0 * L;                   // a multiple of eight elements
+    const int64_t e0 = b0 * L;
     const int n = nb * L;
-    const int nbulk = n & ~7;                    // a ragged last tile ends with up to seven single elements
+    // element i of the tile sits at index i + shift of the linear arrays, so that the
+    // 32-byte aligned part of global memory lands 32-byte aligned in shared memory
+    const int shift = static_cast<int>(e0 & 7);
+    const int head = min(n, (8 - shift) & 7);            // elements before the first 32-byte boundary
+    const int nbulk = (n - head) & ~7;                   // the aligned middle
+    const int lead = min(n, (4 - static_cast<int>(e0 & 3)) & 3);   // elements before the first 16-byte boundary
+    const int nvec = (n - lead) & ~3;                    // elements updated four at a time
     const float lr_wd = t.wd ? sc.lr_wd : 0.f;
     const float gscale = effective_gscale(sc.gscale, sc.gscale_dev);
     float *mg = t.m + e0, *pg = t.p + e0;
     const unsigned char *gg = static_cast<const unsigned char *>(t.g) + e0 * gsz;
+    // long rows: 8 lanes add up a block of up to 256 elements, a whole warp a longer one
+    const int glanes = L <= 256 ? 8 : 32, groups = kThreads / glanes;
 
     if (threadIdx.x == 0) {
         mbar_init(bar, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         if (nbulk > 0) {
             mbar_arrive_expect_tx(bar, static_cast<uint32_t>(nbulk) * (gsz + 8));
-            bulk_load(sraw, gg, nbulk * gsz, bar);
-            bulk_load(sm, mg, nbulk * 4, bar);
-            bulk_load(sp, pg, nbulk * 4, bar);
+            bulk_load(sraw + (shift + head) * gsz, gg + head * gsz, nbulk * gsz, bar);
+            bulk_load(sm + shift + head, mg + head, nbulk * 4, bar);
+            bulk_load(sp + shift + head, pg + head, nbulk * 4, bar);
         }
     }
-    // the ragged end, by plain loads
-    for (int i = nbulk + threadIdx.x; i < n; i += kThreads) {
-        sm[i] = mg[i];
-        sp[i] = pg[i];
-        if (GD == AM_BF16) reinterpret_cast<uint16_t *>(sraw)[i] = reinterpret_cast<const uint16_t *>(gg)[i];
-        else reinterpret_cast<float *>(sraw)[i] = reinterpret_cast<const float *>(gg)[i];
+    // the ends, by plain loads
+    for (int i = threadIdx.x; i < n - nbulk; i += kThreads) {
+        const int k = i < head ? i : i + nbulk;
+        sm[k + shift] = mg[k];
+        sp[k + shift] = pg[k];
+        if (GD == AM_BF16) reinterpret_cast<uint16_t *>(sraw)[k + shift] = reinterpret_cast<const uint16_t *>(gg)[k];
+        else reinterpret_cast<float *>(sraw)[k + shift] = reinterpret_cast<const float *>(gg)[k];
     }
-    // the old v of this thread's blocks, fetched while the copies fly
+    // the old v of this thread's (short rows) or this warp's blocks, fetched while the copies fly
     float *vt = v + t.v_offset + b0;
     float v_old[kTileMaxBlocks / kThreads];
 #pragma unroll
-    for (int r = 0; r < kTileMaxBlocks / kThreads; ++r) {
-        const int b = threadIdx.x + r * kThreads;
-        v_old[r] = b < nb ? vt[b] : 0.f;
+    for (int r = 0; r < kTileMaxBlocks / kThreads; ++r) v_old[r] = 0.f;
+    if (short_rows) {
+#pragma unroll
+        for (int r = 0; r < kTileMaxBlocks / kThreads; ++r) {
+            const int b = threadIdx.x + r * kThreads;
+            if (b < nb) v_old[r] = vt[b];
+        }
+    } else {
+        // a group of `glanes` lanes per block; the group's lane r holds the old v of the group's r-th block
+        const int b = threadIdx.x / glanes + (threadIdx.x % glanes) * groups;
+        if (b < nb) v_old[0] = vt[b];
     }
-    __syncthreads();                             // the barrier exists; the ragged end is in place
+    __syncthreads();                             // the barrier exists; the ends are in place
     if (nbulk > 0) {
         // bounded wait for the copies (phase 0 of the barrier)
         unsigned spins = 0;
@@ -106,60 +144,102 @@ __device__ __forceinline__ void tile_body(const DevTensor &t, int64_t tile, floa
         }
     }
 
-    // gradients, widened and scaled -> rows of odd stride: block b of the tile at sg[b * Ls ...]
-    for (int i = threadIdx.x * 4; i < n; i += kThreads * 4) {
-        float x[4];
-        if (i + 3 < n) {
-            const float4 g = lds_g4<GD>(sraw, i);
-            x[0] = g.x; x[1] = g.y; x[2] = g.z; x[3] = g.w;
-        } else {
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
-                x[j] = i + j < n ? (GD == AM_BF16 ? __uint_as_float(static_cast<uint32_t>(reinterpret_cast<const uint16_t *>(sraw)[i + j]) << 16)
-                                                  : reinterpret_cast<const float *>(sraw)[i + j])
-                                 : 0.f;
-        }
+    // gradients, widened and scaled -> rows: block b of the tile at sg[b * Ls ...]
+    for (int i = threadIdx.x; i < lead; i += kThreads) {
+        const int b = i / L;
+        sg[b * Ls + (i - b * L)] = tile_raw_at<GD>(sraw, i + shift) * gscale;
+    }
+    for (int i = lead + threadIdx.x * 4; i < lead + nvec; i += kThreads * 4) {
+        const float4 g = lds_g4<GD>(sraw, i + shift);            // (i + shift) is a multiple of four
+        const float x[4] = {g.x, g.y, g.z, g.w};
         int b = i / L, k = i - b * L;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            if (i + j < n) sg[b * Ls + k] = x[j] * gscale;
+            sg[b * Ls + k] = x[j] * gscale;
             if (++k == L) { k = 0; ++b; }
         }
     }
-    __syncthreads();
-
-    // one thread per block: statistic, v and the block's step size
-#pragma unroll
-    for (int r = 0; r < kTileMaxBlocks / kThreads; ++r) {
-        const int b = threadIdx.x + r * kThreads;
-        if (b >= nb) break;
-        const float *row = sg + b * Ls;
-        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-        int k = 0;
-        for (; k + 3 < L; k += 4) {
-            s0 = fmaf(row[k], row[k], s0); s1 = fmaf(row[k + 1], row[k + 1], s1);
-            s2 = fmaf(row[k + 2], row[k + 2], s2); s3 = fmaf(row[k + 3], row[k + 3], s3);
-        }
-        for (; k < L; ++k) s0 = fmaf(row[k], row[k], s0);
-        const float sum = (s0 + s1) + (s2 + s3);
-        float stat = L == 1 ? sum : __fdiv_rn(sum, static_cast<float>(L));
-        if (sc.statistic != 0) {
-            // ablation statistics of g*g: max, min, 1-norm, 2-norm
-            double acc = stat_identity(sc.statistic);
-            for (k = 0; k < L; ++k) acc = stat_combine(acc, stat_term(row[k], sc.statistic), sc.statistic);
-            stat = static_cast<float>(stat_finish(acc, static_cast<double>(L), sc.statistic));
-        }
-        float vn;
-        sstep[b] = small_block_step(stat, v_old[r], sc, &vn);
-        vt[b] = vn;
+    for (int i = lead + nvec + threadIdx.x; i < n; i += kThreads) {
+        const int b = i / L;
+        sg[b * Ls + (i - b * L)] = tile_raw_at<GD>(sraw, i + shift) * gscale;
     }
     __syncthreads();
 
-    // elementwise update from shared memory, coalesced stores
-    const int nvec = n & ~3;
-    for (int i = threadIdx.x * 4; i < nvec; i += kThreads * 4) {
-        float4 m = *reinterpret_cast<const float4 *>(sm + i);
-        float4 p = *reinterpret_cast<const float4 *>(sp + i);
+    // block statistics, v and the blocks' step sizes
+    if (short_rows) {
+#pragma unroll
+        for (int r = 0; r < kTileMaxBlocks / kThreads; ++r) {
+            const int b = threadIdx.x + r * kThreads;
+            if (b >= nb) break;
+            const float *row = sg + b * Ls;
+            float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+            int k = 0;
+            for (; k + 3 < L; k += 4) {
+                s0 = fmaf(row[k], row[k], s0); s1 = fmaf(row[k + 1], row[k + 1], s1);
+                s2 = fmaf(row[k + 2], row[k + 2], s2); s3 = fmaf(row[k + 3], row[k + 3], s3);
+            }
+            for (; k < L; ++k) s0 = fmaf(row[k], row[k], s0);
+            const float sum = (s0 + s1) + (s2 + s3);
+            float stat = L == 1 ? sum : __fdiv_rn(sum, static_cast<float>(L));
+            if (sc.statistic != 0) {
+                // ablation statistics of g*g: max, min, 1-norm, 2-norm
+                double acc = stat_identity(sc.statistic);
+                for (k = 0; k < L; ++k) acc = stat_combine(acc, stat_term(row[k], sc.statistic), sc.statistic);
+                stat = static_cast<float>(stat_finish(acc, static_cast<double>(L), sc.statistic));
+            }
+            float vn;
+            sstep[b] = small_block_step(stat, v_old[r], sc, &vn);
+            vt[b] = vn;
+        }
+    } else {
+        const int gid = threadIdx.x / glanes, gl = threadIdx.x % glanes;
+        const int rounds = (nb + groups - 1) / groups;            // the same for every thread: shuffles stay converged
+        for (int r = 0; r < rounds; ++r) {
+            const int b = gid + r * groups;
+            const bool live = b < nb;
+            const float *row = sg + (live ? b : 0) * Ls;
+            const float vo = __shfl_sync(0xffffffffu, v_old[0], r, glanes);
+            double tot;
+            if (sc.statistic == 0 || sc.statistic == 3) {
+                // per lane at most 128 terms over four accumulators, then double
+                float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+                int k = gl;
+                for (; k + 3 * glanes < L; k += 4 * glanes) {
+                    s0 = fmaf(row[k], row[k], s0); s1 = fmaf(row[k + glanes], row[k + glanes], s1);
+                    s2 = fmaf(row[k + 2 * glanes], row[k + 2 * glanes], s2);
+                    s3 = fmaf(row[k + 3 * glanes], row[k + 3 * glanes], s3);
+                }
+                for (; k < L; k += glanes) s0 = fmaf(row[k], row[k], s0);
+                tot = (static_cast<double>(s0) + static_cast<double>(s1)) + (static_cast<double>(s2) + static_cast<double>(s3));
+                for (int o = glanes >> 1; o > 0; o >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, o);
+            } else {
+                tot = stat_identity(sc.statistic);
+                for (int k = gl; k < L; k += glanes) tot = stat_combine(tot, stat_term(row[k], sc.statistic), sc.statistic);
+                for (int o = glanes >> 1; o > 0; o >>= 1)
+                    tot = stat_combine(tot, __shfl_xor_sync(0xffffffffu, tot, o), sc.statistic);
+            }
+            if (live && gl == 0) {
+                const float stat = static_cast<float>(stat_finish(tot, static_cast<double>(L), sc.statistic));
+                float vn;
+                sstep[b] = small_block_step(stat, vo, sc, &vn);
+                vt[b] = vn;
+            }
+        }
+    }
+    __syncthreads();
+
+    // elementwise update from shared memory; 16-byte stores where global memory allows
+    for (int i = threadIdx.x; i < lead; i += kThreads) {
+        const int b = i / L;
+        float m = sm[i + shift], p = sp[i + shift];
+        update_one(sg[b * Ls + (i - b * L)], m, p, sc.beta1, sc.omb1, lr_wd, sstep[b]);
+        mg[i] = m;
+        pg[i] = p;
+        if (t.p_bf16) store_bf16(t.p_bf16 + e0 + i, p);
+    }
+    for (int i = lead + threadIdx.x * 4; i < lead + nvec; i += kThreads * 4) {
+        float4 m = *reinterpret_cast<const float4 *>(sm + i + shift);
+        float4 p = *reinterpret_cast<const float4 *>(sp + i + shift);
         float *mm[4] = {&m.x, &m.y, &m.z, &m.w}, *pp[4] = {&p.x, &p.y, &p.z, &p.w};
         int b = i / L, k = i - b * L;
 #pragma unroll
@@ -171,9 +251,9 @@ __device__ __forceinline__ void tile_body(const DevTensor &t, int64_t tile, floa
         *reinterpret_cast<float4 *>(pg + i) = p;
         if (t.p_bf16) store_bf16x4(t.p_bf16 + e0 + i, p);
     }
-    for (int i = nvec + threadIdx.x; i < n; i += kThreads) {
+    for (int i = lead + nvec + threadIdx.x; i < n; i += kThreads) {
         const int b = i / L;
-        float m = sm[i], p = sp[i];
+        float m = sm[i + shift], p = sp[i + shift];
         update_one(sg[b * Ls + (i - b * L)], m, p, sc.beta1, sc.omb1, lr_wd, sstep[b]);
         mg[i] = m;
         pg[i] = p;
@@ -186,9 +266,9 @@ tile_kernel(const DevTensor *__restrict__ tensors, const Seg *__restrict__ segs,
             float *__restrict__ v, SmallScalars sc, int *error_word) {
     extern __shared__ __align__(128) unsigned char tile_smem[];      // kTileSmemBytes
     float *sm = reinterpret_cast<float *>(tile_smem);
-    float *sp = sm + kTileElems;
-    unsigned char *sraw = reinterpret_cast<unsigned char *>(sp + kTileElems);
-    float *sg = reinterpret_cast<float *>(sraw) + kTileElems;
+    float *sp = sm + kTileLinear;
+    unsigned char *sraw = reinterpret_cast<unsigned char *>(sp + kTileLinear);
+    float *sg = reinterpret_cast<float *>(sraw) + kTileLinear;
     float *sstep = sg + kTileWords;
     unsigned long long *bar = reinterpret_cast<unsigned long long *>(sstep + kTileMaxBlocks);
     if (step_skipped(sc.skip_flag)) return;
