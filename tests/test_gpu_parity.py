@@ -613,3 +613,32 @@ def test_every_short_block_length(grad_dtype):
     for c, p in zip(copies, b.p):
         assert torch.equal(c.view, p.to(torch.bfloat16)) and c.intact()
     oa.close(); ob.close()
+
+
+@pytest.mark.parametrize("grad_dtype", [W.F32, W.BF16], ids=["f32", "bf16"])
+def test_unaligned_block_lengths_up_to_a_tile(grad_dtype):
+    """Block lengths whose blocks start off the 16-byte grid, from just above the
+    short-block limit to the tile size and one past it: several tiles each, so that
+    tiles start at every offset within 32 bytes; with a bf16 copy and guards."""
+    lengths = [65, 66, 67, 69, 100, 127, 255, 257, 1001, 1365, 2047, 4095, 4097]
+    tensors = [W.TensorSpec(f"l{L}", max(3 * (4096 // L) + 3, 5), L, W.ROWS, grad_dtype=grad_dtype,
+                            apply_weight_decay=i % 2) for i, L in enumerate(lengths)]
+    w = W.Workload("unaligned-blocks", 93 + grad_dtype, tensors, W.GradRecipe(-4.0, -1.0), steps=3)
+    H.assert_parity(H.run_parity(w))
+    H.assert_parity(H.run_parity(w, steps=2, statistic=B.STAT_MAX))
+    opt = H.make_optimizer(w)
+    assert opt.query(B.Q_ELEMENTS_TWOPASS) == tensors[-1].numel          # only the 4097-element rows
+    opt.close()
+    a, b = H.DeviceState(w, guarded=False), H.DeviceState(w, guarded=True)
+    copies = [H.Guarded(t.numel, torch.bfloat16, "cuda") for t in w.tensors]
+    oa, ob = H.make_optimizer(w), H.make_optimizer(w)
+    a.draw_grads(1)
+    for x, y in zip(a.g, b.g):
+        y.copy_(x)
+    oa.step(a.p, a.g, a.m, a.v, 1)
+    ob.step_ex(b.p, b.g, b.m, b.v, 1, params_bf16=[c.view for c in copies], grad_scale=1.0)
+    oa.sync_status(); ob.sync_status()
+    assert _same(a, b) and b.guards_intact()
+    for c, p in zip(copies, b.p):
+        assert torch.equal(c.view, p.to(torch.bfloat16)) and c.intact()
+    oa.close(); ob.close()
