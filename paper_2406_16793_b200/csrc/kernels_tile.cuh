@@ -50,6 +50,12 @@ __host__ __device__ inline int tile_blocks(int64_t L) {
     return static_cast<int>(nb & ~int64_t(7));
 }
 
+// i / L for 0 <= i < 2^32 / L by one multiplication: magic = floor((2^32 - 1) / L) + 1 (L >= 2).
+// Exact because i * (magic * L - 2^32) < 2^32 for every index of a tile.
+__device__ __forceinline__ int tile_div(int i, int L, uint32_t magic) {
+    return L == 1 ? i : static_cast<int>(__umulhi(static_cast<uint32_t>(i), magic));
+}
+
 template <int GD>
 __device__ __forceinline__ float tile_raw_at(const unsigned char *sraw, int j) {
     if (GD == AM_BF16) return __uint_as_float(static_cast<uint32_t>(reinterpret_cast<const uint16_t *>(sraw)[j]) << 16);
@@ -83,6 +89,7 @@ __device__ __forceinline__ void tile_body(const DevTensor &t, int64_t tile, floa
     const unsigned char *gg = static_cast<const unsigned char *>(t.g) + e0 * gsz;
     // long rows: 8 lanes add up a block of up to 256 elements, a whole warp a longer one
     const int glanes = L <= 256 ? 8 : 32, groups = kThreads / glanes;
+    const uint32_t magic = L == 1 ? 0u : 0xffffffffu / static_cast<uint32_t>(L) + 1u;
 
     if (threadIdx.x == 0) {
         mbar_init(bar, 1);
@@ -146,13 +153,13 @@ __device__ __forceinline__ void tile_body(const DevTensor &t, int64_t tile, floa
 
     // gradients, widened and scaled -> rows: block b of the tile at sg[b * Ls ...]
     for (int i = threadIdx.x; i < lead; i += kThreads) {
-        const int b = i / L;
+        const int b = tile_div(i, L, magic);
         sg[b * Ls + (i - b * L)] = tile_raw_at<GD>(sraw, i + shift) * gscale;
     }
     for (int i = lead + threadIdx.x * 4; i < lead + nvec; i += kThreads * 4) {
         const float4 g = lds_g4<GD>(sraw, i + shift);            // (i + shift) is a multiple of four
         const float x[4] = {g.x, g.y, g.z, g.w};
-        int b = i / L, k = i - b * L;
+        int b = tile_div(i, L, magic), k = i - b * L;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             sg[b * Ls + k] = x[j] * gscale;
@@ -160,7 +167,7 @@ __device__ __forceinline__ void tile_body(const DevTensor &t, int64_t tile, floa
         }
     }
     for (int i = lead + nvec + threadIdx.x; i < n; i += kThreads) {
-        const int b = i / L;
+        const int b = tile_div(i, L, magic);
         sg[b * Ls + (i - b * L)] = tile_raw_at<GD>(sraw, i + shift) * gscale;
     }
     __syncthreads();
@@ -230,7 +237,7 @@ __device__ __forceinline__ void tile_body(const DevTensor &t, int64_t tile, floa
 
     // elementwise update from shared memory; 16-byte stores where global memory allows
     for (int i = threadIdx.x; i < lead; i += kThreads) {
-        const int b = i / L;
+        const int b = tile_div(i, L, magic);
         float m = sm[i + shift], p = sp[i + shift];
         update_one(sg[b * Ls + (i - b * L)], m, p, sc.beta1, sc.omb1, lr_wd, sstep[b]);
         mg[i] = m;
@@ -241,7 +248,7 @@ __device__ __forceinline__ void tile_body(const DevTensor &t, int64_t tile, floa
         float4 m = *reinterpret_cast<const float4 *>(sm + i + shift);
         float4 p = *reinterpret_cast<const float4 *>(sp + i + shift);
         float *mm[4] = {&m.x, &m.y, &m.z, &m.w}, *pp[4] = {&p.x, &p.y, &p.z, &p.w};
-        int b = i / L, k = i - b * L;
+        int b = tile_div(i, L, magic), k = i - b * L;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             update_one(sg[b * Ls + k], *mm[j], *pp[j], sc.beta1, sc.omb1, lr_wd, sstep[b]);
@@ -252,7 +259,7 @@ __device__ __forceinline__ void tile_body(const DevTensor &t, int64_t tile, floa
         if (t.p_bf16) store_bf16x4(t.p_bf16 + e0 + i, p);
     }
     for (int i = lead + nvec + threadIdx.x; i < n; i += kThreads) {
-        const int b = i / L;
+        const int b = tile_div(i, L, magic);
         float m = sm[i + shift], p = sp[i + shift];
         update_one(sg[b * Ls + (i - b * L)], m, p, sc.beta1, sc.omb1, lr_wd, sstep[b]);
         mg[i] = m;
