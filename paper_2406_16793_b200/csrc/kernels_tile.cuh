@@ -12,8 +12,8 @@
 // scaled into float rows in shared memory.  Then the block sums
 // (Algorithm 1: v = (1-beta2) mean(g*g) + beta2 v):
 //   L <= 64: one thread per block, rows padded to an odd stride (no bank conflicts);
-//   L  > 64: eight lanes per block (up to 256 elements) or a warp per block,
-//            striding over the row.
+//   L  > 64: eight lanes per block (up to 256 elements); beyond, one to eight
+//            warps per block, each adding a slice, so that every warp is busy.
 // The block's step size stays in shared memory, and all threads update the
 // tile's elements from shared memory and write m and p back with coalesced
 // 16-byte stores (single elements up to the first 16-byte boundary and after the
@@ -120,10 +120,12 @@ __device__ __forceinline__ void tile_body(const DevTensor &t, int64_t tile, floa
             const int b = threadIdx.x + r * kThreads;
             if (b < nb) v_old[r] = vt[b];
         }
-    } else {
-        // a group of `glanes` lanes per block; the group's lane r holds the old v of the group's r-th block
+    } else if (glanes == 8) {
+        // a group of eight lanes per block; the group's lane r holds the old v of the group's r-th block
         const int b = threadIdx.x / glanes + (threadIdx.x % glanes) * groups;
         if (b < nb) v_old[0] = vt[b];
+    } else if (threadIdx.x < nb) {
+        v_old[0] = vt[threadIdx.x];              // at most 15 blocks of more than 256 elements: thread b finishes block b
     }
     __syncthreads();                             // the barrier exists; the ends are in place
     if (nbulk > 0) {
@@ -198,7 +200,7 @@ __device__ __forceinline__ void tile_body(const DevTensor &t, int64_t tile, floa
             sstep[b] = small_block_step(stat, v_old[r], sc, &vn);
             vt[b] = vn;
         }
-    } else {
+    } else if (glanes == 8) {
         const int gid = threadIdx.x / glanes, gl = threadIdx.x % glanes;
         const int rounds = (nb + groups - 1) / groups;            // the same for every thread: shuffles stay converged
         for (int r = 0; r < rounds; ++r) {
@@ -231,6 +233,47 @@ __device__ __forceinline__ void tile_body(const DevTensor &t, int64_t tile, floa
                 sstep[b] = small_block_step(stat, vo, sc, &vn);
                 vt[b] = vn;
             }
+        }
+    } else {
+        // few long blocks: every warp adds up a slice of a block (1, 2, 4 or 8 warps per block, so that
+        // all eight warps are busy), then thread b adds the slices of block b in order
+        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+        const int wpb = nb >= 8 ? 1 : nb >= 4 ? 2 : nb >= 2 ? 4 : 8;
+        const int slots = nb * wpb, per = (L + wpb - 1) / wpb;
+        double *spart = reinterpret_cast<double *>(sstep + 64);          // slots <= 15 partial sums
+        const bool plain_sum = sc.statistic == 0 || sc.statistic == 3;
+        for (int slot = warp; slot < slots; slot += kThreads / 32) {
+            const int b = slot / wpb, sl = slot - b * wpb;
+            const float *row = sg + b * Ls;
+            const int k1 = min(L, (sl + 1) * per);
+            double tot;
+            if (plain_sum) {
+                // per lane at most 128 terms over four accumulators, then double
+                float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+                int k = sl * per + lane;
+                for (; k + 96 < k1; k += 128) {
+                    s0 = fmaf(row[k], row[k], s0); s1 = fmaf(row[k + 32], row[k + 32], s1);
+                    s2 = fmaf(row[k + 64], row[k + 64], s2); s3 = fmaf(row[k + 96], row[k + 96], s3);
+                }
+                for (; k < k1; k += 32) s0 = fmaf(row[k], row[k], s0);
+                tot = warp_sum((static_cast<double>(s0) + static_cast<double>(s1)) +
+                               (static_cast<double>(s2) + static_cast<double>(s3)));
+            } else {
+                tot = stat_identity(sc.statistic);
+                for (int k = sl * per + lane; k < k1; k += 32) tot = stat_combine(tot, stat_term(row[k], sc.statistic), sc.statistic);
+                tot = warp_stat(tot, sc.statistic);
+            }
+            if (lane == 0) spart[slot] = tot;
+        }
+        __syncthreads();
+        if (threadIdx.x < nb) {
+            const int b = threadIdx.x;
+            double tot = spart[b * wpb];
+            for (int j = 1; j < wpb; ++j) tot = stat_combine(tot, spart[b * wpb + j], sc.statistic);
+            const float stat = static_cast<float>(stat_finish(tot, static_cast<double>(L), sc.statistic));
+            float vn;
+            sstep[b] = small_block_step(stat, v_old[0], sc, &vn);
+            vt[b] = vn;
         }
     }
     __syncthreads();
