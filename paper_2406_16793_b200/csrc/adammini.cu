@@ -147,7 +147,7 @@ int build_plan(am_handle *h) {
             Seg s;
             s.unit_begin = piece_units;
             s.tensor = i;
-            s.aux = (r.block_len % 4 == 0 && r.kind != AM_PART) ? 1 : 0;   // parts may start at any element
+            s.aux = r.kind != AM_PART ? 1 : 0;   // 16-byte accesses; parts may start at any address: single elements
             piece_segs.push_back(s);
             if (r.kind == AM_PART) {
                 t.part_index = static_cast<int32_t>(part_tensors.size());

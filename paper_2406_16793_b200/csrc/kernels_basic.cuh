@@ -210,8 +210,14 @@ small_kernel(const DevTensor *__restrict__ tensors, const Seg *__restrict__ segs
 struct PieceRef {
     const DevTensor *t;
     int64_t block, start, n, local;
-    bool vec;
+    bool vec;               // the tensor's arrays start 16-byte aligned: 16-byte accesses where the element index allows
 };
+
+// Elements of a piece before the first one on a 16-byte boundary.
+__device__ __forceinline__ int64_t piece_lead(const PieceRef &r) {
+    const int64_t lead = (4 - (r.start & 3)) & 3;
+    return lead < r.n ? lead : r.n;
+}
 
 __device__ __forceinline__ PieceRef decode_piece(const DevTensor *tensors, const Seg *segs, int n_segs,
                                                  int64_t unit) {
@@ -236,9 +242,21 @@ template <int GD>
 __device__ __forceinline__ double piece_sum_sq(const PieceRef &r, float gscale) {
     double tot = 0.0;
     if (r.vec) {
+        // 16-byte accesses from the first element on a 16-byte boundary; up to three single
+        // elements before it and after the last full group (none when the block length is a
+        // multiple of four)
+        const int64_t lead = piece_lead(r), nvec = (r.n - lead) & ~int64_t(3);
         float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
         int chain = 0;
-        for (int64_t i = static_cast<int64_t>(threadIdx.x) * 4; i < r.n; i += kThreads * 4) {
+        if (threadIdx.x < lead) {
+            const float g = load_g1<GD>(r.t->g, r.start + threadIdx.x, gscale);
+            a0 = fmaf(g, g, a0);
+        }
+        for (int64_t i = lead + nvec + threadIdx.x; i < r.n; i += kThreads) {
+            const float g = load_g1<GD>(r.t->g, r.start + i, gscale);
+            a1 = fmaf(g, g, a1);
+        }
+        for (int64_t i = lead + static_cast<int64_t>(threadIdx.x) * 4; i < lead + nvec; i += kThreads * 4) {
             const float4 g = load_g4<GD>(r.t->g, r.start + i, gscale);
             a0 = fmaf(g.x, g.x, a0); a1 = fmaf(g.y, g.y, a1);
             a2 = fmaf(g.z, g.z, a2); a3 = fmaf(g.w, g.w, a3);
@@ -391,7 +409,8 @@ __device__ __forceinline__ void twopass_update_body(const PieceRef &r, const flo
     const float lr_wd = t.wd ? sc.lr_wd : 0.f;
     const float gscale = effective_gscale(sc.gscale, sc.gscale_dev);
     if (r.vec) {
-        for (int64_t i = static_cast<int64_t>(threadIdx.x) * 4; i < r.n; i += kThreads * 4) {
+        const int64_t lead = piece_lead(r), nvec = (r.n - lead) & ~int64_t(3);
+        for (int64_t i = lead + static_cast<int64_t>(threadIdx.x) * 4; i < lead + nvec; i += kThreads * 4) {
             const int64_t e = r.start + i;
             const float4 g = load_g4<GD>(t.g, e, gscale);
             float4 m = *reinterpret_cast<const float4 *>(t.m + e);
@@ -400,6 +419,16 @@ __device__ __forceinline__ void twopass_update_body(const PieceRef &r, const flo
             *reinterpret_cast<float4 *>(t.m + e) = m;
             *reinterpret_cast<float4 *>(t.p + e) = p;
             if (t.p_bf16) store_bf16x4(t.p_bf16 + e, p);
+        }
+        // the up to three single elements either side
+        for (int64_t i = threadIdx.x; i < r.n - nvec; i += kThreads) {
+            const int64_t e = r.start + (i < lead ? i : i + nvec);
+            const float g = load_g1<GD>(t.g, e, gscale);
+            float m = t.m[e], p = t.p[e];
+            update_one(g, m, p, sc.beta1, sc.omb1, lr_wd, st);
+            t.m[e] = m;
+            t.p[e] = p;
+            if (t.p_bf16) store_bf16(t.p_bf16 + e, p);
         }
     } else {
         for (int64_t i = threadIdx.x; i < r.n; i += kThreads) {
