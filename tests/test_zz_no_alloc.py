@@ -22,7 +22,8 @@ CASES = [
     (1, 1 << 20, W.WHOLE, 0, 0, W.F32),        # one block, 32 partial sums
     (256, 4096, W.ROWS, 0, 0, W.BF16),         # 256 row blocks
     (512, 1024, W.HEADS, 4, 0, W.BF16),        # 4 head blocks of 131072 elements
-    (1, 70001, W.FIXED, 0, 70001, W.F32),      # odd length: scalar tail path
+    (1, 70001, W.FIXED, 0, 70001, W.F32),      # odd length: single elements after the last group of four
+    (9, 10007, W.ROWS, 0, 0, W.BF16),          # odd rows: blocks start off the 16-byte grid
     (1, 32768, W.FIXED, 0, 1, W.F32),          # block length 1 at the block limit
 ]
 
