@@ -78,6 +78,11 @@ def pick_workload(name: str):
         return W.flat_sweep(int(parts[0]), numel=1 << (int(parts[1]) if len(parts) > 1 else 30))
     if name.startswith("llama2-7b-layers"):
         return W.llama2_7b(n_layers=int(name[len("llama2-7b-layers"):]))
+    if name.startswith("rows-"):                        # rows-<bf16|f32>-L<row length>-r<rows>: one matrix, a block per row
+        dt, cols, rows = name[5:].split("-")
+        spec = W.TensorSpec("mlp.rows", int(rows[1:]), int(cols[1:]), W.ROWS,
+                            grad_dtype=W.BF16 if dt == "bf16" else W.F32)
+        return W.Workload(name, 2, [spec], W.GradRecipe(-5.0, -1.0), steps=10)
     raise SystemExit(f"unknown workload {name}")
 
 

@@ -8,12 +8,15 @@
 // completion counted on an mbarrier), so that about 50 KB per CTA are in flight
 // without holding a register; the up to seven elements before and after the
 // aligned middle come by plain loads, and every thread fetches the old v of its
-// blocks meanwhile.  When the copies have landed, the gradients are widened and
-// scaled into float rows in shared memory.  Then the block sums
-// (Algorithm 1: v = (1-beta2) mean(g*g) + beta2 v):
-//   L <= 64: one thread per block, rows padded to an odd stride (no bank conflicts);
+// blocks meanwhile.  Then the block sums (Algorithm 1: v = (1-beta2) mean(g*g) +
+// beta2 v):
+//   L <= 64: the gradients are first widened and scaled into float rows padded to
+//            an odd stride (no bank conflicts), then one thread adds up a block;
 //   L  > 64: eight lanes per block (up to 256 elements); beyond, one to eight
 //            warps per block, each adding a slice, so that every warp is busy.
+//            Lanes walk a block with stride one, so they read the gradients as
+//            they arrived (widened and scaled on the fly): no second copy in
+//            shared memory and one barrier less than for short blocks.
 // The block's step size stays in shared memory, and all threads update the
 // tile's elements from shared memory and write m and p back with coalesced
 // 16-byte stores (single elements up to the first 16-byte boundary and after the
@@ -62,14 +65,14 @@ __device__ __forceinline__ float tile_raw_at(const unsigned char *sraw, int j) {
     return reinterpret_cast<const float *>(sraw)[j];
 }
 
-template <int GD>
+template <int GD, bool LONG>
 __device__ __forceinline__ void tile_body(const DevTensor &t, int64_t tile, float *__restrict__ v,
                                           const SmallScalars &sc, int *error_word, float *sm, float *sp,
                                           unsigned char *sraw, float *sg, float *sstep, unsigned long long *bar) {
     constexpr int gsz = GD == AM_BF16 ? 2 : 4;
     const int L = static_cast<int>(t.L);
-    const bool short_rows = L <= kSmallMaxL;
-    const int Ls = short_rows ? (L | 1) : L;     // row stride of the widened gradients
+    constexpr bool short_rows = !LONG;           // LONG: L > kSmallMaxL
+    const int Ls = L | 1;                        // row stride of the widened gradients (short blocks only)
     const int per_tile = tile_blocks(L);
     const int64_t b0 = tile * per_tile;
     const int64_t left = t.n_blocks - b0;
@@ -153,26 +156,30 @@ __device__ __forceinline__ void tile_body(const DevTensor &t, int64_t tile, floa
         }
     }
 
-    // gradients, widened and scaled -> rows: block b of the tile at sg[b * Ls ...]
-    for (int i = threadIdx.x; i < lead; i += kThreads) {
-        const int b = tile_div(i, L, magic);
-        sg[b * Ls + (i - b * L)] = tile_raw_at<GD>(sraw, i + shift) * gscale;
-    }
-    for (int i = lead + threadIdx.x * 4; i < lead + nvec; i += kThreads * 4) {
-        const float4 g = lds_g4<GD>(sraw, i + shift);            // (i + shift) is a multiple of four
-        const float x[4] = {g.x, g.y, g.z, g.w};
-        int b = tile_div(i, L, magic), k = i - b * L;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            sg[b * Ls + k] = x[j] * gscale;
-            if (++k == L) { k = 0; ++b; }
+    // element k of the tile's block b, widened and scaled, straight from the gradients as they arrived
+    auto graw = [&](int b, int k) { return tile_raw_at<GD>(sraw, b * L + k + shift) * gscale; };
+    if (short_rows) {
+        // gradients, widened and scaled -> rows: block b of the tile at sg[b * Ls ...]
+        for (int i = threadIdx.x; i < lead; i += kThreads) {
+            const int b = tile_div(i, L, magic);
+            sg[b * Ls + (i - b * L)] = tile_raw_at<GD>(sraw, i + shift) * gscale;
         }
+        for (int i = lead + threadIdx.x * 4; i < lead + nvec; i += kThreads * 4) {
+            const float4 g = lds_g4<GD>(sraw, i + shift);            // (i + shift) is a multiple of four
+            const float x[4] = {g.x, g.y, g.z, g.w};
+            int b = tile_div(i, L, magic), k = i - b * L;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                sg[b * Ls + k] = x[j] * gscale;
+                if (++k == L) { k = 0; ++b; }
+            }
+        }
+        for (int i = lead + nvec + threadIdx.x; i < n; i += kThreads) {
+            const int b = tile_div(i, L, magic);
+            sg[b * Ls + (i - b * L)] = tile_raw_at<GD>(sraw, i + shift) * gscale;
+        }
+        __syncthreads();
     }
-    for (int i = lead + nvec + threadIdx.x; i < n; i += kThreads) {
-        const int b = tile_div(i, L, magic);
-        sg[b * Ls + (i - b * L)] = tile_raw_at<GD>(sraw, i + shift) * gscale;
-    }
-    __syncthreads();
 
     // block statistics, v and the blocks' step sizes
     if (short_rows) {
@@ -206,7 +213,7 @@ __device__ __forceinline__ void tile_body(const DevTensor &t, int64_t tile, floa
         for (int r = 0; r < rounds; ++r) {
             const int b = gid + r * groups;
             const bool live = b < nb;
-            const float *row = sg + (live ? b : 0) * Ls;
+            const int rb = live ? b : 0;
             const float vo = __shfl_sync(0xffffffffu, v_old[0], r, glanes);
             double tot;
             if (sc.statistic == 0 || sc.statistic == 3) {
@@ -214,16 +221,17 @@ __device__ __forceinline__ void tile_body(const DevTensor &t, int64_t tile, floa
                 float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
                 int k = gl;
                 for (; k + 3 * glanes < L; k += 4 * glanes) {
-                    s0 = fmaf(row[k], row[k], s0); s1 = fmaf(row[k + glanes], row[k + glanes], s1);
-                    s2 = fmaf(row[k + 2 * glanes], row[k + 2 * glanes], s2);
-                    s3 = fmaf(row[k + 3 * glanes], row[k + 3 * glanes], s3);
+                    const float x0 = graw(rb, k), x1 = graw(rb, k + glanes);
+                    const float x2 = graw(rb, k + 2 * glanes), x3 = graw(rb, k + 3 * glanes);
+                    s0 = fmaf(x0, x0, s0); s1 = fmaf(x1, x1, s1);
+                    s2 = fmaf(x2, x2, s2); s3 = fmaf(x3, x3, s3);
                 }
-                for (; k < L; k += glanes) s0 = fmaf(row[k], row[k], s0);
+                for (; k < L; k += glanes) { const float x = graw(rb, k); s0 = fmaf(x, x, s0); }
                 tot = (static_cast<double>(s0) + static_cast<double>(s1)) + (static_cast<double>(s2) + static_cast<double>(s3));
                 for (int o = glanes >> 1; o > 0; o >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, o);
             } else {
                 tot = stat_identity(sc.statistic);
-                for (int k = gl; k < L; k += glanes) tot = stat_combine(tot, stat_term(row[k], sc.statistic), sc.statistic);
+                for (int k = gl; k < L; k += glanes) tot = stat_combine(tot, stat_term(graw(rb, k), sc.statistic), sc.statistic);
                 for (int o = glanes >> 1; o > 0; o >>= 1)
                     tot = stat_combine(tot, __shfl_xor_sync(0xffffffffu, tot, o), sc.statistic);
             }
@@ -244,7 +252,6 @@ __device__ __forceinline__ void tile_body(const DevTensor &t, int64_t tile, floa
         const bool plain_sum = sc.statistic == 0 || sc.statistic == 3;
         for (int slot = warp; slot < slots; slot += kThreads / 32) {
             const int b = slot / wpb, sl = slot - b * wpb;
-            const float *row = sg + b * Ls;
             const int k1 = min(L, (sl + 1) * per);
             double tot;
             if (plain_sum) {
@@ -252,15 +259,16 @@ __device__ __forceinline__ void tile_body(const DevTensor &t, int64_t tile, floa
                 float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
                 int k = sl * per + lane;
                 for (; k + 96 < k1; k += 128) {
-                    s0 = fmaf(row[k], row[k], s0); s1 = fmaf(row[k + 32], row[k + 32], s1);
-                    s2 = fmaf(row[k + 64], row[k + 64], s2); s3 = fmaf(row[k + 96], row[k + 96], s3);
+                    const float x0 = graw(b, k), x1 = graw(b, k + 32), x2 = graw(b, k + 64), x3 = graw(b, k + 96);
+                    s0 = fmaf(x0, x0, s0); s1 = fmaf(x1, x1, s1);
+                    s2 = fmaf(x2, x2, s2); s3 = fmaf(x3, x3, s3);
                 }
-                for (; k < k1; k += 32) s0 = fmaf(row[k], row[k], s0);
+                for (; k < k1; k += 32) { const float x = graw(b, k); s0 = fmaf(x, x, s0); }
                 tot = warp_sum((static_cast<double>(s0) + static_cast<double>(s1)) +
                                (static_cast<double>(s2) + static_cast<double>(s3)));
             } else {
                 tot = stat_identity(sc.statistic);
-                for (int k = sl * per + lane; k < k1; k += 32) tot = stat_combine(tot, stat_term(row[k], sc.statistic), sc.statistic);
+                for (int k = sl * per + lane; k < k1; k += 32) tot = stat_combine(tot, stat_term(graw(b, k), sc.statistic), sc.statistic);
                 tot = warp_stat(tot, sc.statistic);
             }
             if (lane == 0) spart[slot] = tot;
@@ -282,7 +290,7 @@ __device__ __forceinline__ void tile_body(const DevTensor &t, int64_t tile, floa
     for (int i = threadIdx.x; i < lead; i += kThreads) {
         const int b = tile_div(i, L, magic);
         float m = sm[i + shift], p = sp[i + shift];
-        update_one(sg[b * Ls + (i - b * L)], m, p, sc.beta1, sc.omb1, lr_wd, sstep[b]);
+        update_one(short_rows ? sg[b * Ls + (i - b * L)] : graw(0, i), m, p, sc.beta1, sc.omb1, lr_wd, sstep[b]);
         mg[i] = m;
         pg[i] = p;
         if (t.p_bf16) store_bf16(t.p_bf16 + e0 + i, p);
@@ -292,9 +300,14 @@ __device__ __forceinline__ void tile_body(const DevTensor &t, int64_t tile, floa
         float4 p = *reinterpret_cast<const float4 *>(sp + i + shift);
         float *mm[4] = {&m.x, &m.y, &m.z, &m.w}, *pp[4] = {&p.x, &p.y, &p.z, &p.w};
         int b = tile_div(i, L, magic), k = i - b * L;
+        float x[4] = {0.f, 0.f, 0.f, 0.f};
+        if (!short_rows) {
+            const float4 g = lds_g4<GD>(sraw, i + shift);            // (i + shift) is a multiple of four
+            x[0] = g.x * gscale; x[1] = g.y * gscale; x[2] = g.z * gscale; x[3] = g.w * gscale;
+        }
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            update_one(sg[b * Ls + k], *mm[j], *pp[j], sc.beta1, sc.omb1, lr_wd, sstep[b]);
+            update_one(short_rows ? sg[b * Ls + k] : x[j], *mm[j], *pp[j], sc.beta1, sc.omb1, lr_wd, sstep[b]);
             if (++k == L) { k = 0; ++b; }
         }
         *reinterpret_cast<float4 *>(mg + i) = m;
@@ -304,7 +317,7 @@ __device__ __forceinline__ void tile_body(const DevTensor &t, int64_t tile, floa
     for (int i = lead + nvec + threadIdx.x; i < n; i += kThreads) {
         const int b = tile_div(i, L, magic);
         float m = sm[i + shift], p = sp[i + shift];
-        update_one(sg[b * Ls + (i - b * L)], m, p, sc.beta1, sc.omb1, lr_wd, sstep[b]);
+        update_one(short_rows ? sg[b * Ls + (i - b * L)] : graw(0, i), m, p, sc.beta1, sc.omb1, lr_wd, sstep[b]);
         mg[i] = m;
         pg[i] = p;
         if (t.p_bf16) store_bf16(t.p_bf16 + e0 + i, p);
@@ -325,8 +338,14 @@ tile_kernel(const DevTensor *__restrict__ tensors, const Seg *__restrict__ segs,
     const int64_t unit = blockIdx.x;
     const Seg seg = segs[find_seg(segs, n_segs, unit)];
     const DevTensor &t = tensors[seg.tensor];
-    if (t.gdtype == AM_BF16) tile_body<AM_BF16>(t, unit - seg.unit_begin, v, sc, error_word, sm, sp, sraw, sg, sstep, bar);
-    else tile_body<AM_F32>(t, unit - seg.unit_begin, v, sc, error_word, sm, sp, sraw, sg, sstep, bar);
+    const int64_t tile = unit - seg.unit_begin;
+    if (t.L > kSmallMaxL) {
+        if (t.gdtype == AM_BF16) tile_body<AM_BF16, true>(t, tile, v, sc, error_word, sm, sp, sraw, sg, sstep, bar);
+        else tile_body<AM_F32, true>(t, tile, v, sc, error_word, sm, sp, sraw, sg, sstep, bar);
+    } else {
+        if (t.gdtype == AM_BF16) tile_body<AM_BF16, false>(t, tile, v, sc, error_word, sm, sp, sraw, sg, sstep, bar);
+        else tile_body<AM_F32, false>(t, tile, v, sc, error_word, sm, sp, sraw, sg, sstep, bar);
+    }
 }
 
 }  // namespace am

@@ -37,6 +37,8 @@ def test_workload_names():
     assert bench.pick_workload("llama2-7b-layers2").numel == 666914816
     assert bench.pick_workload("flat-L128").n_blocks == 1 << 23
     assert bench.pick_workload("flat-L1-n20").numel == 1 << 20
+    rows = bench.pick_workload("rows-bf16-L1001-r64")
+    assert (rows.numel, rows.n_blocks) == (64 * 1001, 64)
     with pytest.raises(SystemExit):
         bench.pick_workload("nope")
 
