@@ -39,8 +39,11 @@ constexpr int kTileMaxBlocks = 1024;     // ... and at most this many blocks
 constexpr int kTileMaxL = 4096;          // longest block the kernel takes
 constexpr int kTileLinear = kTileElems + 8;   // a tile in shared memory, shifted by up to 7 elements
 constexpr int kTileWords = 5120;         // >= blocks * (L | 1) for every L <= kSmallMaxL, and >= kTileLinear
-// shared memory: m, p, the raw gradients, the gradient rows, the step sizes, the mbarrier
-constexpr int kTileSmemBytes = (3 * kTileLinear + kTileWords + kTileMaxBlocks) * 4 + 16;
+// shared memory: m, p, the gradients as they arrive, the step sizes, the mbarrier and, last, the widened
+// gradient rows that only blocks of up to kSmallMaxL elements use: a launch without such blocks leaves
+// them out and fits four CTAs per SM instead of three
+constexpr int kTileSmemLongBytes = (3 * kTileLinear + kTileMaxBlocks) * 4 + 16;
+constexpr int kTileSmemBytes = kTileSmemLongBytes + kTileWords * 4;
 constexpr int kTileTimeoutCode = 7;
 static_assert(kTileWords >= kTileLinear, "long rows are stored unpadded");
 
@@ -327,13 +330,13 @@ __device__ __forceinline__ void tile_body(const DevTensor &t, int64_t tile, floa
 __global__ void __launch_bounds__(kThreads)
 tile_kernel(const DevTensor *__restrict__ tensors, const Seg *__restrict__ segs, int n_segs,
             float *__restrict__ v, SmallScalars sc, int *error_word) {
-    extern __shared__ __align__(128) unsigned char tile_smem[];      // kTileSmemBytes
+    extern __shared__ __align__(128) unsigned char tile_smem[];      // kTileSmemBytes, or kTileSmemLongBytes (no sg)
     float *sm = reinterpret_cast<float *>(tile_smem);
     float *sp = sm + kTileLinear;
     unsigned char *sraw = reinterpret_cast<unsigned char *>(sp + kTileLinear);
-    float *sg = reinterpret_cast<float *>(sraw) + kTileLinear;
-    float *sstep = sg + kTileWords;
+    float *sstep = reinterpret_cast<float *>(sraw) + kTileLinear;
     unsigned long long *bar = reinterpret_cast<unsigned long long *>(sstep + kTileMaxBlocks);
+    float *sg = reinterpret_cast<float *>(bar + 2);
     if (step_skipped(sc.skip_flag)) return;
     const int64_t unit = blockIdx.x;
     const Seg seg = segs[find_seg(segs, n_segs, unit)];
