@@ -240,7 +240,7 @@ typedef enum {
                                   block_len > 16 (correctness anchor: a second implementation of every
                                   other kernel family's work) */
     AM_OPT_STREAM_CTAS    = 1, /* persistent CTAs of the streaming kernel (0 = one per SM) */
-    AM_OPT_CLUSTER_SIZE   = 2, /* CTAs per cluster for head-sized blocks: 1, 2, 4, 8 (0 = chosen by block size) */
+    AM_OPT_CLUSTER_SIZE   = 2, /* CTAs per cluster for head-sized blocks: 1 to 8 (0 = chosen by block size) */
     AM_OPT_STREAM_THREADS = 3, /* threads per consumer group of the streaming kernels, a multiple of 32
                                   from 64 to 512 (0 = default 256); groups x threads is capped at 512 */
     AM_OPT_PROFILE        = 4, /* n > 0: record CUDA events around each kernel family of every step, keeping

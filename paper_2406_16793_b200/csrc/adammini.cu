@@ -355,6 +355,7 @@ int adammini_set_option(am_handle *h, int32_t key, int64_t value) {
         return AM_ERR_INVALID_ARGUMENT;
     if (key == AM_OPT_STATISTIC && value > 4) return AM_ERR_INVALID_ARGUMENT;
     if (key == AM_OPT_STREAM_GROUPS && value > kMaxGroups) return AM_ERR_INVALID_ARGUMENT;
+    if (key == AM_OPT_CLUSTER_SIZE && value > kMaxCluster) return AM_ERR_INVALID_ARGUMENT;
     if (key == AM_OPT_PROFILE) {
         if (value > 4096) return AM_ERR_INVALID_ARGUMENT;
         for (cudaEvent_t e : h->prof_ev) cudaEventDestroy(e);

@@ -489,9 +489,15 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                     bulk_load(st + P.g_region_bytes + kStageElems * 4, t.p + e0, n * 4, &ctl->full[stage]);
                     advance();
                 } else {
-                    // one long block; a cluster splits it evenly over its CTAs
-                    const int64_t slice = t.L / csize;
-                    const int64_t e0 = local * t.L + crank * slice;
+                    // one long block; a cluster splits it evenly over its CTAs where the slices then start
+                    // on 16-byte boundaries, else (cluster sizes that are no power of two) in multiples of 16 elements
+                    int64_t slice = t.L / csize, begin = crank * slice;
+                    if (slice * csize != t.L || slice % (16 / gsz) != 0) {
+                        const int64_t q = t.L / 16;
+                        begin = q * crank / csize * 16;
+                        slice = (crank + 1 == csize ? t.L : q * (crank + 1) / csize * 16) - begin;
+                    }
+                    const int64_t e0 = local * t.L + begin;
                     const int sum_cap = P.stage_bytes / gsz;
                     for (int64_t off = 0; off < slice && ok; off += sum_cap) {
                         const int c = static_cast<int>(slice - off < sum_cap ? slice - off : sum_cap);
@@ -948,18 +954,21 @@ inline void stream_finish_plan(const StreamPlanInput &in, int cluster_size, int 
     if (!in.cluster_tensors.empty() && n_clusters > 0) {
         // Launch shape for head-sized blocks.  Measured on B200: blocks of up to 1 MB of
         // gradients (bf16 heads of 128 x 4096) run best on clusters of 4 that take one block
-        // at a time from the shared counter; larger blocks on clusters of 8 with fixed ranges.
+        // at a time from the shared counter (33 clusters fit), blocks of up to 2 MB (the same
+        // heads with float32 gradients) on clusters of 6 (22 fit) that do the same, larger
+        // blocks on clusters of 8 (15 fit) with fixed ranges: more clusters use more SMs but keep
+        // more gradients in L2 between their two fetches.
         int64_t max_block_bytes = 0;
         for (const auto &it : in.cluster_tensors)
             max_block_bytes = std::max(max_block_bytes, it.row.block_len * (it.row.grad_dtype == AM_BF16 ? 2 : 4));
-        const bool small_blocks = max_block_bytes <= (int64_t(1) << 20);
+        const int preferred = max_block_bytes <= (int64_t(1) << 20) ? 4 : max_block_bytes <= (int64_t(2) << 20) ? 6 : 8;
         int chunk = in.cluster_chunk;
-        if (in.cluster_size == 0 && small_blocks && cluster_size > 4) {
-            int cs4 = 0, n4 = 0;
-            stream_probe_cluster(in.sm_count, threads * groups, 4, &cs4, &n4);
-            if (cs4 == 4 && n4 > 0) { cluster_size = 4; n_clusters = n4; }
+        if (in.cluster_size == 0 && preferred < cluster_size) {
+            int cs = 0, n = 0;
+            stream_probe_cluster(in.sm_count, threads * groups, preferred, &cs, &n);
+            if (cs == preferred && n > 0) { cluster_size = cs; n_clusters = n; }
         }
-        if (chunk == 0) chunk = (in.cluster_size == 0 && !small_blocks) ? kStaticRanges : 1;
+        if (chunk == 0) chunk = (in.cluster_size == 0 && cluster_size == 8) ? kStaticRanges : 1;
         stream_build_launch(in.cluster_tensors, true, n_clusters, &plan->clus);
         plan->clus.grid *= cluster_size;          // bounds are per cluster
         plan->clus.cluster = cluster_size;

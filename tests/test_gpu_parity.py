@@ -106,7 +106,7 @@ def test_consumer_groups_give_identical_bits():
     assert _same(a, dev)
 
 
-@pytest.mark.parametrize("cluster", [1, 2, 4])
+@pytest.mark.parametrize("cluster", [1, 2, 3, 4, 5, 6, 7])
 def test_other_cluster_sizes(cluster):
     w = W.Workload("heads", 77, [W.TensorSpec("q", 1024, 4096, W.HEADS, n_heads=8, grad_dtype=W.BF16)],
                    W.GradRecipe(-5.0, -1.0), steps=3)
@@ -642,3 +642,36 @@ def test_unaligned_block_lengths_up_to_a_tile(grad_dtype):
     for c, p in zip(copies, b.p):
         assert torch.equal(c.view, p.to(torch.bfloat16)) and c.intact()
     oa.close(); ob.close()
+
+
+@pytest.mark.parametrize("grad_dtype", [W.F32, W.BF16], ids=["f32", "bf16"])
+def test_long_unaligned_blocks_alone_and_beside_short_ones(grad_dtype):
+    """The tile kernel is launched with less shared memory when no tile holds blocks
+    of up to 64 elements.  Rows of more than 64 elements must come out bit for bit
+    the same from such a launch and from one that also holds short blocks, with a
+    gradient scale as well (long blocks apply it while reading the staged gradients),
+    and both must match the oracle."""
+    long_rows = [W.TensorSpec(f"l{L}", 3 * (4096 // L) + 2, L, W.ROWS, grad_dtype=grad_dtype) for L in (67, 255, 1001, 4095)]
+    short_rows = [W.TensorSpec("s7", 2051, 7, W.ROWS, grad_dtype=grad_dtype)]
+    alone = W.Workload("long-alone", 95 + grad_dtype, long_rows, W.GradRecipe(-4.0, -1.0), steps=3)
+    mixed = W.Workload("long-alone", 95 + grad_dtype, long_rows + short_rows, W.GradRecipe(-4.0, -1.0), steps=3)
+    H.assert_parity(H.run_parity(alone))
+    H.assert_parity(H.run_parity(mixed))
+    for scale in (None, 0.25):
+        a, b = H.DeviceState(alone), H.DeviceState(mixed)
+        oa, ob = H.make_optimizer(alone), H.make_optimizer(mixed)
+        for step in (1, 2):
+            a.draw_grads(step); b.draw_grads(step)
+            for i in range(len(long_rows)):
+                assert torch.equal(a.g[i], b.g[i]) and (step > 1 or torch.equal(a.p[i], b.p[i]))
+            if scale is None:
+                oa.step(a.p, a.g, a.m, a.v, step); ob.step(b.p, b.g, b.m, b.v, step)
+            else:
+                oa.step_ex(a.p, a.g, a.m, a.v, step, grad_scale=scale); ob.step_ex(b.p, b.g, b.m, b.v, step, grad_scale=scale)
+        oa.sync_status(); ob.sync_status()
+        n_long = sum(t.n_blocks for t in long_rows)
+        for i in range(len(long_rows)):
+            assert torch.equal(a.p[i], b.p[i]) and torch.equal(a.m[i], b.m[i])
+        assert torch.equal(a.v[:n_long], b.v[:n_long])
+        assert a.guards_intact() and b.guards_intact()
+        oa.close(); ob.close()
