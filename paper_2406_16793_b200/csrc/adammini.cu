@@ -204,9 +204,9 @@ int build_plan(am_handle *h) {
     h->d_tile_segs = reinterpret_cast<Seg *>(base + o_tile);
     h->n_tile_segs = static_cast<int>(tile_segs.size());
     h->tile_units = tile_units;
-    h->tile_short = false;
+    h->tile_short = h->tile_long = false;
     for (const Seg &sg : tile_segs)
-        if (h->rows[sg.tensor].block_len <= kSmallMaxL) h->tile_short = true;
+        (h->rows[sg.tensor].block_len <= kSmallMaxL ? h->tile_short : h->tile_long) = true;
     h->d_piece_segs = reinterpret_cast<Seg *>(base + o_piece);
     h->d_block_segs = reinterpret_cast<Seg *>(base + o_block);
     h->d_partials = reinterpret_cast<double *>(base + o_partials);
@@ -490,9 +490,10 @@ int adammini_step_ex(am_handle *h, void *const *params, const void *const *grads
             AM_CUDA(h, cudaGetLastError());
         }
         if (h->tile_units) {
-            tile_kernel<<<static_cast<unsigned>(h->tile_units), kThreads,
-                          h->tile_short ? kTileSmemBytes : kTileSmemLongBytes, stream>>>(
-                h->d_tensors, h->d_tile_segs, h->n_tile_segs, v, ss, h->error_word);
+            const int tile_smem = !h->tile_short ? kTileSmemLongBytes : h->tile_long ? kTileSmemBytes : kTileSmemShortBytes;
+            tile_kernel<<<static_cast<unsigned>(h->tile_units), kThreads, tile_smem, stream>>>(
+                h->d_tensors, h->d_tile_segs, h->n_tile_segs, v, ss, h->error_word,
+                h->tile_long ? kTileLinear : kTileShortLinear);
             AM_CUDA(h, cudaGetLastError());
         }
     }

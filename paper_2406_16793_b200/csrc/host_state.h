@@ -34,6 +34,7 @@ struct am_handle {
     int n_tile_segs = 0;
     int64_t tile_units = 0;
     bool tile_short = false;             // some tile holds blocks of up to kSmallMaxL elements (they need the widened rows)
+    bool tile_long = false;              // some tile holds longer blocks (they need the longer linear arrays)
     am::Seg *d_wide_segs = nullptr;      // two-pass tensors whose blocks have many partial sums
     int n_wide_segs = 0;
     int64_t wide_units = 0;

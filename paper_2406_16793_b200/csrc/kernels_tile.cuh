@@ -34,24 +34,27 @@
 
 namespace am {
 
-constexpr int kTileElems = 4096;         // elements per tile ...
-constexpr int kTileMaxBlocks = 1024;     // ... and at most this many blocks
+constexpr int kTileElems = 4096;         // elements per tile of blocks longer than kSmallMaxL ...
+constexpr int kTileShortElems = 3072;    // ... and of shorter ones,
+constexpr int kTileMaxBlocks = 1024;     // with at most this many blocks
 constexpr int kTileMaxL = 4096;          // longest block the kernel takes
-constexpr int kTileLinear = kTileElems + 8;   // a tile in shared memory, shifted by up to 7 elements
-constexpr int kTileWords = 5120;         // >= blocks * (L | 1) for every L <= kSmallMaxL, and >= kTileLinear
-// shared memory: m, p, the gradients as they arrive, the step sizes, the mbarrier and, last, the widened
-// gradient rows that only blocks of up to kSmallMaxL elements use: a launch without such blocks leaves
-// them out and fits four CTAs per SM instead of three
+constexpr int kTileLinear = kTileElems + 8;            // a tile in shared memory, shifted by up to 7 elements
+constexpr int kTileShortLinear = kTileShortElems + 8;
+constexpr int kTileWords = 3840;         // >= blocks * (L | 1) for every tile of blocks of up to kSmallMaxL elements
+// Shared memory: m, p and the gradients as they arrive (`linear` words each), the step sizes, the
+// mbarrier and, last, the widened gradient rows that only blocks of up to kSmallMaxL elements use.
+// A launch with only long or only short blocks takes what those need and fits four CTAs per SM;
+// a mixed one takes the larger of each part and fits three.
 constexpr int kTileSmemLongBytes = (3 * kTileLinear + kTileMaxBlocks) * 4 + 16;
+constexpr int kTileSmemShortBytes = (3 * kTileShortLinear + kTileMaxBlocks + kTileWords) * 4 + 16;
 constexpr int kTileSmemBytes = kTileSmemLongBytes + kTileWords * 4;
 constexpr int kTileTimeoutCode = 7;
-static_assert(kTileWords >= kTileLinear, "long rows are stored unpadded");
 
 // Blocks per tile.  Short blocks: a multiple of eight, so that every tile starts
 // on a 32-byte boundary; longer ones: as many as fit.
 __host__ __device__ inline int tile_blocks(int64_t L) {
-    int64_t nb = kTileElems / L;
-    if (L > kSmallMaxL) return static_cast<int>(nb < 1 ? 1 : nb);
+    if (L > kSmallMaxL) return static_cast<int>(kTileElems / L < 1 ? 1 : kTileElems / L);
+    int64_t nb = kTileShortElems / L;
     if (nb > kTileMaxBlocks) nb = kTileMaxBlocks;
     return static_cast<int>(nb & ~int64_t(7));
 }
@@ -329,12 +332,13 @@ __device__ __forceinline__ void tile_body(const DevTensor &t, int64_t tile, floa
 
 __global__ void __launch_bounds__(kThreads)
 tile_kernel(const DevTensor *__restrict__ tensors, const Seg *__restrict__ segs, int n_segs,
-            float *__restrict__ v, SmallScalars sc, int *error_word) {
-    extern __shared__ __align__(128) unsigned char tile_smem[];      // kTileSmemBytes, or kTileSmemLongBytes (no sg)
+            float *__restrict__ v, SmallScalars sc, int *error_word, int linear) {
+    // linear: kTileLinear (with kTileSmemBytes, or kTileSmemLongBytes and no sg) or kTileShortLinear (kTileSmemShortBytes)
+    extern __shared__ __align__(128) unsigned char tile_smem[];
     float *sm = reinterpret_cast<float *>(tile_smem);
-    float *sp = sm + kTileLinear;
-    unsigned char *sraw = reinterpret_cast<unsigned char *>(sp + kTileLinear);
-    float *sstep = reinterpret_cast<float *>(sraw) + kTileLinear;
+    float *sp = sm + linear;
+    unsigned char *sraw = reinterpret_cast<unsigned char *>(sp + linear);
+    float *sstep = reinterpret_cast<float *>(sraw) + linear;
     unsigned long long *bar = reinterpret_cast<unsigned long long *>(sstep + kTileMaxBlocks);
     float *sg = reinterpret_cast<float *>(bar + 2);
     if (step_skipped(sc.skip_flag)) return;
