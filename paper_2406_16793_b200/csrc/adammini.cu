@@ -175,6 +175,25 @@ int build_plan(am_handle *h) {
         }
     }
     if (part_units > 0x7fffffffLL || wide_units > 0x7fffffffLL) return AM_ERR_TOO_LARGE;
+    // Tiles of short blocks first, then those of longer ones: the two kinds are launched
+    // separately, each with the shared-memory layout it needs (four CTAs per SM for both).
+    int64_t tile_short_units = 0;
+    {
+        std::vector<Seg> ordered;
+        int64_t next = 0;
+        for (int pass = 0; pass < 2; ++pass) {
+            for (const Seg &sg : tile_segs) {
+                const am_table_row &r = h->rows[sg.tensor];
+                if ((r.block_len <= kSmallMaxL) != (pass == 0)) continue;
+                Seg o = sg;
+                o.unit_begin = next;
+                next += ceil_div(r.n_blocks, tile_blocks(r.block_len));
+                ordered.push_back(o);
+            }
+            if (pass == 0) tile_short_units = next;
+        }
+        tile_segs.swap(ordered);
+    }
     if (small_units > 0x7fffffffLL || tile_units > 0x7fffffffLL || piece_units > 0x7fffffffLL || ceil_div(block_units, kThreads / 32) > 0x7fffffffLL)
         return AM_ERR_TOO_LARGE;
 
@@ -204,9 +223,7 @@ int build_plan(am_handle *h) {
     h->d_tile_segs = reinterpret_cast<Seg *>(base + o_tile);
     h->n_tile_segs = static_cast<int>(tile_segs.size());
     h->tile_units = tile_units;
-    h->tile_short = h->tile_long = false;
-    for (const Seg &sg : tile_segs)
-        (h->rows[sg.tensor].block_len <= kSmallMaxL ? h->tile_short : h->tile_long) = true;
+    h->tile_short_units = tile_short_units;
     h->d_piece_segs = reinterpret_cast<Seg *>(base + o_piece);
     h->d_block_segs = reinterpret_cast<Seg *>(base + o_block);
     h->d_partials = reinterpret_cast<double *>(base + o_partials);
@@ -243,7 +260,7 @@ int build_plan(am_handle *h) {
         if (e != cudaSuccess) return cuda_fail(h, e);
     }
 
-    h->launches = (small_units ? 1 : 0) + (tile_units ? 1 : 0) + (piece_units ? 3 : 0) + (wide_units ? 1 : 0) + sp.launches();
+    h->launches = (small_units ? 1 : 0) + (tile_short_units ? 1 : 0) + (tile_units > tile_short_units ? 1 : 0) + (piece_units ? 3 : 0) + (wide_units ? 1 : 0) + sp.launches();
     h->planned = true;
     return AM_OK;
 }
@@ -490,11 +507,17 @@ int adammini_step_ex(am_handle *h, void *const *params, const void *const *grads
             AM_CUDA(h, cudaGetLastError());
         }
         if (h->tile_units) {
-            const int tile_smem = !h->tile_short ? kTileSmemLongBytes : h->tile_long ? kTileSmemBytes : kTileSmemShortBytes;
-            tile_kernel<<<static_cast<unsigned>(h->tile_units), kThreads, tile_smem, stream>>>(
-                h->d_tensors, h->d_tile_segs, h->n_tile_segs, v, ss, h->error_word,
-                h->tile_long ? kTileLinear : kTileShortLinear);
-            AM_CUDA(h, cudaGetLastError());
+            const int64_t n_short = h->tile_short_units, n_long = h->tile_units - n_short;
+            if (n_short) {
+                tile_kernel<<<static_cast<unsigned>(n_short), kThreads, kTileSmemShortBytes, stream>>>(
+                    h->d_tensors, h->d_tile_segs, h->n_tile_segs, v, ss, h->error_word, kTileShortLinear, 0);
+                AM_CUDA(h, cudaGetLastError());
+            }
+            if (n_long) {
+                tile_kernel<<<static_cast<unsigned>(n_long), kThreads, kTileSmemLongBytes, stream>>>(
+                    h->d_tensors, h->d_tile_segs, h->n_tile_segs, v, ss, h->error_word, kTileLinear, n_short);
+                AM_CUDA(h, cudaGetLastError());
+            }
         }
     }
     h->stream.bf16_copies = ex && ex->params_bf16;

@@ -33,8 +33,7 @@ struct am_handle {
     am::Seg *d_tile_segs = nullptr;      // short blocks handled a tile at a time
     int n_tile_segs = 0;
     int64_t tile_units = 0;
-    bool tile_short = false;             // some tile holds blocks of up to kSmallMaxL elements (they need the widened rows)
-    bool tile_long = false;              // some tile holds longer blocks (they need the longer linear arrays)
+    int64_t tile_short_units = 0;        // the first so many tiles hold blocks of up to kSmallMaxL elements, the rest longer ones
     am::Seg *d_wide_segs = nullptr;      // two-pass tensors whose blocks have many partial sums
     int n_wide_segs = 0;
     int64_t wide_units = 0;

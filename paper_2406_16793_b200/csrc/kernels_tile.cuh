@@ -43,11 +43,11 @@ constexpr int kTileShortLinear = kTileShortElems + 8;
 constexpr int kTileWords = 3840;         // >= blocks * (L | 1) for every tile of blocks of up to kSmallMaxL elements
 // Shared memory: m, p and the gradients as they arrive (`linear` words each), the step sizes, the
 // mbarrier and, last, the widened gradient rows that only blocks of up to kSmallMaxL elements use.
-// A launch with only long or only short blocks takes what those need and fits four CTAs per SM;
-// a mixed one takes the larger of each part and fits three.
+// Tiles of short and of longer blocks are launched separately, each kind with what it needs, so
+// that four CTAs fit an SM.
 constexpr int kTileSmemLongBytes = (3 * kTileLinear + kTileMaxBlocks) * 4 + 16;
 constexpr int kTileSmemShortBytes = (3 * kTileShortLinear + kTileMaxBlocks + kTileWords) * 4 + 16;
-constexpr int kTileSmemBytes = kTileSmemLongBytes + kTileWords * 4;
+constexpr int kTileSmemBytes = kTileSmemShortBytes > kTileSmemLongBytes ? kTileSmemShortBytes : kTileSmemLongBytes;
 constexpr int kTileTimeoutCode = 7;
 
 // Blocks per tile.  Short blocks: a multiple of eight, so that every tile starts
@@ -332,8 +332,9 @@ __device__ __forceinline__ void tile_body(const DevTensor &t, int64_t tile, floa
 
 __global__ void __launch_bounds__(kThreads)
 tile_kernel(const DevTensor *__restrict__ tensors, const Seg *__restrict__ segs, int n_segs,
-            float *__restrict__ v, SmallScalars sc, int *error_word, int linear) {
-    // linear: kTileLinear (with kTileSmemBytes, or kTileSmemLongBytes and no sg) or kTileShortLinear (kTileSmemShortBytes)
+            float *__restrict__ v, SmallScalars sc, int *error_word, int linear, int64_t first_unit) {
+    // linear: kTileLinear (kTileSmemLongBytes, no sg) or kTileShortLinear (kTileSmemShortBytes); the grid covers
+    // the tiles from first_unit on
     extern __shared__ __align__(128) unsigned char tile_smem[];
     float *sm = reinterpret_cast<float *>(tile_smem);
     float *sp = sm + linear;
@@ -342,7 +343,7 @@ tile_kernel(const DevTensor *__restrict__ tensors, const Seg *__restrict__ segs,
     unsigned long long *bar = reinterpret_cast<unsigned long long *>(sstep + kTileMaxBlocks);
     float *sg = reinterpret_cast<float *>(bar + 2);
     if (step_skipped(sc.skip_flag)) return;
-    const int64_t unit = blockIdx.x;
+    const int64_t unit = first_unit + blockIdx.x;
     const Seg seg = segs[find_seg(segs, n_segs, unit)];
     const DevTensor &t = tensors[seg.tensor];
     const int64_t tile = unit - seg.unit_begin;

@@ -646,11 +646,11 @@ def test_unaligned_block_lengths_up_to_a_tile(grad_dtype):
 
 @pytest.mark.parametrize("grad_dtype", [W.F32, W.BF16], ids=["f32", "bf16"])
 def test_long_unaligned_blocks_alone_and_beside_short_ones(grad_dtype):
-    """The tile kernel is launched with less shared memory when no tile holds blocks
-    of up to 64 elements.  Rows of more than 64 elements must come out bit for bit
-    the same from such a launch and from one that also holds short blocks, with a
-    gradient scale as well (long blocks apply it while reading the staged gradients),
-    and both must match the oracle."""
+    """Tiles of blocks of up to 64 elements and tiles of longer blocks are launched
+    separately, each with its own shared-memory layout.  Rows of more than 64 elements
+    must come out bit for bit the same from a table of their own and from one that
+    also holds short blocks, with a gradient scale as well (long blocks apply it while
+    reading the staged gradients), and both must match the oracle."""
     long_rows = [W.TensorSpec(f"l{L}", 3 * (4096 // L) + 2, L, W.ROWS, grad_dtype=grad_dtype) for L in (67, 255, 1001, 4095)]
     short_rows = [W.TensorSpec("s7", 2051, 7, W.ROWS, grad_dtype=grad_dtype)]
     alone = W.Workload("long-alone", 95 + grad_dtype, long_rows, W.GradRecipe(-4.0, -1.0), steps=3)
@@ -660,6 +660,7 @@ def test_long_unaligned_blocks_alone_and_beside_short_ones(grad_dtype):
     for scale in (None, 0.25):
         a, b = H.DeviceState(alone), H.DeviceState(mixed)
         oa, ob = H.make_optimizer(alone), H.make_optimizer(mixed)
+        assert (oa.query(B.Q_LAUNCHES_PER_STEP), ob.query(B.Q_LAUNCHES_PER_STEP)) == (1, 2)
         for step in (1, 2):
             a.draw_grads(step); b.draw_grads(step)
             for i in range(len(long_rows)):
