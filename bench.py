@@ -9,6 +9,9 @@ parameters, bf16 gradients, fp32 master parameters and moments).  One JSON
 line is printed by rank 0.  With N > 1 (launched by torch.distributed.run)
 every rank steps its own Llama-2-7B-sized shard of a model N times larger:
 blocks are independent, so the step needs no collective (weak scaling).
+`--shard blocks` / `--shard flat` make the ranks share ONE table instead
+(whole-block shards without a collective / flat shards whose cut blocks get
+their sums through one all-gather per step): strong scaling.
 
 `--impl reference` times the float64 CPU checker from oracle/ on the host
 cores, on a bounded sample of the same workload.
@@ -33,29 +36,51 @@ if ROOT not in sys.path:
 METRIC = "adam_mini_step_throughput"
 UNIT = "Gparams/s"
 
-# DRAM traffic of the streaming kernel from the ncu capture summarised under
-# profiles/ (dram__bytes_read.sum + dram__bytes_write.sum per parameter), valid
-# only for the kernel sources with this digest.
-NCU_TRAFFIC = {"digest": "b54ab5e4dc5f67f5", "bytes_per_param": 17.91}
+NOMINAL_HBM_GBS = 8000.0      # HBM3e of a B200, nominal (quoted beside the measured-peak fraction)
+
+# DRAM traffic per parameter (dram__bytes_read.sum + dram__bytes_write.sum) of each kernel
+# family from the ncu captures summarised under profiles/.  An entry counts only while the
+# sources its kernel is compiled from still have the digest they had at the capture.
+NCU_TRAFFIC = [
+    {"family": "stream_kernel<false>", "grad": "bf16", "sources": "stream", "digest": "b54ab5e4dc5f67f5",
+     "bytes_per_param": 17.91, "elements_query": lambda B: B.Q_ELEMENTS_STREAM,
+     "capture": "profiles/stream_kernel_llama2_7b.md (2-layer case, scaled by parameters)"},
+    {"family": "stream_kernel<true>", "grad": "bf16", "sources": "stream", "digest": "b54ab5e4dc5f67f5",
+     "bytes_per_param": 17.41, "elements_query": lambda B: B.Q_ELEMENTS_CLUSTER,
+     "capture": "profiles/stream_kernel_llama2_7b.md (2-layer case, scaled by parameters)"},
+]
+
+
+def _stripped(text: str) -> bytes:
+    import re
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    text = re.sub(r"//[^\n]*", "", text)
+    return "".join(text.split()).encode()
+
+
+def kernel_digests() -> dict:
+    """Digests of the sources each kernel family is compiled from, comments and
+    whitespace removed: "stream" = the shared device helpers at the top of
+    kernels_basic.cuh + the device code of kernels_stream.cuh; "tile" = those +
+    kernels_tile.cuh; "basic" = all of kernels_basic.cuh (one-element blocks, two-pass)."""
+    csrc = os.path.join(ROOT, "paper_2406_16793_b200", "csrc")
+    basic = open(os.path.join(csrc, "kernels_basic.cuh")).read()
+    stream = open(os.path.join(csrc, "kernels_stream.cuh")).read()
+    tile = open(os.path.join(csrc, "kernels_tile.cuh")).read()
+    helpers = basic[:basic.index("// Short blocks (L <= 64)")]
+    stream_dev = stream[:stream.index("host-side planning")]
+    out = {}
+    for name, parts in (("stream", (helpers, stream_dev)), ("tile", (helpers, stream_dev, tile)), ("basic", (basic,))):
+        h = hashlib.sha256()
+        for part in parts:
+            h.update(_stripped(part))
+        out[name] = h.hexdigest()[:16]
+    return out
 
 
 def kernel_digest() -> str:
-    """Digest of the sources the streaming kernel is compiled from (its own file
-    and the shared device helpers at the top of kernels_basic.cuh), with
-    comments and whitespace removed."""
-    import re
-    h = hashlib.sha256()
-    csrc = os.path.join(ROOT, "paper_2406_16793_b200", "csrc")
-    for name in ("kernels_basic.cuh", "kernels_stream.cuh"):
-        text = open(os.path.join(csrc, name)).read()
-        if name == "kernels_basic.cuh":
-            text = text[:text.index("// Short blocks (L <= 64)")]
-        else:
-            text = text[:text.index("host-side planning")]          # device code only
-        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-        text = re.sub(r"//[^\n]*", "", text)
-        h.update("".join(text.split()).encode())
-    return h.hexdigest()[:16]
+    """Digest of the streaming kernel's sources."""
+    return kernel_digests()["stream"]
 
 
 def measured_peak_gbs():
@@ -191,11 +216,90 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+class PlainJob:
+    """The whole table on this GPU: one handle, adammini_step."""
+
+    def __init__(self, w, dev, world, rank):
+        import torch
+        import paper_2406_16793_b200 as am
+        from paper_2406_16793_b200 import workloads as W
+        n_t = len(w.tensors)
+        self.specs = list(w.tensors)
+        self.p = [W.gen_param(w, i, dev) for i in range(n_t)]
+        self.m = [torch.zeros_like(x) for x in self.p]
+        self.g = [W.gen_grad(w, i, 1, dev) for i in range(n_t)]
+        self.part = am.Partition(w.tensors)
+        self.v = torch.zeros(max(self.part.total_blocks, 1), dtype=torch.float32, device=dev)
+        self.opt = am.AdamMini(self.part, **w.hparams)
+        self.numel = w.numel                      # parameters this rank steps
+        self.extra_launches = 0
+
+    def step(self, t):
+        self.opt.step(self.p, self.g, self.m, self.v, t)
+
+
+class ShardedJob:
+    """This rank's share of ONE table that all ranks step together (strong scaling).
+    `blocks`: contiguous runs of whole blocks, no collective.  `flat`: equal ranges of
+    the flat parameter space; blocks cut by a range boundary get their sum of g*g through
+    one all-gather of part sums per step, inside the timed region."""
+
+    def __init__(self, w, dev, world, rank, mode):
+        import torch
+        from paper_2406_16793_b200 import sharding, workloads as W
+        self.mode = mode
+        if mode == "blocks":
+            self.sh = sharding.ShardedStep(w.tensors, world, rank, **w.hparams)
+        else:
+            self.sh = sharding.ShardedFlatStep(w.tensors, world, rank, device=dev, **w.hparams)
+            self.exchange = sharding.all_gather_exchange if world > 1 else (lambda local: local.unsqueeze(0))
+        self.opt, self.specs = self.sh.optimizer, self.sh.specs
+        self.p, self.m, self.g = [], [], []
+        cache = {}
+        for piece in self.sh.pieces:              # this rank's slices of the full tensors' seeded inputs
+            if piece.tensor not in cache:
+                cache.clear()
+                cache[piece.tensor] = (W.gen_param(w, piece.tensor, dev), W.gen_grad(w, piece.tensor, 1, dev))
+            fp, fg = cache[piece.tensor]
+            self.p.append(fp[piece.elem_begin:piece.elem_end].clone())
+            self.g.append(fg[piece.elem_begin:piece.elem_end].clone())
+            self.m.append(torch.zeros_like(self.p[-1]))
+        cache.clear()
+        self.v = torch.zeros(max(self.sh.local_blocks, 1), dtype=torch.float32, device=dev)
+        self.numel = sum(x.numel() for x in self.p)
+        # flat: two kernels for the part sums when this rank holds parts (torch's tiny index/copy kernels are not counted)
+        self.extra_launches = 2 if mode == "flat" and self.sh.n_parts else 0
+
+    def step(self, t):
+        if self.mode == "blocks":
+            self.sh.step_local(self.p, self.g, self.m, self.v, t)
+        else:
+            self.sh.step_local(self.p, self.g, self.m, self.v, t, self.exchange)
+
+
+def ncu_traffic(family: str, job, B):
+    """DRAM bytes per launch of the dominant kernel family from the ncu captures
+    summarised under profiles/, scaled by the parameters the family processes; None
+    when the kernel sources have changed since the capture or no capture matches."""
+    digests = kernel_digests()
+    bf16 = all(t.grad_dtype == 1 for t in job.specs)
+    f32 = all(t.grad_dtype == 0 for t in job.specs)
+    unit_blocks = all(t.block_len == 1 for t in job.specs)
+    for e in NCU_TRAFFIC:
+        if e["family"] != family or digests.get(e["sources"]) != e["digest"]:
+            continue
+        if (e["grad"] == "bf16" and not bf16) or (e["grad"] == "f32" and not f32):
+            continue
+        if e.get("unit_blocks") is not None and e["unit_blocks"] != unit_blocks:
+            continue
+        return e["bytes_per_param"] * job.opt.query(e["elements_query"](B)), e["capture"]
+    return None, None
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
     from paper_2406_16793_b200 import build as lib_build
-    import paper_2406_16793_b200 as am
     from paper_2406_16793_b200 import binding as B, workloads as W
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -213,26 +317,21 @@ def run_ours(args):
         dist.barrier()
 
     w = pick_workload(args.workload)
-    n_t = len(w.tensors)
-    p = [W.gen_param(w, i, dev) for i in range(n_t)]
-    m = [torch.zeros_like(x) for x in p]
-    g = [W.gen_grad(w, i, 1, dev) for i in range(n_t)]
-    part = am.Partition(w.tensors)
-    v = torch.zeros(max(part.total_blocks, 1), dtype=torch.float32, device=dev)
-    opt = am.AdamMini(part, **w.hparams)
+    job = PlainJob(w, dev, world, rank) if args.shard == "none" else ShardedJob(w, dev, world, rank, args.shard)
+    opt = job.opt
     for key, val in ((B.OPT_STREAM_THREADS, args.stream_threads), (B.OPT_STREAM_CTAS, args.stream_ctas),
                      (B.OPT_CLUSTER_SIZE, args.cluster_size), (B.OPT_PATH, args.path),
                      (B.OPT_STREAM_CHUNK, args.stream_chunk), (B.OPT_CLUSTER_CHUNK, args.cluster_chunk),
-                     (B.OPT_STREAM_GROUPS, args.stream_groups)):
+                     (B.OPT_STREAM_GROUPS, args.stream_groups), (B.OPT_STATISTIC, args.statistic)):
         if val:
             opt.set_option(key, val)
-    launches = opt.query(B.Q_LAUNCHES_PER_STEP)
+    launches = opt.query(B.Q_LAUNCHES_PER_STEP) + job.extra_launches
     alg_bytes = opt.query(B.Q_ALGORITHMIC_BYTES)
 
     t = 0
     for _ in range(args.warmup):
         t += 1
-        opt.step(p, g, m, v, t)
+        job.step(t)
     opt.sync_status()
 
     def barrier():
@@ -251,7 +350,7 @@ def run_ours(args):
     e0.record()
     for _ in range(args.steps):
         t += 1
-        opt.step(p, g, m, v, t)
+        job.step(t)
     e1.record()
     barrier()
     ms_total = e0.elapsed_time(e1)
@@ -262,7 +361,9 @@ def run_ours(args):
         dist.all_reduce(tt, op=dist.ReduceOp.MAX)
         ms_total = float(tt.item())
     ms_step = ms_total / args.steps
-    value = world * w.numel / (ms_step * 1e-3) / 1e9
+    # whole-job throughput: the parameters all ranks stepped (replicas: world x the table; shards: the table once)
+    total_params = world * w.numel if args.shard == "none" else w.numel
+    value = total_params / (ms_step * 1e-3) / 1e9
     fam_ms, prof_steps = opt.get_profile()
     opt.set_option(B.OPT_PROFILE, 0)
     fam_bytes = [opt.query(q) for q in (B.Q_BYTES_SMALL, B.Q_BYTES_STREAM, B.Q_BYTES_CLUSTER, B.Q_BYTES_TWOPASS)]
@@ -275,45 +376,55 @@ def run_ours(args):
                             "frac": by / (ms_k * 1e-3) / 1e9 / peak}
     top = max(range(4), key=lambda k: fam_ms[k] if fam_bytes[k] else -1.0)
     achieved = fam_bytes[top] / (fam_ms[top] * 1e-3) / 1e9
-    traffic = None
-    if NCU_TRAFFIC["digest"] == kernel_digest() and NCU_TRAFFIC["bytes_per_param"] and top == 1:
-        traffic = NCU_TRAFFIC["bytes_per_param"] * opt.query(B.Q_ELEMENTS_STREAM)
+    traffic, capture = ncu_traffic(fam_names[top], job, B)
+    whole_gbs = alg_bytes / (ms_step * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": fam_names[top], "achieved": achieved, "peak": peak,
                 "peak_source": f"{peak_kind} copy bandwidth", "unit": "GB/s", "frac": achieved / peak,
-                "traffic": traffic, "algorithmic_bytes_per_launch": fam_bytes[top],
-                "whole_step_gbs": alg_bytes / (ms_step * 1e-3) / 1e9,
-                "whole_step_frac": alg_bytes / (ms_step * 1e-3) / 1e9 / peak}
+                "frac_of_nominal": achieved / NOMINAL_HBM_GBS, "nominal_peak": NOMINAL_HBM_GBS,
+                "traffic": traffic, "traffic_capture": capture, "algorithmic_bytes_per_launch": fam_bytes[top],
+                "whole_step_gbs": whole_gbs, "whole_step_frac": whole_gbs / peak,
+                "whole_step_frac_of_nominal": whole_gbs / NOMINAL_HBM_GBS}
 
     e2e = None
     if not args.no_e2e:
-        e2e = run_e2e(args, opt, w, world, dev, p, g, m, v)
+        if args.shard == "flat" and opt.query(B.Q_PART_TENSORS) > 0:
+            e2e = {"value": None, "unit": UNIT, "skipped": "this rank holds parts of cut blocks: the host-buffer step has no exchange"}
+        else:
+            e2e = run_e2e(args, opt, job.specs, total_params / world, world, dev, job.p, job.g, job.m, job.v, w.name)
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu_baseline = oracle_sample(w)[0]
 
     if rank == 0:
+        parallelism = {"none": f"dp{world} (independent replicas of the table, no collective)",
+                       "blocks": f"dp{world} (whole-block shards of one table, no collective)",
+                       "flat": f"dp{world} (flat shards of one table, one all-gather of part sums per step)"}[args.shard]
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "weak" if args.shard == "none" else "strong",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": w.name, "params": w.numel, "blocks": w.n_blocks, "tensors": n_t,
+            "config": {"workload": w.name, "params": w.numel, "blocks": w.n_blocks, "tensors": len(w.tensors),
                        "grad_dtype": "bf16" if w.tensors[0].grad_dtype == W.BF16 else "f32",
                        "l2": "inputs larger than L2 (no flush needed)" if alg_bytes > (1 << 29) else "inputs fit L2",
-                       "parallelism": f"dp{world} (independent shards, no collective)"},
+                       "shard": args.shard, "statistic": args.statistic, "parallelism": parallelism},
             "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu_baseline, "e2e": e2e,
             "gpu_launches": launches * args.steps, "clocks": clocks,
             "gpu": {"name": props.name, "uuid_tail": str(getattr(props, "uuid", ""))[-8:]},
             "stream_ctas": opt.query(B.Q_STREAM_CTAS), "cluster": [opt.query(B.Q_CLUSTER_COUNT), opt.query(B.Q_CLUSTER_SIZE)],
         }
         print(json.dumps(line), flush=True)
-    opt.close()
+    if args.shard == "none":
+        opt.close()
+    else:
+        job.sh.close()
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
 
 
-def run_e2e(args, opt, w, world, dev, p, g, m, v):
+def run_e2e(args, opt, specs, params_per_rank, world, dev, p, g, m, v, workload_name):
     """The same step through adammini_step_host: parameters, moments, v and
     gradients in pinned host memory; host->device and device->host copies are
     inside the timed region (CUDA events cannot bracket a call that blocks on
@@ -321,7 +432,7 @@ def run_e2e(args, opt, w, world, dev, p, g, m, v):
     the blocking C call, max over ranks)."""
     import torch
     import torch.distributed as dist
-    need = sum(t.numel * (8 + (2 if t.grad_dtype else 4)) for t in w.tensors)
+    need = sum(t.numel * (8 + (2 if t.grad_dtype else 4)) for t in specs)
     avail = 0
     for line in open("/proc/meminfo"):
         if line.startswith("MemAvailable"):
@@ -354,9 +465,9 @@ def run_e2e(args, opt, w, world, dev, p, g, m, v):
         tt = torch.tensor([dt], device=dev, dtype=torch.float64)
         dist.all_reduce(tt, op=dist.ReduceOp.MAX)
         dt = float(tt.item())
-    return {"value": world * w.numel * steps / dt / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
+    return {"value": world * params_per_rank * steps / dt / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
             "d2h_bytes_per_step": d2h, "ms_per_step": 1e3 * dt / steps, "steps": steps,
-            "h2d_plus_d2h_gbs": (h2d + d2h) * steps / dt / 1e9, "workload": w.name,
+            "h2d_plus_d2h_gbs": (h2d + d2h) * steps / dt / 1e9, "workload": workload_name,
             "api": "adammini_step_host (pinned host buffers, 3 staging slots)"}
 
 
@@ -374,6 +485,10 @@ def main():
     ap.add_argument("--stream-chunk", type=int, default=0, help="items per grab from the shared work counter (0 = automatic, 1000000 = static ranges)")
     ap.add_argument("--cluster-chunk", type=int, default=0, help="blocks per grab of a cluster (0 = automatic, 1000000 = static)")
     ap.add_argument("--path", type=int, default=0, help="1 = force the two-pass kernels")
+    ap.add_argument("--statistic", type=int, default=0, help="block statistic: 0 mean (Algorithm 1); 1 max, 2 min, 3 one-norm, 4 two-norm (the paper's ablation)")
+    ap.add_argument("--shard", default="none", choices=["none", "blocks", "flat"],
+                    help="none: every rank steps its own copy of the table (weak scaling); blocks / flat: the ranks "
+                         "share ONE table as whole-block shards / as flat shards with one exchange of part sums (strong scaling)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -214,10 +214,13 @@ int adammini_step_host(am_handle *h, void *const *params, const void *const *gra
  *   <= AM_NOALLOC_MAX_PIECES; larger requests return AM_ERR_TOO_LARGE and do
  *   nothing.
  *
- * The result equals adammini_step's on its two-pass path (same arithmetic).
- * The first call on a device looks up the array's device address (once per
- * device, with that device current); make that first call outside any stream
- * capture.  Every call on a device shares the one array, which keeps whatever
+ * The arithmetic is that of adammini_step's two-pass path, and so are the bits
+ * as long as a block has fewer than 256 partial sums (beyond that the other
+ * path adds a block's partial sums in a different order).  cuda_stream must
+ * belong to the device that is current at the call: that device's array is
+ * used.  The first call on a device looks up the array's device address (once
+ * per device, with that device current); make that first call outside any
+ * stream capture.  Every call on a device shares the one array, which keeps whatever
  * the previous call left there: each call overwrites the entries it uses before
  * it reads them, so nothing needs clearing, but two calls whose kernels overlap
  * on the GPU (different streams, or different threads or processes' streams on
@@ -239,10 +242,11 @@ typedef enum {
     AM_OPT_PATH           = 0, /* 0 = automatic; 1 = force the two-pass path for every tensor with
                                   block_len > 16 (correctness anchor: a second implementation of every
                                   other kernel family's work) */
-    AM_OPT_STREAM_CTAS    = 1, /* persistent CTAs of the streaming kernel (0 = one per SM) */
+    AM_OPT_STREAM_CTAS    = 1, /* persistent CTAs of the streaming kernel (0 = one per SM; at most 4096) */
     AM_OPT_CLUSTER_SIZE   = 2, /* CTAs per cluster for head-sized blocks: 1 to 8 (0 = chosen by block size) */
     AM_OPT_STREAM_THREADS = 3, /* threads per consumer group of the streaming kernels, a multiple of 32
-                                  from 64 to 512 (0 = default 256); groups x threads is capped at 512 */
+                                  from 64 to 512 (0 = default 256; anything else is rejected);
+                                  groups x threads is capped at 512 */
     AM_OPT_PROFILE        = 4, /* n > 0: record CUDA events around each kernel family of every step, keeping
                                   the latest n steps (n <= 4096); read them with adammini_get_profile.
                                   Setting the option again restarts the record */

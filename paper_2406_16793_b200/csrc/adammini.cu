@@ -5,6 +5,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <atomic>
 #include <cmath>
 #include <cstdio>
 #include <cstring>
@@ -373,6 +374,10 @@ int adammini_set_option(am_handle *h, int32_t key, int64_t value) {
     if (key == AM_OPT_STATISTIC && value > 4) return AM_ERR_INVALID_ARGUMENT;
     if (key == AM_OPT_STREAM_GROUPS && value > kMaxGroups) return AM_ERR_INVALID_ARGUMENT;
     if (key == AM_OPT_CLUSTER_SIZE && value > kMaxCluster) return AM_ERR_INVALID_ARGUMENT;
+    // a consumer group is made of whole warps (its shuffles and barriers count warps)
+    if (key == AM_OPT_STREAM_THREADS && value != 0 && (value % 32 != 0 || value < 64 || value > 512))
+        return AM_ERR_INVALID_ARGUMENT;
+    if (key == AM_OPT_STREAM_CTAS && value > kMaxStreamCtas) return AM_ERR_INVALID_ARGUMENT;
     if (key == AM_OPT_PROFILE) {
         if (value > 4096) return AM_ERR_INVALID_ARGUMENT;
         for (cudaEvent_t e : h->prof_ev) cudaEventDestroy(e);
@@ -655,8 +660,10 @@ constexpr int kNoAllocMaxDevices = 64;
 static __device__ __align__(256) unsigned char g_noalloc_scratch[AM_NOALLOC_SCRATCH_BYTES];
 
 // Device address of the array on each device; the symbol itself is only a
-// host-side handle and must never be handed to a kernel.
-void *g_noalloc_addr[kNoAllocMaxDevices] = {};
+// host-side handle and must never be handed to a kernel.  Atomic: host threads
+// may make their first calls on a device at the same time (they all look up
+// the same address).
+std::atomic<void *> g_noalloc_addr[kNoAllocMaxDevices] = {};
 
 __device__ __forceinline__ PieceRef noalloc_piece(const DevTensor &t, int64_t local, bool vec) {
     PieceRef r;
@@ -754,14 +761,14 @@ extern "C" int adammini_step_tensor_noalloc(void *param, const void *grad, void 
     int dev = -1;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess || dev < 0 || dev >= kNoAllocMaxDevices) return AM_ERR_CUDA;
-    if (!g_noalloc_addr[dev]) {
-        void *ptr = nullptr;
-        e = cudaGetSymbolAddress(&ptr, g_noalloc_scratch);
-        if (e != cudaSuccess || !ptr) return AM_ERR_CUDA;
-        g_noalloc_addr[dev] = ptr;
+    void *scratch = g_noalloc_addr[dev].load(std::memory_order_acquire);
+    if (!scratch) {
+        e = cudaGetSymbolAddress(&scratch, g_noalloc_scratch);
+        if (e != cudaSuccess || !scratch) return AM_ERR_CUDA;
+        g_noalloc_addr[dev].store(scratch, std::memory_order_release);
     }
-    double *partials = static_cast<double *>(g_noalloc_addr[dev]);
-    float *block_steps = reinterpret_cast<float *>(static_cast<unsigned char *>(g_noalloc_addr[dev]) +
+    double *partials = static_cast<double *>(scratch);
+    float *block_steps = reinterpret_cast<float *>(static_cast<unsigned char *>(scratch) +
                                                    AM_NOALLOC_MAX_PIECES * sizeof(double));
 
     const double bc1 = 1.0 - std::pow(hp->beta1, static_cast<double>(step));

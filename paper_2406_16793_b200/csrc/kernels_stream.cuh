@@ -52,6 +52,7 @@ constexpr int kExchangeSlots = 4;                 // slots of the cluster exchan
 constexpr int kMaxCluster = 8;
 constexpr int kItemSlots = 8;                     // block indices in flight from a cluster's first CTA to its peers
 constexpr int kStaticRanges = 1000000;            // AM_OPT_STREAM_CHUNK value that selects static ranges
+constexpr int kMaxStreamCtas = 4096;              // most persistent CTAs AM_OPT_STREAM_CTAS accepts
 constexpr int64_t kStreamMaxBlockBytes = 256 << 10;   // longest block one CTA handles alone (bytes of g)
 constexpr int64_t kClusterMaxBlockBytes = 4 << 20;    // longest block a cluster handles (bytes of g)
 constexpr unsigned long long kWaitTimeoutNs = 2000000000ull;   // 2 s

@@ -116,6 +116,11 @@ class ShardedStep:
         self.optimizer.step(self._views(params, False), self._views(grads, True), self._views(m, False),
                             v_local, step, stream)
 
+    def step_local(self, params, grads, m, v_local, step: int, stream: int = 0) -> None:
+        """The same for a rank that keeps only its own share: params/grads/m hold one
+        buffer per piece of self.pieces (piece k: self.specs[k].numel elements)."""
+        self.optimizer.step(params, grads, m, v_local, step, stream)
+
     def close(self) -> None:
         self.optimizer.close()
         self.partition.close()
@@ -251,7 +256,7 @@ class ShardedFlatStep:
     step with the whole-block sums.  `exchange(local)` receives this rank's
     float64 device tensor of part sums (padded to `max_parts`) and must return
     the [world, max_parts] tensor of every rank's sums (an all-gather);
-    `nccl_all_gather` does that with torch.distributed.
+    `all_gather_exchange` does that with torch.distributed.
     """
 
     def __init__(self, tensors: Sequence[TensorSpec], world_size: int, rank: int, device="cuda", **hparams):
@@ -296,15 +301,31 @@ class ShardedFlatStep:
         self.combine(exchange(self.local_sums(grads)))
         self.apply(params, grads, m, v_local, step)
 
+    def step_local(self, params, grads, m, v_local, step: int, exchange) -> None:
+        """step() for a rank that keeps only its own share: one buffer per piece of
+        self.pieces (piece k: self.specs[k].numel elements)."""
+        self.local.zero_()
+        if self.n_parts:
+            self.optimizer.part_sums(grads, self.local)
+        self.combine(exchange(self.local))
+        self.optimizer.step_ex(params, grads, m, v_local, step, part_sums=self.totals if self.n_parts else None)
+
     def close(self) -> None:
         self.optimizer.close()
         self.partition.close()
 
 
-def nccl_all_gather(local):
-    """The exchange of ShardedFlatStep over torch.distributed (NCCL on GPUs)."""
+def all_gather_exchange(local, group=None):
+    """The exchange of ShardedFlatStep over torch.distributed, whatever the
+    backend of the process group (NCCL between GPUs, gloo between CPU ranks):
+    returns the [world, len(local)] tensor of every rank's part sums, rank r's
+    in row r.  A few doubles per rank: a latency-sized collective."""
     import torch
     import torch.distributed as dist
-    out = torch.empty(dist.get_world_size(), local.numel(), dtype=local.dtype, device=local.device)
-    dist.all_gather_into_tensor(out, local)
+    world = dist.get_world_size(group)
+    out = torch.empty(world, local.numel(), dtype=local.dtype, device=local.device)
+    dist.all_gather(list(out.unbind(0)), local.contiguous(), group=group)
     return out
+
+
+nccl_all_gather = all_gather_exchange

@@ -28,36 +28,76 @@ GUARD = 64          # float32 guard words either side of every test buffer
 SENTINEL = -7.0e33
 
 
-MIN_SCALE_RUN = 64
+OWN_SCALE_MIN_L = 4     # blocks shorter than this also get the per-element floor of ShortBlockScale
 
 
-def block_relative_error(got: np.ndarray, want: np.ndarray, L: int) -> float:
-    """max_i |got-want| / max(|want_i|, rms(want over i's block)); NaN/inf must match.
+def block_error_detail(got: np.ndarray, want: np.ndarray, L: int, floor: Optional[np.ndarray] = None):
+    """(max_i |got_i - want_i| / max(|want_i|, rms of want over i's OWN block), index of that element,
+    its scale); NaN/inf must match (else the error is inf).
 
-    For blocks shorter than 64 elements the RMS is taken over the aligned run
-    of 64 consecutive elements that holds the block (a one-element block has no
-    scale of its own: an entry of m or p that crosses zero would otherwise make
-    the ratio meaningless)."""
+    The scale of an element is taken from its own block only, never from a
+    neighbouring block.  Blocks of fewer than OWN_SCALE_MIN_L elements have no
+    dependable scale of their own (every element of such a block can come out of
+    a cancellation at once, and a one-element block has nothing but the element
+    itself); for those the caller passes `floor`, a per-element magnitude of the
+    operands the entry was computed from (see ShortBlockScale), and the scale is
+    max(|want_i|, block rms, floor_i)."""
     got = np.asarray(got, dtype=np.float64).reshape(-1)
     want = np.asarray(want, dtype=np.float64).reshape(-1)
     if want.size == 0:
-        return 0.0
+        return 0.0, -1, 0.0
     fin = np.isfinite(want)
     if not np.array_equal(fin, np.isfinite(got)):
-        return float("inf")
+        return float("inf"), int(np.argmax(fin != np.isfinite(got))), 0.0
     if not fin.all():
         same = np.where(fin, True, (np.isnan(want) & np.isnan(got)) | (want == got))
         if not same.all():
-            return float("inf")
+            return float("inf"), int(np.argmin(same)), 0.0
     w = np.where(fin, want, 0.0)
-    run = L if L >= MIN_SCALE_RUN else MIN_SCALE_RUN
-    starts = np.arange(0, w.size, run)
-    counts = np.diff(np.append(starts, w.size))
-    rms = np.sqrt(np.add.reduceat(w * w, starts) / counts)
-    scale = np.maximum(np.abs(w), np.repeat(rms, counts))
+    assert w.size % L == 0
+    if L == 1:
+        scale = np.abs(w)
+    else:
+        rms = np.sqrt((w.reshape(-1, L) ** 2).mean(axis=1))
+        scale = np.maximum(np.abs(w), np.repeat(rms, L))
+    if floor is not None:
+        assert L < OWN_SCALE_MIN_L, "the floor is for blocks too short to have a scale of their own"
+        f = np.asarray(floor, dtype=np.float64).reshape(-1)
+        scale = np.maximum(scale, np.where(np.isfinite(f), f, 0.0))
     scale = np.where(scale > 0, scale, 1.0)
     err = np.where(fin, np.abs(got - w) / scale, 0.0)
-    return float(err.max())
+    k = int(err.argmax())
+    return float(err[k]), k, float(scale[k])
+
+
+def block_relative_error(got: np.ndarray, want: np.ndarray, L: int, floor: Optional[np.ndarray] = None) -> float:
+    return block_error_detail(got, want, L, floor)[0]
+
+
+class ShortBlockScale:
+    """Error scale for the elements of blocks of fewer than OWN_SCALE_MIN_L
+    elements, each element from its own history.
+
+    An element's m (or p) can pass through zero: m_t = (1-beta1) g_t + beta1 m_{t-1}
+    with operands of opposite sign.  float32 then carries an absolute error of the
+    order of an ulp of the OPERANDS, so the ratio to |m_t| says nothing about the
+    arithmetic; in a block of one, two or three elements all of them can do so at
+    once (seen in the seeded tests: see the design notes), and the block's RMS is
+    then no better a scale.  The scale kept here is the magnitude of those operands,
+    followed along the oracle's own trajectory of that element:
+        S_m(t) = max(|m_t|, (1-beta1)|g_t| + beta1 S_m(t-1)),  S_m(0) = 0
+        S_p(t) = max(|p_t|, S_p(t-1)),                         S_p(0) = |p_0|
+    (rounding errors of earlier steps stay in the state, scaled by beta1 for m
+    and by 1 - eta*lambda, about one, for p).  No other element enters."""
+
+    def __init__(self, p0: np.ndarray):
+        self.p = np.abs(np.asarray(p0, dtype=np.float64)).copy()
+        self.m = np.zeros_like(self.p)
+
+    def update(self, g64: np.ndarray, p: np.ndarray, m: np.ndarray, beta1: float) -> None:
+        with np.errstate(invalid="ignore"):
+            self.m = np.maximum(np.abs(m), (1.0 - beta1) * np.abs(g64) + beta1 * self.m)
+            self.p = np.maximum(self.p, np.abs(p))
 
 
 def v_relative_error(got: np.ndarray, want: np.ndarray) -> float:
@@ -163,6 +203,8 @@ def run_parity(w: W.Workload, steps: Optional[int] = None, options: Optional[Dic
     opt = make_optimizer(w, options, **(hp_override or {}))
     ora = ostep.OracleState([p.cpu() for p in dev.p], [t.block_len for t in w.tensors],
                             [bool(t.apply_weight_decay) for t in w.tensors])
+    unit = {i: ShortBlockScale(ora.p[i]) for i, t in enumerate(w.tensors)
+            if t.block_len < (2 if os.environ.get("ADAMMINI_FLOOR_ONLY_UNIT_BLOCKS") == "1" else OWN_SCALE_MIN_L)}
     pool = cf.ThreadPoolExecutor(max_workers=min(16, os.cpu_count() or 1))
     try:
         for t in range(1, steps + 1):
@@ -176,6 +218,8 @@ def run_parity(w: W.Workload, steps: Optional[int] = None, options: Optional[Dic
             opt.step(dev.p, dev.g, dev.m, dev.v, t)
             grads_cpu = [g.cpu() for g in dev.g]
             oracle_step_all(ora, grads_cpu, t, hp_t, pool, statistic)
+            for i, u in unit.items():
+                u.update(ostep.widen(grads_cpu[i]), ora.p[i], ora.m[i], hp_t["beta1"])
         opt.sync_status()
     finally:
         pool.shutdown()
@@ -184,8 +228,15 @@ def run_parity(w: W.Workload, steps: Optional[int] = None, options: Optional[Dic
     v_gpu = dev.v.cpu().numpy()
     off = 0
     for i, t in enumerate(w.tensors):
-        worst["p"] = max(worst["p"], block_relative_error(dev.p[i].cpu().numpy(), ora.p[i], t.block_len))
-        worst["m"] = max(worst["m"], block_relative_error(dev.m[i].cpu().numpy(), ora.m[i], t.block_len))
+        u = unit.get(i)
+        for key, got, want, floor in (("p", dev.p[i], ora.p[i], u.p if u else None), ("m", dev.m[i], ora.m[i], u.m if u else None)):
+            got = got.cpu().numpy()
+            err, k, scale = block_error_detail(got, want, t.block_len, floor)
+            if err > worst[key]:
+                worst[key] = err
+                # where the worst element is, for the failure message
+                worst[key + "_at"] = (f"{t.name}[{k}] L={t.block_len} gpu={got[k]!r} oracle={want[k]!r} scale={scale:.3e}"
+                                      f" g={float(ostep.widen(grads_cpu[i][k:k + 1])[0]):.3e}")
         worst["v"] = max(worst["v"], v_relative_error(v_gpu[off:off + t.n_blocks], ora.v[i]))
         off += t.n_blocks
     opt.close()
@@ -246,17 +297,21 @@ def run_sampled_runs(w: W.Workload, steps: int, run_elems: int, n_runs: int, dev
     samples = []
     for k in picks:
         sl = slice(k * run_elems, (k + 1) * run_elems)
-        samples.append([sl, ostep.widen(dev.p[0][sl].cpu()), np.zeros(run_elems), np.zeros(run_elems // L)])
+        p0 = ostep.widen(dev.p[0][sl].cpu())
+        samples.append([sl, p0, np.zeros(run_elems), np.zeros(run_elems // L), ShortBlockScale(p0) if L < OWN_SCALE_MIN_L else None])
     for step in range(1, steps + 1):
         dev.draw_grads(step)
         opt.step(dev.p, dev.g, dev.m, dev.v, step)
-        for sl, po, mo, vo in samples:
-            ostep.adammini_step(po, mo, vo, dev.g[0][sl].cpu(), L, step=step, **w.hparams)
+        for sl, po, mo, vo, unit in samples:
+            g = dev.g[0][sl].cpu()
+            ostep.adammini_step(po, mo, vo, g, L, step=step, **w.hparams)
+            if unit is not None:
+                unit.update(ostep.widen(g), po, mo, w.hparams["beta1"])
     opt.sync_status()
     worst = {"p": 0.0, "m": 0.0, "v": 0.0, "blocks": len(samples) * (run_elems // L)}
-    for sl, po, mo, vo in samples:
-        worst["p"] = max(worst["p"], block_relative_error(dev.p[0][sl].cpu().numpy(), po, L))
-        worst["m"] = max(worst["m"], block_relative_error(dev.m[0][sl].cpu().numpy(), mo, L))
+    for sl, po, mo, vo, unit in samples:
+        worst["p"] = max(worst["p"], block_relative_error(dev.p[0][sl].cpu().numpy(), po, L, unit.p if unit else None))
+        worst["m"] = max(worst["m"], block_relative_error(dev.m[0][sl].cpu().numpy(), mo, L, unit.m if unit else None))
         vs = slice(sl.start // L, sl.stop // L)
         worst["v"] = max(worst["v"], v_relative_error(dev.v[vs].cpu().numpy(), vo))
     opt.close()

@@ -83,19 +83,24 @@ def test_gradient_scale_against_the_oracle():
     s = float(np.float32(scale_host)) * float(np.float32(scale_dev))
     ora = ostep.OracleState([p.cpu() for p in dev.p], [t.block_len for t in w.tensors],
                             [bool(t.apply_weight_decay) for t in w.tensors])
+    unit = {i: H.ShortBlockScale(ora.p[i]) for i, t in enumerate(w.tensors) if t.block_len < H.OWN_SCALE_MIN_L}
     for t in range(1, 5):
         dev.draw_grads(t)
         opt.step_ex(dev.p, dev.g, dev.m, dev.v, t, grad_scale=scale_host, grad_scale_device=dscale)
         for i, g in enumerate(dev.g):
-            ostep.adammini_step(ora.p[i], ora.m[i], ora.v[i], ostep.widen(g.cpu()) * s, ora.block_lens[i], step=t,
+            g64 = ostep.widen(g.cpu()) * s
+            ostep.adammini_step(ora.p[i], ora.m[i], ora.v[i], g64, ora.block_lens[i], step=t,
                                 apply_wd=ora.wd_flags[i], **w.hparams)
+            if i in unit:
+                unit[i].update(g64, ora.p[i], ora.m[i], w.hparams["beta1"])
     opt.sync_status()
     assert dev.guards_intact()
     worst = {"p": 0.0, "m": 0.0, "v": 0.0}
     v_gpu, off = dev.v.cpu().numpy(), 0
     for i, t in enumerate(w.tensors):
-        worst["p"] = max(worst["p"], H.block_relative_error(dev.p[i].cpu().numpy(), ora.p[i], t.block_len))
-        worst["m"] = max(worst["m"], H.block_relative_error(dev.m[i].cpu().numpy(), ora.m[i], t.block_len))
+        u = unit.get(i)
+        worst["p"] = max(worst["p"], H.block_relative_error(dev.p[i].cpu().numpy(), ora.p[i], t.block_len, u.p if u else None))
+        worst["m"] = max(worst["m"], H.block_relative_error(dev.m[i].cpu().numpy(), ora.m[i], t.block_len, u.m if u else None))
         worst["v"] = max(worst["v"], H.v_relative_error(v_gpu[off:off + t.n_blocks], ora.v[i]))
         off += t.n_blocks
     H.assert_parity(worst)

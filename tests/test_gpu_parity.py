@@ -201,6 +201,30 @@ def test_argument_errors():
     opt.close()
 
 
+def test_launch_options_are_validated():
+    """Consumer groups are whole warps: thread counts that are not a multiple of 32
+    from 64 to 512 (and absurd CTA counts) are refused before anything is planned or
+    launched, and the handle keeps working with the plan it had."""
+    w = W.scaled_rows(W.llama2_7b(n_layers=1, vocab=256), 128)
+    ref = _run_steps(w, 1, 2)
+    dev = H.DeviceState(w, guarded=False)
+    opt = H.make_optimizer(w)
+    before = [opt.query(q) for q in (B.Q_LAUNCHES_PER_STEP, B.Q_STREAM_CTAS, B.Q_CLUSTER_SIZE, B.Q_SCRATCH_BYTES)]
+    for key, bad in ((B.OPT_STREAM_THREADS, 48), (B.OPT_STREAM_THREADS, 100), (B.OPT_STREAM_THREADS, 1000),
+                     (B.OPT_STREAM_THREADS, 32), (B.OPT_STREAM_CTAS, 1 << 20), (B.OPT_STREAM_GROUPS, 3),
+                     (B.OPT_CLUSTER_SIZE, 9), (B.OPT_STATISTIC, 5), (B.OPT_PATH, 2)):
+        with pytest.raises(am.AdamMiniError) as e:
+            opt.set_option(key, bad)
+        assert e.value.status == -1, (key, bad)
+    assert before == [opt.query(q) for q in (B.Q_LAUNCHES_PER_STEP, B.Q_STREAM_CTAS, B.Q_CLUSTER_SIZE, B.Q_SCRATCH_BYTES)]
+    for t in (1, 2):
+        dev.draw_grads(t)
+        opt.step(dev.p, dev.g, dev.m, dev.v, t)
+    opt.sync_status()
+    opt.close()
+    assert _same(ref, dev)
+
+
 def test_empty_partition_and_queries():
     opt = am.AdamMini(am.Partition([]))
     opt.step([], [], [], 0, 1)
@@ -465,10 +489,16 @@ def test_flat_shards_that_cut_blocks(world):
     v_local = [torch.zeros(max(r.local_blocks, 1), device="cuda") for r in ranks]
     for t in range(1, w.steps + 1):
         dev.draw_grads(t)
-        gathered = torch.stack([r.local_sums(dev.g).clone() for r in ranks])      # stands in for the all-gather
-        for r, v in zip(ranks, v_local):
-            r.combine(gathered)
-            r.apply(dev.p, dev.g, dev.m, v, t)
+        # The ranks run one after the other here, so what the all-gather would return is put
+        # together first (gradients do not change during a step); every rank then runs its
+        # whole step() -- local sums, exchange, combine, apply -- with a stand-in exchange that
+        # checks what the rank contributes and hands back the gathered rows.
+        gathered = torch.stack([r.local_sums(dev.g).clone() for r in ranks])
+        for k, (r, v) in enumerate(zip(ranks, v_local)):
+            def exchange(local, k=k):
+                assert torch.equal(local, gathered[k])
+                return gathered
+            r.step(dev.p, dev.g, dev.m, v, t, exchange)
         H.oracle_step_all(ora, [g.cpu() for g in dev.g], t, w.hparams)
     torch.cuda.synchronize()
     assert dev.guards_intact()
@@ -585,7 +615,7 @@ def test_random_tables_and_launch_options():
         w = W.Workload(f"random{seed}", 800 + seed, _random_table(rng), W.GradRecipe(-4.0, -1.0), steps=2)
         options = _random_options(rng)
         worst = H.run_parity(w, options=options)
-        assert max(worst.values()) <= H.TOL, (seed, options, worst)
+        assert max(worst[k] for k in "pmv") <= H.TOL, (seed, options, worst)
 
 
 @pytest.mark.parametrize("grad_dtype", [W.F32, W.BF16], ids=["f32", "bf16"])

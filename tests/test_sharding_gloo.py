@@ -141,9 +141,9 @@ def _flat_rank_main(rank, world, port, result_dir):
             g = grads[p.tensor][p.elem_begin:p.elem_end]
             local[k] = float((g * g).sum())
             k += 1
-    gathered = [torch.zeros_like(local) for _ in range(world)]
-    dist.all_gather(gathered, local)                                    # the step's one exchange
-    totals = plan.combine(torch.stack(gathered))
+    gathered = sharding.all_gather_exchange(local)                      # the step's one exchange, as the GPU path calls it
+    assert gathered.shape == (world, plan.max_parts) and torch.equal(gathered[rank], local)
+    totals = plan.combine(gathered)
     torch.save((plan.part_keys, totals[:plan.n_parts]), os.path.join(result_dir, f"rank{rank}.pt"))
     dist.barrier()
     dist.destroy_process_group()
