@@ -243,7 +243,8 @@ typedef enum {
                                   block_len > 16 (correctness anchor: a second implementation of every
                                   other kernel family's work) */
     AM_OPT_STREAM_CTAS    = 1, /* persistent CTAs of the streaming kernel (0 = one per SM; at most 4096) */
-    AM_OPT_CLUSTER_SIZE   = 2, /* CTAs per cluster for head-sized blocks: 1 to 8 (0 = chosen by block size) */
+    AM_OPT_CLUSTER_SIZE   = 2, /* CTAs per cluster for head-sized blocks: 1 to 8, lowered to the next size the
+                                  device can run (0 = chosen by adammini_choose_cluster_size) */
     AM_OPT_STREAM_THREADS = 3, /* threads per consumer group of the streaming kernels, a multiple of 32
                                   from 64 to 512 (0 = default 256; anything else is rejected);
                                   groups x threads is capped at 512 */
@@ -259,10 +260,22 @@ typedef enum {
     AM_OPT_STATISTIC      = 7, /* block statistic that feeds v: 0 = mean(g*g), Algorithm 1.  The ablation
                                   of the paper's appendix ("Ablation Studies on the Design of Adam-mini"),
                                   which it reports to train worse: 1 = max, 2 = min, 3 = 1-norm (sum),
-                                  4 = 2-norm of the vector g*g.  Non-zero values run on the short-block
-                                  kernels (block_len <= 64) and the two-pass kernels (g read twice) */
-    AM_OPT_STREAM_GROUPS  = 8  /* consumer groups per CTA of the streaming kernel, which own alternate
+                                  4 = 2-norm of the vector g*g.  Every kernel family takes the statistic
+                                  as a parameter of its block reduction (g is still read once).  Blocks
+                                  that hold a NaN gradient: their max / min is unspecified.  Tables with
+                                  AM_PART tensors support the mean only */
+    AM_OPT_STREAM_GROUPS  = 8, /* consumer groups per CTA of the streaming kernel, which own alternate
                                   work items: 1 or 2 (0 = default: 2; the cluster kernel runs one) */
+    AM_OPT_WAIT_LIMIT_US  = 9, /* how long a device-side wait (for a staged copy, a barrier of a consumer
+                                  group, a cluster exchange) polls before it gives up, in microseconds:
+                                  100 to 60 000 000 (0 = default: 2 s).  A wait that gives up ends its
+                                  kernel through the normal exit; adammini_sync_status then returns
+                                  AM_ERR_TIMEOUT and the tensors of that step are partly updated */
+    AM_OPT_TEST_STALL     = 10 /* for tests of that error path: n > 0 makes the thread that stages data
+                                  withhold its n-th and later stages in every CTA of the streaming
+                                  kernels (the tile kernel announces its copies without issuing them),
+                                  so that the waits above run out.  Nothing faults and nothing waits
+                                  without a limit.  0 = off */
 } am_option;
 int adammini_set_option(am_handle *h, int32_t key, int64_t value);
 
@@ -286,9 +299,25 @@ typedef enum {
     AM_Q_STREAM_CTAS       = 13, /* launch shape of the streaming kernel */
     AM_Q_CLUSTER_SIZE      = 14,
     AM_Q_CLUSTER_COUNT     = 15,
-    AM_Q_PART_TENSORS      = 16  /* number of AM_PART tensors in the table */
+    AM_Q_PART_TENSORS      = 16, /* number of AM_PART tensors in the table */
+    AM_Q_L2_BYTES          = 17, /* what planning read from the device: L2 size, */
+    AM_Q_SMEM_BYTES        = 18, /* most dynamic shared memory a CTA may ask for, */
+    AM_Q_RESIDENT_CLUSTERS = 19  /* and, at 19 + (c - 1) for c = 1..8, how many clusters of c CTAs of the
+                                    streaming kernel fit the device at once (with the handle's current
+                                    threads per CTA): the inputs of adammini_choose_cluster_size */
 } am_query;
 int adammini_query(const am_handle *h, int32_t what, int64_t *value);
+
+/* The planning rule behind AM_Q_CLUSTER_SIZE, as a function of what a handle reads from its
+ * device (host only; no CUDA call): the CTAs per cluster chosen for head-sized blocks whose
+ * gradients take `block_bytes`, on a device with `l2_bytes` of L2 that keeps
+ * resident_clusters[c] clusters of c CTAs of the streaming kernel resident at once
+ * (host array of 9 entries, c = 1..8; entry 0 is ignored; 0 = clusters of that size cannot
+ * run).  A cluster reads a block's gradients twice and the second read should hit L2, so the
+ * rule takes the smallest size (most clusters, most SMs busy) whose resident clusters keep no
+ * more than a fixed share of L2 in flight, the largest size that can run otherwise, and 0 when
+ * no cluster can run (such blocks then take the two-pass kernels).  Negative: am_status. */
+int32_t adammini_choose_cluster_size(const int32_t *resident_clusters, int64_t l2_bytes, int64_t block_bytes);
 
 /* With AM_OPT_PROFILE set: waits for the recorded steps and writes the mean device time in
  * milliseconds per step of each kernel family to ms[0..3] (host array): short-block

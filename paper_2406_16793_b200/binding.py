@@ -17,12 +17,13 @@ LIBRARY = os.environ.get("ADAMMINI_LIBRARY") or os.path.join(_HERE, "libadammini
 WHOLE, ROWS, HEADS, TOKENS, FIXED, PART = 0, 1, 2, 3, 4, 5
 F32, BF16 = 0, 1
 
-OPT_PATH, OPT_STREAM_CTAS, OPT_CLUSTER_SIZE, OPT_STREAM_THREADS, OPT_PROFILE, OPT_STREAM_CHUNK, OPT_CLUSTER_CHUNK, OPT_STATISTIC, OPT_STREAM_GROUPS = 0, 1, 2, 3, 4, 5, 6, 7, 8
+(OPT_PATH, OPT_STREAM_CTAS, OPT_CLUSTER_SIZE, OPT_STREAM_THREADS, OPT_PROFILE, OPT_STREAM_CHUNK, OPT_CLUSTER_CHUNK,
+ OPT_STATISTIC, OPT_STREAM_GROUPS, OPT_WAIT_LIMIT_US, OPT_TEST_STALL) = range(11)
 STAT_MEAN, STAT_MAX, STAT_MIN, STAT_ONE_NORM, STAT_TWO_NORM = 0, 1, 2, 3, 4
 (Q_LAUNCHES_PER_STEP, Q_SCRATCH_BYTES, Q_TOTAL_BLOCKS, Q_TOTAL_ELEMENTS, Q_ELEMENTS_SMALL,
  Q_ELEMENTS_STREAM, Q_ELEMENTS_CLUSTER, Q_ELEMENTS_TWOPASS, Q_ALGORITHMIC_BYTES, Q_BYTES_SMALL,
  Q_BYTES_STREAM, Q_BYTES_CLUSTER, Q_BYTES_TWOPASS, Q_STREAM_CTAS, Q_CLUSTER_SIZE, Q_CLUSTER_COUNT,
- Q_PART_TENSORS) = range(17)
+ Q_PART_TENSORS, Q_L2_BYTES, Q_SMEM_BYTES, Q_RESIDENT_CLUSTERS) = range(20)
 
 
 class TensorDesc(ctypes.Structure):
@@ -79,6 +80,7 @@ _SIGNATURES = {
     "adammini_sync_status": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p]),
     "adammini_set_option": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64]),
     "adammini_query": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.POINTER(ctypes.c_int64)]),
+    "adammini_choose_cluster_size": (ctypes.c_int32, [ctypes.POINTER(ctypes.c_int32), ctypes.c_int64, ctypes.c_int64]),
     "adammini_get_profile": (ctypes.c_int, [ctypes.c_void_p, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32)]),
     "adammini_last_cuda_error": (ctypes.c_int, [ctypes.c_void_p]),
     "adammini_destroy": (ctypes.c_int, [ctypes.c_void_p]),
@@ -125,6 +127,15 @@ def _check(status: int, handle=None) -> None:
 def kind_from_name(name: str) -> int:
     """Algorithm 3's name tests (embed/output, query/key, value/attn.proj/mlp, else)."""
     return int(load().adammini_kind_from_name(name.encode()))
+
+
+def choose_cluster_size(resident_clusters: Sequence[int], l2_bytes: int, block_bytes: int) -> int:
+    """The library's choice of CTAs per cluster for head-sized blocks (host logic only):
+    resident_clusters[c] = clusters of c CTAs the device keeps resident, c = 1..8 (entry 0 unused)."""
+    arr = (ctypes.c_int32 * 9)(*([0] * 9))
+    for c, n in enumerate(list(resident_clusters)[:9]):
+        arr[c] = int(n)
+    return int(load().adammini_choose_cluster_size(arr, int(l2_bytes), int(block_bytes)))
 
 
 NOALLOC_MAX_BLOCKS = 32768

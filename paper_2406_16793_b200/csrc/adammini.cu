@@ -22,7 +22,7 @@ using namespace am;
 
 namespace {
 
-constexpr int kNumOptions = 9;
+constexpr int kNumOptions = 11;
 
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
@@ -75,7 +75,6 @@ int build_plan(am_handle *h) {
     h->algorithmic_bytes = 0;
 
     StreamPlanInput sin;
-    sin.sm_count = h->sm_count;
     sin.ctas = static_cast<int>(h->opt[AM_OPT_STREAM_CTAS]);
     sin.cluster_size = static_cast<int>(h->opt[AM_OPT_CLUSTER_SIZE]);
     sin.threads = static_cast<int>(h->opt[AM_OPT_STREAM_THREADS]);
@@ -86,7 +85,16 @@ int build_plan(am_handle *h) {
     {
         int threads, groups;
         stream_consumer_shape(sin.threads, sin.groups, &threads, &groups);
-        stream_probe_cluster(h->sm_count, threads * groups, sin.cluster_size, &h->cluster_size, &h->n_clusters);
+        stream_probe_clusters(&h->caps, 32 + threads * groups);
+        sin.caps = h->caps;
+    }
+    bool clusters_ok = false;
+    for (int c = 1; c <= kMaxCluster; ++c) clusters_ok |= h->caps.resident[c] > 0;
+    bool stream_ok;         // the ring needs at least two stages of the larger layout
+    {
+        int g_region, stage_bytes, n_stages;
+        stream_stage_layout(true, h->caps.smem_optin, &g_region, &stage_bytes, &n_stages);
+        stream_ok = n_stages >= 2;
     }
 
     for (int i = 0; i < n; ++i) {
@@ -105,9 +113,9 @@ int build_plan(am_handle *h) {
         int path;
         if (r.kind == AM_PART) path = PATH_TWOPASS;          // its sum of squares comes from outside
         else if (r.block_len <= kSmallMaxL && !(h->opt[AM_OPT_PATH] == 1 && r.block_len > 16)) path = PATH_SMALL;
-        else if (h->opt[AM_OPT_PATH] == 1 || h->opt[AM_OPT_STATISTIC] != 0) path = PATH_TWOPASS;
+        else if (h->opt[AM_OPT_PATH] == 1) path = PATH_TWOPASS;
         else {
-            path = stream_classify(r.block_len, r.grad_dtype, h->n_clusters > 0);
+            path = stream_ok ? stream_classify(r.block_len, r.grad_dtype, clusters_ok) : PATH_TWOPASS;
             // block starts off the 16-byte grid: the tile kernel copes, up to its tile size
             if (path == PATH_TWOPASS && r.block_len <= kTileMaxL) path = PATH_SMALL;
         }
@@ -199,7 +207,7 @@ int build_plan(am_handle *h) {
         return AM_ERR_TOO_LARGE;
 
     StreamPlan &sp = h->stream;
-    stream_finish_plan(sin, h->cluster_size, h->n_clusters, &sp);
+    stream_finish_plan(sin, &sp);
     sp.v_len = h->total_blocks;
 
     // device arena: tensor table, unit tables, scratch
@@ -327,6 +335,9 @@ int adammini_create(const am_partition *part, const am_hparams *hp, am_handle **
     if (e == cudaSuccess) e = cudaGetDeviceProperties(&prop, h->device);
     if (e == cudaSuccess) {
         h->sm_count = prop.multiProcessorCount;
+        h->caps.sm_count = prop.multiProcessorCount;
+        h->caps.smem_optin = prop.sharedMemPerBlockOptin;
+        h->caps.l2_bytes = prop.l2CacheSize;
         const size_t n = std::max<size_t>(h->rows.size(), 1);
         for (int k = 0; k < 2 && e == cudaSuccess; ++k) {
             e = cudaMallocHost(&h->pinned[k], sizeof(DevTensor) * n);
@@ -335,7 +346,7 @@ int adammini_create(const am_partition *part, const am_hparams *hp, am_handle **
     }
     if (e == cudaSuccess) e = cudaMallocHost(&h->error_word, sizeof(int));
     if (e == cudaSuccess) *h->error_word = 0;
-    if (e == cudaSuccess) e = stream_configure_kernels();
+    if (e == cudaSuccess) e = stream_configure_kernels(h->caps.smem_optin);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(tile_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileSmemBytes);
     if (e != cudaSuccess) {
         g_create_cuda_error = static_cast<int>(e);
@@ -378,6 +389,12 @@ int adammini_set_option(am_handle *h, int32_t key, int64_t value) {
     if (key == AM_OPT_STREAM_THREADS && value != 0 && (value % 32 != 0 || value < 64 || value > 512))
         return AM_ERR_INVALID_ARGUMENT;
     if (key == AM_OPT_STREAM_CTAS && value > kMaxStreamCtas) return AM_ERR_INVALID_ARGUMENT;
+    if (key == AM_OPT_WAIT_LIMIT_US && value != 0 && (value < 100 || value > 60000000)) return AM_ERR_INVALID_ARGUMENT;
+    if (key == AM_OPT_WAIT_LIMIT_US || key == AM_OPT_TEST_STALL) {      // read at every launch: nothing to plan again
+        h->opt[key] = value;
+        if (h->host_step) host_step_release(h);
+        return AM_OK;
+    }
     if (key == AM_OPT_PROFILE) {
         if (value > 4096) return AM_ERR_INVALID_ARGUMENT;
         for (cudaEvent_t e : h->prof_ev) cudaEventDestroy(e);
@@ -425,9 +442,23 @@ int adammini_query(const am_handle *h, int32_t what, int64_t *value) {
     case AM_Q_CLUSTER_SIZE: *value = h->stream.clus.active() ? h->stream.clus.cluster : 0; break;
     case AM_Q_PART_TENSORS: *value = h->n_parts; break;
     case AM_Q_CLUSTER_COUNT: *value = h->stream.clus.active() ? h->stream.clus.grid / h->stream.clus.cluster : 0; break;
-    default: return AM_ERR_INVALID_ARGUMENT;
+    case AM_Q_L2_BYTES: *value = h->caps.l2_bytes; break;
+    case AM_Q_SMEM_BYTES: *value = static_cast<int64_t>(h->caps.smem_optin); break;
+    default:
+        if (what >= AM_Q_RESIDENT_CLUSTERS && what < AM_Q_RESIDENT_CLUSTERS + kMaxCluster) {
+            *value = h->caps.resident[what - AM_Q_RESIDENT_CLUSTERS + 1];
+            break;
+        }
+        return AM_ERR_INVALID_ARGUMENT;
     }
     return AM_OK;
+}
+
+int32_t adammini_choose_cluster_size(const int32_t *resident_clusters, int64_t l2_bytes, int64_t block_bytes) {
+    if (!resident_clusters || l2_bytes < 0 || block_bytes < 0) return AM_ERR_INVALID_ARGUMENT;
+    int resident[kMaxCluster + 1] = {};
+    for (int c = 1; c <= kMaxCluster; ++c) resident[c] = resident_clusters[c];
+    return choose_cluster_size(resident, l2_bytes, block_bytes);
 }
 
 int adammini_last_cuda_error(const am_handle *h) { return h ? h->last_cuda_error : g_create_cuda_error; }
@@ -489,6 +520,10 @@ int adammini_step_ex(am_handle *h, void *const *params, const void *const *grads
     sc.pad = 0;
     sc.part_sums = ex ? ex->part_sums : nullptr;
 
+    const unsigned long long wait_limit_ns =
+        h->opt[AM_OPT_WAIT_LIMIT_US] ? static_cast<unsigned long long>(h->opt[AM_OPT_WAIT_LIMIT_US]) * 1000ull : kWaitTimeoutNs;
+    h->stream.wait_limit_ns = wait_limit_ns;
+    h->stream.stall_after = static_cast<int>(std::min<int64_t>(h->opt[AM_OPT_TEST_STALL], 1 << 30));
     const bool prof = h->opt[AM_OPT_PROFILE] != 0;
     cudaEvent_t *pev = prof ? &h->prof_ev[(h->prof_steps % h->opt[AM_OPT_PROFILE]) * 5] : nullptr;
     if (prof) AM_CUDA(h, cudaEventRecord(pev[0], stream));
@@ -506,6 +541,8 @@ int adammini_step_ex(am_handle *h, void *const *params, const void *const *grads
         ss.gscale_dev = sc.gscale_dev;
         ss.skip_flag = sc.skip_flag;
         ss.statistic = sc.statistic;
+        ss.stall = h->opt[AM_OPT_TEST_STALL] != 0;
+        ss.wait_limit_ns = wait_limit_ns;
         if (h->small_units) {
             small_kernel<<<static_cast<unsigned>(h->small_units), kThreads, 0, stream>>>(
                 h->d_tensors, h->d_small_segs, h->n_small_segs, v, ss);

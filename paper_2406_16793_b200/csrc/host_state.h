@@ -18,7 +18,7 @@ struct am_handle {
     int64_t total_blocks = 0;
     int64_t total_elems = 0;
     am_hparams hp{};
-    int64_t opt[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};
+    int64_t opt[11] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
 
     // launch plan
     bool planned = false;
@@ -44,7 +44,7 @@ struct am_handle {
     double *d_partials = nullptr;
     float *d_block_steps = nullptr;
     am::StreamPlan stream;
-    int cluster_size = 0, n_clusters = 0;   // what the device can keep resident (0: no cluster path)
+    am::DeviceCaps caps;                 // SMs, shared memory, L2, resident clusters per cluster size
     int launches = 0;
     int64_t elems_by_path[4] = {0, 0, 0, 0};
     int64_t algorithmic_bytes = 0;

@@ -131,23 +131,39 @@ extern "C" int adammini_step_host(am_handle *h, void *const *params, const void 
     int dev = -1;
     AM_CUDA(h, cudaGetDevice(&dev));
     if (dev != h->device) return AM_ERR_INVALID_ARGUMENT;
-    int rc = host_step_prepare(h, staging_bytes);
-    if (rc != AM_OK) return rc;
+    int rc;
+    try {
+        rc = host_step_prepare(h, staging_bytes);      // (its tables grow by push_back)
+    } catch (...) {
+        rc = AM_ERR_ALLOC;
+    }
+    if (rc != AM_OK) {
+        host_step_release(h);                           // a half-built pipeline is not kept
+        return rc;
+    }
     HostStepState *s = h->host_step;
 
+    // One exit: whatever fails, the copies already enqueued still read and write the caller's
+    // buffers, so the loop is left through the synchronisation of all three streams below.
     int result = AM_OK;
+    auto copy = [&](void *dst, const void *src, size_t bytes, cudaMemcpyKind kind, cudaStream_t st) {
+        if (result != AM_OK) return;
+        const cudaError_t e = cudaMemcpyAsync(dst, src, bytes, kind, st);
+        if (e != cudaSuccess) result = cuda_fail(h, e);
+    };
     for (size_t gi = 0; gi < s->groups.size() && result == AM_OK; ++gi) {
         HostGroup &g = s->groups[gi];
         cudaStream_t st = s->streams[gi % kHostSlots];
         g.sub->hp = h->hp;
-        AM_CUDA(h, cudaMemcpyAsync(g.d_v, v + g.v_begin, g.v_count * 4, cudaMemcpyHostToDevice, st));
+        copy(g.d_v, v + g.v_begin, g.v_count * 4, cudaMemcpyHostToDevice, st);
         for (int k = 0; k < g.count; ++k) {
             const am_table_row &r = h->rows[g.first + k];
             const size_t gsz = r.grad_dtype == AM_BF16 ? 2 : 4;
-            AM_CUDA(h, cudaMemcpyAsync(const_cast<void *>(g.d_g[k]), grads[g.first + k], r.numel * gsz, cudaMemcpyHostToDevice, st));
-            AM_CUDA(h, cudaMemcpyAsync(g.d_m[k], m[g.first + k], r.numel * 4, cudaMemcpyHostToDevice, st));
-            AM_CUDA(h, cudaMemcpyAsync(g.d_p[k], params[g.first + k], r.numel * 4, cudaMemcpyHostToDevice, st));
+            copy(const_cast<void *>(g.d_g[k]), grads[g.first + k], r.numel * gsz, cudaMemcpyHostToDevice, st);
+            copy(g.d_m[k], m[g.first + k], r.numel * 4, cudaMemcpyHostToDevice, st);
+            copy(g.d_p[k], params[g.first + k], r.numel * 4, cudaMemcpyHostToDevice, st);
         }
+        if (result != AM_OK) break;
         result = adammini_step(g.sub, g.d_p.data(), g.d_g.data(), g.d_m.data(), g.d_v, step, st);
         if (result != AM_OK) {
             h->last_cuda_error = g.sub->last_cuda_error;
@@ -155,10 +171,10 @@ extern "C" int adammini_step_host(am_handle *h, void *const *params, const void 
         }
         for (int k = 0; k < g.count; ++k) {
             const am_table_row &r = h->rows[g.first + k];
-            AM_CUDA(h, cudaMemcpyAsync(m[g.first + k], g.d_m[k], r.numel * 4, cudaMemcpyDeviceToHost, st));
-            AM_CUDA(h, cudaMemcpyAsync(params[g.first + k], g.d_p[k], r.numel * 4, cudaMemcpyDeviceToHost, st));
+            copy(m[g.first + k], g.d_m[k], r.numel * 4, cudaMemcpyDeviceToHost, st);
+            copy(params[g.first + k], g.d_p[k], r.numel * 4, cudaMemcpyDeviceToHost, st);
         }
-        AM_CUDA(h, cudaMemcpyAsync(v + g.v_begin, g.d_v, g.v_count * 4, cudaMemcpyDeviceToHost, st));
+        copy(v + g.v_begin, g.d_v, g.v_count * 4, cudaMemcpyDeviceToHost, st);
     }
     for (int k = 0; k < kHostSlots; ++k) {
         const cudaError_t e = cudaStreamSynchronize(s->streams[k]);

@@ -152,6 +152,8 @@ struct SmallScalars {
     const float *gscale_dev;
     const float *skip_flag;
     int statistic;
+    int stall;                          // test hook of the tile kernel: the bulk copies are announced but not issued
+    unsigned long long wait_limit_ns;   // polling time after which the tile kernel's wait gives up
 };
 
 __device__ __forceinline__ float small_block_step(float mean_sq, float v_old, const SmallScalars &s,

@@ -106,6 +106,9 @@ struct StreamParams {
     unsigned long long *counter;
     int64_t total_items;
     int64_t v_len;              // floats in v (staging never reads past it)
+    unsigned long long wait_limit_ns;   // polling time after which a wait gives up
+    int32_t stall_after;        // test hook: > 0: the producer withholds its n-th and later stages (n = stall_after)
+    int32_t pad;
 };
 
 struct Control {            // first kCtrlBytes of dynamic shared memory
@@ -209,8 +212,8 @@ __device__ __forceinline__ unsigned long long global_ns() {
 // flag) if the phase did not complete within the limit or another thread of
 // the CTA already gave up.
 template <bool CLUSTER_ACQUIRE>
-__device__ __forceinline__ bool wait_phase(void *bar, uint32_t parity, Control *ctl, int *error_word,
-                                           int code, unsigned long long limit_ns = kWaitTimeoutNs) {
+__device__ __forceinline__ bool wait_phase_one(void *bar, uint32_t parity, Control *ctl, int *error_word,
+                                               int code, unsigned long long limit_ns) {
     uint32_t spins = 0;
     unsigned long long last = 0, waited = 0;
     for (;;) {
@@ -233,6 +236,14 @@ __device__ __forceinline__ bool wait_phase(void *bar, uint32_t parity, Control *
             }
         }
     }
+}
+// The same for a whole warp that waits together (the consumers): the lanes agree on the
+// outcome, so a warp never splits between going on and giving up.
+template <bool CLUSTER_ACQUIRE>
+__device__ __forceinline__ bool wait_phase(void *bar, uint32_t parity, Control *ctl, int *error_word,
+                                           int code, unsigned long long limit_ns) {
+    const bool ok = wait_phase_one<CLUSTER_ACQUIRE>(bar, parity, ctl, error_word, code, limit_ns);
+    return __all_sync(0xffffffffu, ok) != 0;
 }
 
 // ------------------------- consumer-side building blocks -------------------------
@@ -289,20 +300,66 @@ __device__ __forceinline__ void apply_span(const unsigned char *gs, const float 
     else apply_span_impl<GD, false, CS>(gs, ms, ps, mg, pg, pb, first, n, tid, nthr, beta1, omb1, lr_wd, step);
 }
 
-template <int GD>
+// The reduction a launch runs over the g*g of a block.  Algorithm 1 needs the sum (for the mean);
+// the ablation of the paper's appendix replaces the mean by the max, the min, the 1-norm (the sum
+// again, not divided) or the 2-norm (root of the sum of (g*g)^2) of the vector g*g.
+enum StatOp : int { ST_SUM = 0, ST_MAX = 1, ST_MIN = 2, ST_SUM4 = 3 };
+
+__host__ __device__ inline int stat_op_of(int statistic) {      // am_option AM_OPT_STATISTIC -> StatOp
+    return statistic == 1 ? ST_MAX : statistic == 2 ? ST_MIN : statistic == 4 ? ST_SUM4 : ST_SUM;
+}
+
+// Per-thread accumulator: float, except for the sum of fourth powers, whose terms
+// (down to 1e-40 for gradients of 1e-10) are below float's normal range.
+template <int ST> struct StatAcc { typedef float T; };
+template <> struct StatAcc<ST_SUM4> { typedef double T; };
+
+template <int ST>
+__device__ __forceinline__ typename StatAcc<ST>::T stat_acc_init() {
+    return ST == ST_MIN ? static_cast<typename StatAcc<ST>::T>(__int_as_float(0x7f800000)) : static_cast<typename StatAcc<ST>::T>(0);
+}
+template <int ST>
+__device__ __forceinline__ void stat_acc_add(typename StatAcc<ST>::T &a, float g) {
+    if (ST == ST_SUM) a = fmaf(g, g, a);
+    else if (ST == ST_MAX) a = fmaxf(a, g * g);
+    else if (ST == ST_MIN) a = fminf(a, g * g);
+    else { const double sq = static_cast<double>(g * g); a = static_cast<typename StatAcc<ST>::T>(fma(sq, sq, static_cast<double>(a))); }
+}
+// Two partial results of the same statistic.
+template <int ST>
+__device__ __forceinline__ double stat_op_combine(double a, double b) {
+    if (ST == ST_MAX) return a > b ? a : b;
+    if (ST == ST_MIN) return a < b ? a : b;
+    return a + b;
+}
+// From the reduced value to the statistic's numerator: the block step divides a
+// sum by the block length for the mean and takes everything else as it is.
+template <int ST>
+__device__ __forceinline__ double stat_op_finish(double acc) { return ST == ST_SUM4 ? sqrt(acc) : acc; }
+
+template <int GD, int ST>
 __device__ __forceinline__ void sum_span(const unsigned char *gs, int first, int n, int tid, int nthr,
-                                         float &a0, float &a1, float &a2, float &a3) {
+                                         typename StatAcc<ST>::T &a0, typename StatAcc<ST>::T &a1,
+                                         typename StatAcc<ST>::T &a2, typename StatAcc<ST>::T &a3) {
 #pragma unroll 2
     for (int i = first + tid * 4; i < first + n; i += nthr * 4) {
         const float4 g = lds_g4<GD>(gs, i);
-        a0 = fmaf(g.x, g.x, a0); a1 = fmaf(g.y, g.y, a1);
-        a2 = fmaf(g.z, g.z, a2); a3 = fmaf(g.w, g.w, a3);
+        stat_acc_add<ST>(a0, g.x); stat_acc_add<ST>(a1, g.y);
+        stat_acc_add<ST>(a2, g.z); stat_acc_add<ST>(a3, g.w);
     }
 }
 
-__device__ __forceinline__ double fold4(float a0, float a1, float a2, float a3) {
-    return (static_cast<double>(a0) + static_cast<double>(a1)) +
-           (static_cast<double>(a2) + static_cast<double>(a3));
+template <int ST, typename A>
+__device__ __forceinline__ double fold4(A a0, A a1, A a2, A a3) {
+    return stat_op_combine<ST>(stat_op_combine<ST>(static_cast<double>(a0), static_cast<double>(a1)),
+                               stat_op_combine<ST>(static_cast<double>(a2), static_cast<double>(a3)));
+}
+
+template <int ST>
+__device__ __forceinline__ double warp_combine(double x) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x = stat_op_combine<ST>(x, __shfl_xor_sync(0xffffffffu, x, o));
+    return x;
 }
 
 // State of the consumer group's own barrier (an mbarrier so that it is bounded).
@@ -311,21 +368,22 @@ struct GroupSync {
     int buf;
 };
 
-// Sum `mine` over the threads of one consumer group in a fixed order; also
+// Combine `mine` over the threads of one consumer group in a fixed order; also
 // broadcasts v_old read by the group's first thread.  Returns false on abort.
-__device__ __forceinline__ bool group_reduce(Control *ctl, GroupSync &gs, int *error_word, int group, int gtid,
-                                             int n_warps, double mine, const float *v_ptr, double *total,
-                                             float *v_old) {
-    const double w = warp_sum(mine);
+template <int ST>
+__device__ __forceinline__ bool group_reduce(Control *ctl, GroupSync &gs, int *error_word, unsigned long long limit_ns,
+                                             int group, int gtid, int n_warps, double mine, const float *v_ptr,
+                                             double *total, float *v_old) {
+    const double w = warp_combine<ST>(mine);
     const int lane = gtid & 31;
     if (lane == 0) {
         ctl->red[group][gs.buf][gtid >> 5] = w;
         if (gtid == 0) ctl->redv[group][gs.buf] = *v_ptr;
         mbar_arrive(&ctl->redbar[group]);
     }
-    if (!wait_phase<false>(&ctl->redbar[group], gs.parity, ctl, error_word, 3)) return false;
-    double s = 0.0;
-    for (int k = 0; k < n_warps; ++k) s += ctl->red[group][gs.buf][k];
+    if (!wait_phase<false>(&ctl->redbar[group], gs.parity, ctl, error_word, 3, limit_ns)) return false;
+    double s = ctl->red[group][gs.buf][0];
+    for (int k = 1; k < n_warps; ++k) s = stat_op_combine<ST>(s, ctl->red[group][gs.buf][k]);
     *total = s;
     *v_old = ctl->redv[group][gs.buf];
     gs.parity ^= 1;
@@ -336,12 +394,14 @@ __device__ __forceinline__ bool group_reduce(Control *ctl, GroupSync &gs, int *e
 // ------------------------------------ kernel ------------------------------------
 // Template parameters keep the code of one launch small (the consumer loop is
 // sensitive to instruction-cache misses): GDM says which gradient dtypes the
-// launch's tensors have, COPY whether any tensor wants a bf16 copy.
+// launch's tensors have, COPY whether any tensor wants a bf16 copy, ST the block
+// statistic (StatOp; ST_SUM is Algorithm 1's mean).
 enum GradMode : int { GDM_F32 = 0, GDM_BF16 = 1, GDM_MIXED = 2 };
 
-template <bool CLUSTER, int GDM, bool COPY>
+template <bool CLUSTER, int GDM, bool COPY, int ST>
 __global__ void __launch_bounds__(32 + kMaxConsumerWarps * 32, 1)
 stream_kernel(const __grid_constant__ StreamParams P) {
+    typedef typename StatAcc<ST>::T Acc;
     extern __shared__ __align__(128) unsigned char smem[];
     if (step_skipped(P.sc.skip_flag)) return;      // uniform over the grid: nobody reaches a barrier
     Control *ctl = reinterpret_cast<Control *>(smem);
@@ -388,8 +448,12 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                 }
                 seg = lo;
             }
+            // (test hook: from the stall_after-th stage on the producer behaves as if its wait had
+            // failed, without raising the abort flag: it arms nothing more, sends no DONE, lets its
+            // copies land and leaves, so that the consumers' next wait runs out)
             auto acquire = [&]() -> bool {
-                return wait_phase<false>(&ctl->empty[stage], phase ^ 1u, ctl, P.error_word, 1);
+                if (P.stall_after > 0 && armed >= P.stall_after - 1) return false;
+                return wait_phase_one<false>(&ctl->empty[stage], phase ^ 1u, ctl, P.error_word, 1, P.wait_limit_ns);
             };
             auto advance = [&]() {
                 ++armed;
@@ -426,8 +490,28 @@ stream_kernel(const __grid_constant__ StreamParams P) {
             auto cluster_take = [&]() -> int64_t {
                 const uint32_t slot = taken & (kItemSlots - 1), par = (taken / kItemSlots) & 1u;
                 ++taken;
-                if (!wait_phase<true>(&ctl->ibar[slot], par, ctl, P.error_word, 5)) { ok = false; return P.total_items; }
+                if (!wait_phase_one<true>(&ctl->ibar[slot], par, ctl, P.error_word, 5, P.wait_limit_ns)) { ok = false; return P.total_items; }
                 return *reinterpret_cast<volatile long long *>(&ctl->next_item[slot]);
+            };
+            // The segment an item lies in, and what the stages of its tensor need, are looked up when
+            // the walk enters a segment and kept in registers: per item the producer only computes
+            // offsets (its time per stage counts: a free stage that is not armed at once is
+            // bandwidth not asked for).
+            StreamSeg sg = {};
+            DevTensor t = {};
+            int64_t seg_hi = -1;                    // first slot past the cached segment (-1: nothing cached yet)
+            int gsz = 4, base_flags = 0;
+            double inv_L = 1.0;
+            const unsigned char *gbase = nullptr;
+            auto load_segment = [&](int64_t item) {
+                while (seg + 1 < P.n_segs && P.segs[seg + 1].item_begin <= item) ++seg;
+                sg = P.segs[seg];
+                seg_hi = P.segs[seg + 1].item_begin;        // (the table ends with a sentinel)
+                t = P.tensors[sg.tensor];
+                gsz = t.gdtype == AM_BF16 ? 2 : 4;
+                base_flags = (t.gdtype == AM_BF16 ? SF_BF16 : 0) | (t.wd ? SF_WD : 0);
+                gbase = static_cast<const unsigned char *>(t.g);
+                inv_L = P.sc.statistic == 0 ? 1.0 / static_cast<double>(t.L) : 1.0;
             };
             int64_t it = item_lo, hi = item_hi, next = 0;
             if (dynamic) {
@@ -452,9 +536,7 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                         next = static_cast<int64_t>(atomicAdd(P.counter, static_cast<unsigned long long>(P.chunk)));
                     }
                 }
-                while (seg + 1 < P.n_segs && P.segs[seg + 1].item_begin <= it) ++seg;
-                const StreamSeg sg = P.segs[seg];
-                const DevTensor &t = P.tensors[sg.tensor];
+                if (it >= seg_hi) load_segment(it);     // (items only move forward)
                 int64_t local = it - sg.item_begin;
                 if (sg.slots > 1) {
                     const int64_t rem = local % sg.slots;
@@ -464,9 +546,6 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                     }
                     local /= sg.slots;
                 }
-                const int gsz = t.gdtype == AM_BF16 ? 2 : 4;
-                const int base_flags = (t.gdtype == AM_BF16 ? SF_BF16 : 0) | (t.wd ? SF_WD : 0);
-                const unsigned char *gbase = static_cast<const unsigned char *>(t.g);
                 if (sg.bpi > 0) {
                     const int64_t b0 = local * sg.bpi;
                     const int64_t left = t.n_blocks - b0;
@@ -477,7 +556,7 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                     StageMeta &mt = ctl->meta[stage];
                     mt.m = t.m + e0; mt.p = t.p + e0; mt.v = P.v + t.v_offset + b0;
                     mt.pb = t.p_bf16 ? t.p_bf16 + e0 : nullptr; mt.group = item_group;
-                    mt.inv_L = 1.0 / static_cast<double>(t.L);
+                    mt.inv_L = inv_L;
                     mt.n = n; mt.L = static_cast<int>(t.L); mt.kind = STAGE_PACKED; mt.flags = base_flags | SF_WRITE_V;
                     const uint32_t vbytes = stage_v(mt, t.v_offset + b0, nb);
                     unsigned char *st = stages + static_cast<size_t>(stage) * P.stage_bytes;
@@ -505,7 +584,7 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                         if (!(ok = acquire())) break;
                         StageMeta &mt = ctl->meta[stage];
                         mt.m = nullptr; mt.p = nullptr; mt.v = P.v + t.v_offset + local; mt.pb = nullptr; mt.group = item_group;
-                        mt.inv_L = 1.0 / static_cast<double>(t.L);
+                        mt.inv_L = inv_L;
                         mt.n = c; mt.L = 0; mt.kind = STAGE_SUM;
                         mt.flags = base_flags | (off + c == slice ? SF_LAST : 0) | (crank == 0 ? SF_WRITE_V : 0);
                         const uint32_t vbytes = (off + c == slice) ? stage_v(mt, t.v_offset + local, 1) : 0u;
@@ -555,6 +634,7 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                 }
             }
         }
+        if (CLUSTER) __syncwarp();       // the producer's warp reaches the cluster's exit barrier together
     } else {
         // ------------------------------ consumers ------------------------------
         // The consumer warps form P.n_groups groups.  Every group follows the ring in order and
@@ -577,11 +657,11 @@ stream_kernel(const __grid_constant__ StreamParams P) {
             int stage = 0;
             uint32_t phase = 0;
             GroupSync gsync{0u, 0};
-            float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;   // running sums of a long block
+            Acc a0 = stat_acc_init<ST>(), a1 = a0, a2 = a0, a3 = a0;   // running statistic of a long block
             float long_step = 0.f;
             uint32_t long_seen = 0;      // long blocks seen by this CTA, whoever owns them (exchange slot/parity)
             for (;;) {
-                if (!wait_phase<false>(&ctl->full[stage], phase, ctl, P.error_word, 2)) break;
+                if (!wait_phase<false>(&ctl->full[stage], phase, ctl, P.error_word, 2, P.wait_limit_ns)) break;
                 const StageMeta mt = ctl->meta[stage];
                 if (mt.kind == STAGE_DONE) break;
                 const bool last_sum = mt.kind == STAGE_SUM && (mt.flags & SF_LAST);
@@ -606,17 +686,23 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                     if (L <= kWarpBlockMaxL) {
                         for (int b = warp; b < nb; b += n_gwarps) {
                             const int e = b * L;
-                            float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-                            if (bf16) sum_span<AM_BF16>(gs, e, L, lane, 32, s0, s1, s2, s3);
-                            else sum_span<AM_F32>(gs, e, L, lane, 32, s0, s1, s2, s3);
-                            // at most 8 terms per accumulator and a 5-level tree: float is enough
-                            float tot = (s0 + s1) + (s2 + s3);
+                            Acc s0 = stat_acc_init<ST>(), s1 = s0, s2 = s0, s3 = s0;
+                            if (bf16) sum_span<AM_BF16, ST>(gs, e, L, lane, 32, s0, s1, s2, s3);
+                            else sum_span<AM_F32, ST>(gs, e, L, lane, 32, s0, s1, s2, s3);
+                            double wtot;
+                            if (ST == ST_SUM) {
+                                // at most 8 terms per accumulator and a 5-level tree: float is enough
+                                float tot = (static_cast<float>(s0) + static_cast<float>(s1)) + (static_cast<float>(s2) + static_cast<float>(s3));
 #pragma unroll
-                            for (int o = 16; o > 0; o >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, o);
+                                for (int o = 16; o > 0; o >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, o);
+                                wtot = static_cast<double>(tot);
+                            } else {
+                                wtot = stat_op_finish<ST>(warp_combine<ST>(fold4<ST>(s0, s1, s2, s3)));
+                            }
                             float v_old = lane == 0 ? v_src[b] : 0.f;
                             v_old = __shfl_sync(0xffffffffu, v_old, 0);
                             float vn;
-                            const float step = stream_block_step(static_cast<double>(tot) * gscale_sq, mt.inv_L, v_old, P.sc, &vn);
+                            const float step = stream_block_step(wtot * gscale_sq, mt.inv_L, v_old, P.sc, &vn);
                             if (lane == 0) mt.v[b] = vn;
                             if (bf16) apply_span<AM_BF16, COPY, CLUSTER>(gs, ms, ps, mt.m, mt.p, mt.pb, e, L, lane, 32, beta1, omb1, lr_wd, step);
                             else apply_span<AM_F32, COPY, CLUSTER>(gs, ms, ps, mt.m, mt.p, mt.pb, e, L, lane, 32, beta1, omb1, lr_wd, step);
@@ -624,16 +710,16 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                     } else {
                         for (int b = 0; b < nb && alive; ++b) {
                             const int e = b * L;
-                            float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-                            if (bf16) sum_span<AM_BF16>(gs, e, L, gtid, nthr, s0, s1, s2, s3);
-                            else sum_span<AM_F32>(gs, e, L, gtid, nthr, s0, s1, s2, s3);
+                            Acc s0 = stat_acc_init<ST>(), s1 = s0, s2 = s0, s3 = s0;
+                            if (bf16) sum_span<AM_BF16, ST>(gs, e, L, gtid, nthr, s0, s1, s2, s3);
+                            else sum_span<AM_F32, ST>(gs, e, L, gtid, nthr, s0, s1, s2, s3);
                             double tot;
                             float v_old;
-                            alive = group_reduce(ctl, gsync, P.error_word, group, gtid, n_gwarps, fold4(s0, s1, s2, s3),
-                                                 v_src + b, &tot, &v_old);
+                            alive = group_reduce<ST>(ctl, gsync, P.error_word, P.wait_limit_ns, group, gtid, n_gwarps, fold4<ST>(s0, s1, s2, s3),
+                                                     v_src + b, &tot, &v_old);
                             if (!alive) break;
                             float vn;
-                            const float step = stream_block_step(tot * gscale_sq, mt.inv_L, v_old, P.sc, &vn);
+                            const float step = stream_block_step(stat_op_finish<ST>(tot) * gscale_sq, mt.inv_L, v_old, P.sc, &vn);
                             if (gtid == 0) mt.v[b] = vn;
                             if (bf16) apply_span<AM_BF16, COPY, CLUSTER>(gs, ms, ps, mt.m, mt.p, mt.pb, e, L, gtid, nthr, beta1, omb1, lr_wd, step);
                             else apply_span<AM_F32, COPY, CLUSTER>(gs, ms, ps, mt.m, mt.p, mt.pb, e, L, gtid, nthr, beta1, omb1, lr_wd, step);
@@ -643,19 +729,19 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&ctl->empty[stage]);
                 } else if (mt.kind == STAGE_SUM) {
-                    if (bf16) sum_span<AM_BF16>(gs, 0, mt.n, gtid, nthr, a0, a1, a2, a3);
-                    else sum_span<AM_F32>(gs, 0, mt.n, gtid, nthr, a0, a1, a2, a3);
+                    if (bf16) sum_span<AM_BF16, ST>(gs, 0, mt.n, gtid, nthr, a0, a1, a2, a3);
+                    else sum_span<AM_F32, ST>(gs, 0, mt.n, gtid, nthr, a0, a1, a2, a3);
                     if (!last_sum) {
                         __syncwarp();
                         if (lane == 0) mbar_arrive(&ctl->empty[stage]);
                     } else {
                         double tot;
                         float v_old;
-                        if (!group_reduce(ctl, gsync, P.error_word, group, gtid, n_gwarps, fold4(a0, a1, a2, a3), v_src, &tot, &v_old))
+                        if (!group_reduce<ST>(ctl, gsync, P.error_word, P.wait_limit_ns, group, gtid, n_gwarps, fold4<ST>(a0, a1, a2, a3), v_src, &tot, &v_old))
                             break;
                         __syncwarp();                       // the stage (and its v area) has been read
                         if (lane == 0) mbar_arrive(&ctl->empty[stage]);
-                        a0 = a1 = a2 = a3 = 0.f;
+                        a0 = a1 = a2 = a3 = stat_acc_init<ST>();
                         if (CLUSTER) {
                             // Exchange the CTAs' sums through distributed shared memory.  Every CTA of
                             // the cluster walks the same blocks in the same order, so block number
@@ -671,13 +757,13 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                                     mbar_arrive_remote(map_to_rank(bar, r));
                                 }
                             }
-                            if (!wait_phase<true>(&ctl->xbar[slot], (long_seen / kExchangeSlots) & 1u, ctl, P.error_word, 4)) break;
-                            tot = 0.0;
-                            for (uint32_t r = 0; r < csize; ++r) tot += ctl->xpart[slot][r];
+                            if (!wait_phase<true>(&ctl->xbar[slot], (long_seen / kExchangeSlots) & 1u, ctl, P.error_word, 4, P.wait_limit_ns)) break;
+                            tot = ctl->xpart[slot][0];
+                            for (uint32_t r = 1; r < csize; ++r) tot = stat_op_combine<ST>(tot, ctl->xpart[slot][r]);
                         }
                         ++long_seen;
                         float vn;
-                        long_step = stream_block_step(tot * gscale_sq, mt.inv_L, v_old, P.sc, &vn);
+                        long_step = stream_block_step(stat_op_finish<ST>(tot) * gscale_sq, mt.inv_L, v_old, P.sc, &vn);
                         if (gtid == 0 && (mt.flags & SF_WRITE_V)) *mt.v = vn;
                     }
                 } else {   // STAGE_APPLY
@@ -691,12 +777,25 @@ stream_kernel(const __grid_constant__ StreamParams P) {
         }
     }
     // common exit: nobody leaves a cluster while a peer may still write into it
-    if (CLUSTER) cluster_sync_all();
+    if (CLUSTER) {
+        __syncwarp();
+        cluster_sync_all();
+    }
 }
 
 // ------------------------------- host-side planning -------------------------------
+// What planning needs to know about the device (queried when a handle is created).
+struct DeviceCaps {
+    int sm_count = 0;
+    size_t smem_optin = 0;                  // most dynamic shared memory a CTA may ask for
+    int64_t l2_bytes = 0;
+    int resident[kMaxCluster + 1] = {};     // resident[c]: clusters of c CTAs of the streaming kernel the device
+                                            // keeps resident at once (0: such clusters cannot run)
+};
+
 struct StreamPlanInput {
-    int sm_count = 0, ctas = 0, cluster_size = 0, threads = 0, groups = 0, chunk = 0, cluster_chunk = 0;
+    DeviceCaps caps;
+    int ctas = 0, cluster_size = 0, threads = 0, groups = 0, chunk = 0, cluster_chunk = 0;
     struct Item { int tensor; am_table_row row; };
     std::vector<Item> stream_tensors, cluster_tensors;
 };
@@ -717,19 +816,31 @@ inline void stream_add_tensor(StreamPlanInput &in, int index, const am_table_row
 
 typedef void (*StreamKernelFn)(const StreamParams);
 
-template <bool CLUSTER>
+// One instantiation per use keeps the mean's consumer loop small; the ablation
+// statistics are compiled with the bf16-copy path in (taken only where a tensor has a copy).
+template <bool CLUSTER, int ST>
 inline StreamKernelFn stream_kernel_for(int gdm, bool copy) {
+    if (ST != ST_SUM) copy = true;
     switch (gdm * 2 + (copy ? 1 : 0)) {
-    case 0: return stream_kernel<CLUSTER, GDM_F32, false>;
-    case 1: return stream_kernel<CLUSTER, GDM_F32, true>;
-    case 2: return stream_kernel<CLUSTER, GDM_BF16, false>;
-    case 3: return stream_kernel<CLUSTER, GDM_BF16, true>;
-    case 4: return stream_kernel<CLUSTER, GDM_MIXED, false>;
-    default: return stream_kernel<CLUSTER, GDM_MIXED, true>;
+    case 0: return stream_kernel<CLUSTER, GDM_F32, ST != ST_SUM, ST>;
+    case 1: return stream_kernel<CLUSTER, GDM_F32, true, ST>;
+    case 2: return stream_kernel<CLUSTER, GDM_BF16, ST != ST_SUM, ST>;
+    case 3: return stream_kernel<CLUSTER, GDM_BF16, true, ST>;
+    case 4: return stream_kernel<CLUSTER, GDM_MIXED, ST != ST_SUM, ST>;
+    default: return stream_kernel<CLUSTER, GDM_MIXED, true, ST>;
     }
 }
-inline StreamKernelFn stream_kernel_for(bool cluster, int gdm, bool copy) {
-    return cluster ? stream_kernel_for<true>(gdm, copy) : stream_kernel_for<false>(gdm, copy);
+template <bool CLUSTER>
+inline StreamKernelFn stream_kernel_for(int gdm, bool copy, int st) {
+    switch (st) {
+    case ST_MAX: return stream_kernel_for<CLUSTER, ST_MAX>(gdm, copy);
+    case ST_MIN: return stream_kernel_for<CLUSTER, ST_MIN>(gdm, copy);
+    case ST_SUM4: return stream_kernel_for<CLUSTER, ST_SUM4>(gdm, copy);
+    default: return stream_kernel_for<CLUSTER, ST_SUM>(gdm, copy);
+    }
+}
+inline StreamKernelFn stream_kernel_for(bool cluster, int gdm, bool copy, int st) {
+    return cluster ? stream_kernel_for<true>(gdm, copy, st) : stream_kernel_for<false>(gdm, copy, st);
 }
 
 struct StreamLaunch {
@@ -743,8 +854,6 @@ struct StreamLaunch {
     bool active() const { return grid > 0; }
     size_t smem_bytes() const { return kCtrlBytes + static_cast<size_t>(n_stages) * (stage_bytes + kVAreaFloats * 4); }
 };
-
-constexpr size_t kSmemBudget = 227 * 1024;
 
 struct StreamPlan {
     StreamLaunch main, clus;
@@ -775,6 +884,8 @@ struct StreamPlan {
 
     int64_t v_len = 0;
     bool bf16_copies = false;      // set per step: some tensor has a bf16 copy to write
+    unsigned long long wait_limit_ns = kWaitTimeoutNs;
+    int stall_after = 0;
 
     cudaError_t launch_one(const StreamLaunch &L, bool cluster, const DevTensor *tensors, float *v,
                            const StepScalars &sc, int *error_word, cudaStream_t stream) const {
@@ -784,6 +895,7 @@ struct StreamPlan {
         P.stage_bytes = L.stage_bytes; P.g_region_bytes = L.g_region_bytes; P.consumer_threads = L.threads;
         P.n_groups = L.groups;
         P.v_len = v_len;
+        P.wait_limit_ns = wait_limit_ns; P.stall_after = stall_after; P.pad = 0;
         P.chunk = L.chunk; P.counter = L.d_counter; P.total_items = L.bounds.empty() ? 0 : L.bounds.back();
         if (P.chunk > 0) {
             cudaError_t e = cudaMemsetAsync(L.d_counter, 0, sizeof(unsigned long long), stream);
@@ -803,7 +915,7 @@ struct StreamPlan {
             cfg.attrs = attr;
             cfg.numAttrs = 1;
         }
-        return cudaLaunchKernelEx(&cfg, stream_kernel_for(cluster, L.gdm, bf16_copies), P);
+        return cudaLaunchKernelEx(&cfg, stream_kernel_for(cluster, L.gdm, bf16_copies, stat_op_of(sc.statistic)), P);
     }
 
     cudaError_t launch_main(const DevTensor *tensors, float *v, const StepScalars &sc, int *error_word,
@@ -816,9 +928,18 @@ struct StreamPlan {
     }
 };
 
+// Shared-memory layout of a launch: a stage holds kStageElems gradients (2 or 4 bytes each), first
+// moments and parameters; as many stages as the CTA's shared memory allows.
+inline void stream_stage_layout(bool any_f32, size_t smem_optin, int *g_region_bytes, int *stage_bytes, int *n_stages) {
+    *g_region_bytes = kStageElems * (any_f32 ? 4 : 2);
+    *stage_bytes = *g_region_bytes + kStageElems * 8;
+    const size_t per_stage = static_cast<size_t>(*stage_bytes) + kVAreaFloats * 4;
+    *n_stages = smem_optin > kCtrlBytes ? std::min<int>(kMaxStages, static_cast<int>((smem_optin - kCtrlBytes) / per_stage)) : 0;
+}
+
 // Build segment tables and balanced item ranges for one launch.
 inline void stream_build_launch(const std::vector<StreamPlanInput::Item> &tensors, bool cluster, int workers,
-                                StreamLaunch *out) {
+                                size_t smem_optin, StreamLaunch *out) {
     out->segs.clear();
     out->bounds.clear();
     out->grid = 0;
@@ -829,9 +950,7 @@ inline void stream_build_launch(const std::vector<StreamPlanInput::Item> &tensor
         any_bf16 |= it.row.grad_dtype == AM_BF16;
     }
     out->gdm = any_f32 && any_bf16 ? GDM_MIXED : (any_bf16 ? GDM_BF16 : GDM_F32);
-    out->g_region_bytes = kStageElems * (any_f32 ? 4 : 2);
-    out->stage_bytes = out->g_region_bytes + kStageElems * 8;
-    out->n_stages = std::min<int>(kMaxStages, static_cast<int>((kSmemBudget - kCtrlBytes) / (out->stage_bytes + kVAreaFloats * 4)));
+    stream_stage_layout(any_f32, smem_optin, &out->g_region_bytes, &out->stage_bytes, &out->n_stages);
 
     std::vector<double> item_cost;      // per segment
     int64_t slots = 0, n_items = 0;
@@ -897,17 +1016,18 @@ inline void stream_build_launch(const std::vector<StreamPlanInput::Item> &tensor
     out->grid = workers;
 }
 
-// Largest cluster size (<= wanted) the device can keep resident with this
-// kernel's shared memory, and how many such clusters fit at once.
-inline void stream_probe_cluster(int sm_count, int consumer_threads, int wanted, int *cluster_size, int *n_clusters) {
-    *cluster_size = 0;
-    *n_clusters = 0;
-    const int threads = consumer_threads > 0 ? consumer_threads : 512;
-    const size_t smem = kCtrlBytes + 5 * (kStageElems * 10 + kVAreaFloats * 4);   // the larger of the two stage layouts
-    for (int cs = wanted > 0 ? wanted : kMaxCluster; cs >= 1; cs >>= 1) {
+// How many clusters of every size the device keeps resident at once, for CTAs of
+// `block_threads` threads with the larger of the two stage layouts.
+inline void stream_probe_clusters(DeviceCaps *caps, int block_threads) {
+    int g_region, stage_bytes, n_stages;
+    stream_stage_layout(true, caps->smem_optin, &g_region, &stage_bytes, &n_stages);
+    const size_t smem = kCtrlBytes + static_cast<size_t>(n_stages) * (stage_bytes + kVAreaFloats * 4);
+    for (int cs = 1; cs <= kMaxCluster; ++cs) {
+        caps->resident[cs] = 0;
+        if (n_stages < 2) continue;
         cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(std::max(sm_count / cs, 1) * cs);
-        cfg.blockDim = dim3(32 + threads);
+        cfg.gridDim = dim3(std::max(caps->sm_count / cs, 1) * cs);
+        cfg.blockDim = dim3(block_threads);
         cfg.dynamicSmemBytes = smem;
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -917,13 +1037,46 @@ inline void stream_probe_cluster(int sm_count, int consumer_threads, int wanted,
         cfg.attrs = attr;
         cfg.numAttrs = 1;
         int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, stream_kernel<true, GDM_MIXED, true>, &cfg) == cudaSuccess && n > 0) {
-            *cluster_size = cs;
-            *n_clusters = n;
-            return;
-        }
-        (void)cudaGetLastError();
+        if (cudaOccupancyMaxActiveClusters(&n, stream_kernel<true, GDM_MIXED, true, ST_SUM>, &cfg) == cudaSuccess && n > 0)
+            caps->resident[cs] = n;
+        else
+            (void)cudaGetLastError();
     }
+}
+
+// Cluster size for head-sized blocks whose gradients take `block_bytes`.
+//
+// A cluster reads a block's gradients twice (to reduce them, then to apply the
+// update), and the second read should find them in L2.  Every resident cluster
+// has one block between its two reads, so resident[c] * block_bytes is what L2
+// must keep besides the m and p streaming through it.  Smaller clusters mean
+// more clusters, which use more SMs but keep more in L2: the choice is the
+// smallest size whose in-flight gradients stay within kL2ShareForHeads of L2,
+// or the largest size that can run when none does.  A size that keeps no more
+// clusters resident than a larger one is passed over (it only idles SMs).
+//
+// kL2ShareForHeads is a measured boundary, not a derived one (B200, 126 MB of
+// L2 in two halves, resident = 148/74/45/33/26/22/15/15 for sizes 1..8): 45
+// clusters x 1 MB ran at 0.94 of the copy bandwidth against 0.97 for 33 x 1 MB,
+// and 22 x 2 MB at 0.95 against 0.93 for 33 x 2 MB; 74 x 0.31 MB and 45 x 0.5 MB
+// (1.01 and 0.99) beat the clusters of 4 that a fixed rule had given them (0.83
+// and 0.93).
+constexpr double kL2ShareForHeads = 0.353;
+
+inline int choose_cluster_size(const int *resident, int64_t l2_bytes, int64_t block_bytes) {
+    int largest = 0;
+    for (int c = 1; c <= kMaxCluster; ++c)
+        if (resident[c] > 0) largest = c;
+    if (largest == 0) return 0;
+    const double room = kL2ShareForHeads * static_cast<double>(l2_bytes);
+    for (int c = 1; c < largest; ++c) {
+        if (resident[c] <= 0) continue;
+        bool passed_over = false;
+        for (int d = c + 1; d <= largest; ++d) passed_over |= resident[d] >= resident[c];
+        if (passed_over) continue;
+        if (static_cast<double>(resident[c]) * static_cast<double>(block_bytes) <= room) return c;
+    }
+    return largest;
 }
 
 // Consumer groups and threads per group of a launch (0 = defaults: two groups of 256).
@@ -933,11 +1086,11 @@ inline void stream_consumer_shape(int threads_opt, int groups_opt, int *threads,
     while (*threads * *groups > kMaxConsumerWarps * 32) *threads -= 32;
 }
 
-inline void stream_finish_plan(const StreamPlanInput &in, int cluster_size, int n_clusters, StreamPlan *plan) {
+inline void stream_finish_plan(const StreamPlanInput &in, StreamPlan *plan) {
     int threads, groups;
     stream_consumer_shape(in.threads, in.groups, &threads, &groups);
-    const int ctas = in.ctas > 0 ? in.ctas : in.sm_count;
-    stream_build_launch(in.stream_tensors, false, ctas, &plan->main);
+    const int ctas = in.ctas > 0 ? in.ctas : in.caps.sm_count;
+    stream_build_launch(in.stream_tensors, false, ctas, in.caps.smem_optin, &plan->main);
     plan->main.threads = threads;
     plan->main.groups = groups;
     plan->main.cluster = 1;
@@ -952,42 +1105,43 @@ inline void stream_finish_plan(const StreamPlanInput &in, int cluster_size, int 
                                : static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(64, items / (int64_t(32) * std::max(ctas, 1)))));
     }
     plan->clus = StreamLaunch();
-    if (!in.cluster_tensors.empty() && n_clusters > 0) {
-        // Launch shape for head-sized blocks.  Measured on B200: blocks of up to 1 MB of
-        // gradients (bf16 heads of 128 x 4096) run best on clusters of 4 that take one block
-        // at a time from the shared counter (33 clusters fit), blocks of up to 2 MB (the same
-        // heads with float32 gradients) on clusters of 6 (22 fit) that do the same, larger
-        // blocks on clusters of 8 (15 fit) with fixed ranges: more clusters use more SMs but keep
-        // more gradients in L2 between their two fetches.
-        int64_t max_block_bytes = 0;
-        for (const auto &it : in.cluster_tensors)
-            max_block_bytes = std::max(max_block_bytes, it.row.block_len * (it.row.grad_dtype == AM_BF16 ? 2 : 4));
-        const int preferred = max_block_bytes <= (int64_t(1) << 20) ? 4 : max_block_bytes <= (int64_t(2) << 20) ? 6 : 8;
-        int chunk = in.cluster_chunk;
-        if (in.cluster_size == 0 && preferred < cluster_size) {
-            int cs = 0, n = 0;
-            stream_probe_cluster(in.sm_count, threads * groups, preferred, &cs, &n);
-            if (cs == preferred && n > 0) { cluster_size = cs; n_clusters = n; }
-        }
-        if (chunk == 0) chunk = (in.cluster_size == 0 && cluster_size == 8) ? kStaticRanges : 1;
-        stream_build_launch(in.cluster_tensors, true, n_clusters, &plan->clus);
-        plan->clus.grid *= cluster_size;          // bounds are per cluster
-        plan->clus.cluster = cluster_size;
-        plan->clus.threads = threads;
-        plan->clus.groups = in.groups > 0 ? groups : 1;     // measured: a second group does not help the head kernel
-        plan->clus.chunk = chunk == kStaticRanges ? 0 : chunk;
+    if (in.cluster_tensors.empty()) return;
+    // Launch shape for head-sized blocks: the cluster size follows from the largest block, the L2
+    // size and how many clusters of each size fit the device (choose_cluster_size), unless the
+    // caller fixed it (then the largest size up to the caller's that can run).  Clusters take one
+    // block at a time from the shared counter; clusters of the largest size, which hold the
+    // biggest blocks, walk fixed ranges (measured).
+    int64_t max_block_bytes = 0;
+    for (const auto &it : in.cluster_tensors)
+        max_block_bytes = std::max(max_block_bytes, it.row.block_len * (it.row.grad_dtype == AM_BF16 ? 2 : 4));
+    int cluster_size = 0;
+    if (in.cluster_size > 0) {
+        for (int c = std::min(in.cluster_size, kMaxCluster); c >= 1 && cluster_size == 0; --c)
+            if (in.caps.resident[c] > 0) cluster_size = c;
+    } else {
+        cluster_size = choose_cluster_size(in.caps.resident, in.caps.l2_bytes, max_block_bytes);
     }
+    if (cluster_size == 0) return;
+    int chunk = in.cluster_chunk;
+    if (chunk == 0) chunk = (in.cluster_size == 0 && cluster_size == kMaxCluster) ? kStaticRanges : 1;
+    stream_build_launch(in.cluster_tensors, true, in.caps.resident[cluster_size], in.caps.smem_optin, &plan->clus);
+    plan->clus.grid *= cluster_size;          // bounds are per cluster
+    plan->clus.cluster = cluster_size;
+    plan->clus.threads = threads;
+    plan->clus.groups = in.groups > 0 ? groups : 1;     // measured: a second group does not help the head kernel
+    plan->clus.chunk = chunk == kStaticRanges ? 0 : chunk;
 }
 
-inline cudaError_t stream_configure_kernels() {
+inline cudaError_t stream_configure_kernels(size_t smem_optin) {
     for (int cluster = 0; cluster < 2; ++cluster)
         for (int gdm = 0; gdm < 3; ++gdm)
-            for (int copy = 0; copy < 2; ++copy) {
-                const cudaError_t e = cudaFuncSetAttribute(stream_kernel_for(cluster != 0, gdm, copy != 0),
-                                                           cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                           static_cast<int>(kSmemBudget));
-                if (e != cudaSuccess) return e;
-            }
+            for (int copy = 0; copy < 2; ++copy)
+                for (int st = 0; st < 4; ++st) {
+                    const cudaError_t e = cudaFuncSetAttribute(stream_kernel_for(cluster != 0, gdm, copy != 0, st),
+                                                               cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                               static_cast<int>(smem_optin));
+                    if (e != cudaSuccess) return e;
+                }
     return cudaSuccess;
 }
 

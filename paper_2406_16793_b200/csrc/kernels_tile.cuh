@@ -105,9 +105,11 @@ __device__ __forceinline__ void tile_body(const DevTensor &t, int64_t tile, floa
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         if (nbulk > 0) {
             mbar_arrive_expect_tx(bar, static_cast<uint32_t>(nbulk) * (gsz + 8));
-            bulk_load(sraw + (shift + head) * gsz, gg + head * gsz, nbulk * gsz, bar);
-            bulk_load(sm + shift + head, mg + head, nbulk * 4, bar);
-            bulk_load(sp + shift + head, pg + head, nbulk * 4, bar);
+            if (!sc.stall) {        // (test hook: bytes announced that never arrive make the wait below run out)
+                bulk_load(sraw + (shift + head) * gsz, gg + head * gsz, nbulk * gsz, bar);
+                bulk_load(sm + shift + head, mg + head, nbulk * 4, bar);
+                bulk_load(sp + shift + head, pg + head, nbulk * 4, bar);
+            }
         }
     }
     // the ends, by plain loads
@@ -150,14 +152,15 @@ __device__ __forceinline__ void tile_body(const DevTensor &t, int64_t tile, floa
                     waited += gap < kWaitGapCapNs ? gap : kWaitGapCapNs;
                 }
                 last = now;
-                if (waited > kWaitTimeoutNs) { ok = false; break; }
+                if (waited > sc.wait_limit_ns) { ok = false; break; }
             }
         }
         if (!ok) {
             // give up: report, let the copies land (again bounded) before the CTA's memory is released, leave
             *reinterpret_cast<volatile int *>(error_word) = kTileTimeoutCode;
             const unsigned long long t0 = global_ns();
-            while (!mbar_try_wait(bar, 0) && global_ns() - t0 < kDrainTimeoutNs) {}
+            const unsigned long long drain = sc.wait_limit_ns < kDrainTimeoutNs ? sc.wait_limit_ns : kDrainTimeoutNs;
+            while (!mbar_try_wait(bar, 0) && global_ns() - t0 < drain) {}
             return;
         }
     }

@@ -165,6 +165,23 @@ class DeviceState:
         return all(g.intact() for g in self.guards)
 
 
+def mixed_workload():
+    """Every kernel family at once: tiny blocks, packed rows, long rows, a clustered head, a two-pass block."""
+    T = W.TensorSpec
+    bf = dict(grad_dtype=W.BF16)
+    tensors = [
+        T("tiny", 1, 4096, W.FIXED, fixed_block_len=1, **bf),
+        T("rows", 96, 4096, W.ROWS, **bf),
+        T("short", 300, 768, W.ROWS, **bf),
+        T("long", 24, 11008, W.ROWS, **bf),
+        T("head", 256, 4096, W.HEADS, n_heads=2, **bf),
+        T("whole", 1, 3 << 20, W.WHOLE, **bf),
+        T("odd", 5, 1001, W.ROWS, **bf),
+        T("f32rows", 64, 512, W.ROWS, grad_dtype=W.F32),
+    ]
+    return W.Workload("mixed", 61, tensors, W.GradRecipe(-4.0, -1.0), steps=3)
+
+
 def make_optimizer(w: W.Workload, options: Optional[Dict[int, int]] = None, **hp) -> am.AdamMini:
     part = am.Partition(w.tensors)
     opt = am.AdamMini(part, **{**w.hparams, **hp})
@@ -189,18 +206,19 @@ def oracle_step_all(state: ostep.OracleState, grads_cpu: Sequence, step: int, hp
 
 def run_parity(w: W.Workload, steps: Optional[int] = None, options: Optional[Dict[int, int]] = None,
                device="cuda", hp_override: Optional[Dict[str, float]] = None, mutate_grads=None,
-               lr_schedule=None, statistic: int = 0) -> Dict[str, float]:
+               lr_schedule=None, statistic: int = 0, optimizer: Optional[am.AdamMini] = None) -> Dict[str, float]:
     """Run `steps` steps on the GPU and in the oracle; returns the worst errors.
 
     mutate_grads(step, list_of_device_grads) may edit the gradients in place
-    (zero rows, infinities) before both sides consume them.
+    (zero rows, infinities) before both sides consume them.  `optimizer`: step
+    with this handle (made for `w`) instead of a new one; it is left open.
     """
     steps = steps or w.steps
     hp = {**w.hparams, **(hp_override or {})}
     dev = DeviceState(w, device)
     if statistic:
         options = {**(options or {}), am.binding.OPT_STATISTIC: statistic}
-    opt = make_optimizer(w, options, **(hp_override or {}))
+    opt = optimizer or make_optimizer(w, options, **(hp_override or {}))
     ora = ostep.OracleState([p.cpu() for p in dev.p], [t.block_len for t in w.tensors],
                             [bool(t.apply_weight_decay) for t in w.tensors])
     unit = {i: ShortBlockScale(ora.p[i]) for i, t in enumerate(w.tensors)
@@ -239,7 +257,8 @@ def run_parity(w: W.Workload, steps: Optional[int] = None, options: Optional[Dic
                                       f" g={float(ostep.widen(grads_cpu[i][k:k + 1])[0]):.3e}")
         worst["v"] = max(worst["v"], v_relative_error(v_gpu[off:off + t.n_blocks], ora.v[i]))
         off += t.n_blocks
-    opt.close()
+    if optimizer is None:
+        opt.close()
     return worst
 
 

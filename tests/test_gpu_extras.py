@@ -12,21 +12,7 @@ from test_gpu_parity import ragged_workload, _same
 pytestmark = pytest.mark.gpu
 
 
-def mixed_workload():
-    """Every kernel family at once: tiny blocks, packed rows, long rows, a clustered head, a two-pass block."""
-    T = W.TensorSpec
-    bf = dict(grad_dtype=W.BF16)
-    tensors = [
-        T("tiny", 1, 4096, W.FIXED, fixed_block_len=1, **bf),
-        T("rows", 96, 4096, W.ROWS, **bf),
-        T("short", 300, 768, W.ROWS, **bf),
-        T("long", 24, 11008, W.ROWS, **bf),
-        T("head", 256, 4096, W.HEADS, n_heads=2, **bf),
-        T("whole", 1, 3 << 20, W.WHOLE, **bf),
-        T("odd", 5, 1001, W.ROWS, **bf),
-        T("f32rows", 64, 512, W.ROWS, grad_dtype=W.F32),
-    ]
-    return W.Workload("mixed", 61, tensors, W.GradRecipe(-4.0, -1.0), steps=3)
+mixed_workload = H.mixed_workload
 
 
 def test_bf16_copy_is_the_rounded_parameter():
@@ -137,6 +123,38 @@ def test_ablation_statistics(statistic, grad_dtype):
     H.assert_parity(H.run_parity(ragged_workload(grad_dtype), steps=4, statistic=statistic))
 
 
-def test_ablation_statistics_on_model_shapes():
+@pytest.mark.parametrize("statistic", [B.STAT_MAX, B.STAT_MIN, B.STAT_ONE_NORM, B.STAT_TWO_NORM],
+                         ids=["max", "min", "one-norm", "two-norm"])
+def test_ablation_statistics_on_model_shapes(statistic):
+    """Llama-2-7B block lengths: the statistic is a parameter of the single-read
+    reductions (packed rows, long rows re-read from L2, heads on clusters with the
+    exchange through distributed shared memory), so nothing falls back to the
+    two-pass kernels."""
     w = W.scaled_rows(W.llama2_7b(n_layers=1, vocab=128), 128)
-    H.assert_parity(H.run_parity(w, steps=3, statistic=B.STAT_TWO_NORM))
+    opt = H.make_optimizer(w, {B.OPT_STATISTIC: statistic})
+    assert opt.query(B.Q_ELEMENTS_TWOPASS) == 0 and opt.query(B.Q_ELEMENTS_CLUSTER) == 2 * 128 * 4096
+    assert opt.query(B.Q_LAUNCHES_PER_STEP) == 2
+    opt.close()
+    H.assert_parity(H.run_parity(w, steps=3, statistic=statistic))
+
+
+def test_ablation_statistics_with_float32_heads_and_a_gradient_scale():
+    """float32 gradients on clusters of six, consumer groups of other sizes, and a
+    gradient scale that must come out as scale^2 on every statistic of g*g."""
+    T = W.TensorSpec
+    w = W.Workload("stat-f32", 66, [T("q", 256, 4096, W.HEADS, n_heads=2), T("rows", 40, 11008, W.ROWS),
+                                    T("packed", 100, 2048, W.ROWS)], W.GradRecipe(-4.0, -1.0), steps=2)
+    for statistic in (B.STAT_MAX, B.STAT_TWO_NORM):
+        H.assert_parity(H.run_parity(w, statistic=statistic, options={B.OPT_STREAM_THREADS: 128}))
+    a, b = H.DeviceState(w, guarded=False), H.DeviceState(w, guarded=False)
+    oa = H.make_optimizer(w, {B.OPT_STATISTIC: B.STAT_MIN})
+    ob = H.make_optimizer(w, {B.OPT_STATISTIC: B.STAT_MIN})
+    for t in (1, 2):
+        a.draw_grads(t)
+        for x, y in zip(a.g, b.g):
+            y.copy_(x * 0.25)
+        oa.step_ex(a.p, a.g, a.m, a.v, t, grad_scale=0.25)
+        ob.step(b.p, b.g, b.m, b.v, t)
+    oa.sync_status(); ob.sync_status()
+    assert _same(a, b)
+    oa.close(); ob.close()

@@ -225,6 +225,28 @@ def test_launch_options_are_validated():
     assert _same(ref, dev)
 
 
+def test_cluster_shape_follows_the_device():
+    """The cluster size of a table is what the chooser gives for the properties the handle
+    read from this device; on a B200 (148 SMs, 126 MB of L2) that is 33 clusters of 4 for
+    bf16 heads of 128 x 4096 and 22 clusters of 6 for the same heads with float32 gradients."""
+    for gd, block_bytes, on_b200 in ((W.BF16, 1 << 20, (33, 4)), (W.F32, 2 << 20, (22, 6))):
+        w = W.Workload("heads", 78, [W.TensorSpec("q", 8192, 4096, W.HEADS, n_heads=64, grad_dtype=gd)],
+                       W.GradRecipe(-5.0, -1.0), steps=1)
+        opt = H.make_optimizer(w)
+        resident = [0] + [opt.query(B.Q_RESIDENT_CLUSTERS + c - 1) for c in range(1, 9)]
+        l2, smem = opt.query(B.Q_L2_BYTES), opt.query(B.Q_SMEM_BYTES)
+        want = B.choose_cluster_size(resident, l2, block_bytes)
+        assert want >= 1 and opt.query(B.Q_CLUSTER_SIZE) == want
+        assert opt.query(B.Q_CLUSTER_COUNT) == min(resident[want], w.n_blocks)
+        props = torch.cuda.get_device_properties(0)
+        assert l2 == props.L2_cache_size and smem >= 48 * 1024
+        if "B200" in props.name and props.multi_processor_count == 148:
+            assert (opt.query(B.Q_CLUSTER_COUNT), opt.query(B.Q_CLUSTER_SIZE)) == on_b200, (resident, l2)
+        opt.set_option(B.OPT_CLUSTER_SIZE, 7)               # a caller's size is kept when it can run
+        assert opt.query(B.Q_CLUSTER_SIZE) == max(c for c in range(1, 8) if resident[c] > 0)
+        opt.close()
+
+
 def test_empty_partition_and_queries():
     opt = am.AdamMini(am.Partition([]))
     opt.step([], [], [], 0, 1)
@@ -354,9 +376,11 @@ def test_full_size_flat_sweep_sampled_blocks(L):
 
 def test_full_size_whole_tensor_block():
     """2^30 elements as ONE block (the two-pass path at full size): the oracle
-    runs the whole tensor for two steps."""
+    runs the whole tensor for the ten steps of the partition-degeneracy sweep."""
     _need_free_memory(20)
-    H.assert_parity(H.run_parity(W.flat_sweep(1 << 30), steps=2))
+    w = W.flat_sweep(1 << 30)
+    assert w.steps == 10
+    H.assert_parity(H.run_parity(w))
 
 
 @pytest.mark.parametrize("world", [2, 3])
