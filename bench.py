@@ -100,7 +100,9 @@ def pick_workload(name: str):
         return table[name]()
     if name.startswith("flat-L"):                      # flat-L<block length>[-n<log2 of the element count>]
         parts = name[6:].split("-n")
-        return W.flat_sweep(int(parts[0]), numel=1 << (int(parts[1]) if len(parts) > 1 else 30))
+        L, numel = int(parts[0]), 1 << (int(parts[1]) if len(parts) > 1 else 30)
+        unit = 64 * L if 64 % L else 64                                # whole blocks and whole 64-element chunks of one sigma
+        return W.flat_sweep(L, numel=numel // unit * unit)
     if name.startswith("llama2-7b-layers"):
         return W.llama2_7b(n_layers=int(name[len("llama2-7b-layers"):]))
     if name.startswith("rows-"):                        # rows-<bf16|f32>-L<row length>-r<rows>: one matrix, a block per row

@@ -111,11 +111,12 @@ int build_plan(am_handle *h) {
         const int64_t gsz = r.grad_dtype == AM_BF16 ? 2 : 4;
 
         int path;
+        bool edges = false;
         if (r.kind == AM_PART) path = PATH_TWOPASS;          // its sum of squares comes from outside
         else if (r.block_len <= kSmallMaxL && !(h->opt[AM_OPT_PATH] == 1 && r.block_len > 16)) path = PATH_SMALL;
         else if (h->opt[AM_OPT_PATH] == 1) path = PATH_TWOPASS;
         else {
-            path = stream_ok ? stream_classify(r.block_len, r.grad_dtype, clusters_ok) : PATH_TWOPASS;
+            path = stream_ok ? stream_classify(r.block_len, r.grad_dtype, clusters_ok, &edges) : PATH_TWOPASS;
             // block starts off the 16-byte grid: the tile kernel copes, up to its tile size
             if (path == PATH_TWOPASS && r.block_len <= kTileMaxL) path = PATH_SMALL;
         }
@@ -132,10 +133,10 @@ int build_plan(am_handle *h) {
         if (path == PATH_SMALL) {
             Seg s;
             s.tensor = i;
-            s.aux = (r.block_len == 1 && r.v_offset % 4 == 0 && r.numel % 4 == 0) ? 1 : 0;
-            if (s.aux) {                // the AdamW case: four one-element blocks per thread
+            s.aux = small_vec_ok(r.block_len, r.numel, r.v_offset) ? 1 : 0;
+            if (s.aux) {                // blocks of one to three elements, aligned: straight from registers
                 s.unit_begin = small_units;
-                small_units += ceil_div(r.numel, kSmallUnitVec);
+                small_units += ceil_div(r.numel, small_vec_unit(r.block_len));
                 small_segs.push_back(s);
             } else {                    // tiles of whole blocks staged in shared memory
                 s.unit_begin = tile_units;
@@ -180,10 +181,29 @@ int build_plan(am_handle *h) {
             piece_units += r.n_blocks * ppb;
             block_units += r.n_blocks;
         } else {
-            stream_add_tensor(sin, i, r, path);
+            stream_add_tensor(sin, i, r, path, edges);
         }
     }
     if (part_units > 0x7fffffffLL || wide_units > 0x7fffffffLL) return AM_ERR_TOO_LARGE;
+    // Segments of the register kernel by block length (one launch per length present).
+    int64_t small_units_by_len[kSmallVecMaxL + 1] = {};
+    {
+        std::vector<Seg> ordered;
+        int64_t next = 0;
+        for (int len = 1; len <= kSmallVecMaxL; ++len) {
+            const int64_t begin = next;
+            for (const Seg &sg : small_segs) {
+                const am_table_row &r = h->rows[sg.tensor];
+                if (r.block_len != len) continue;
+                Seg o = sg;
+                o.unit_begin = next;
+                next += ceil_div(r.numel, small_vec_unit(len));
+                ordered.push_back(o);
+            }
+            small_units_by_len[len] = next - begin;
+        }
+        small_segs.swap(ordered);
+    }
     // Tiles of short blocks first, then those of longer ones: the two kinds are launched
     // separately, each with the shared-memory layout it needs (four CTAs per SM for both).
     int64_t tile_short_units = 0;
@@ -254,6 +274,7 @@ int build_plan(am_handle *h) {
         AM_CUDA(h, cudaMemcpy(h->d_part_tensors, part_tensors.data(), sizeof(int32_t) * part_tensors.size(), cudaMemcpyHostToDevice));
     }
     h->small_units = small_units;
+    for (int len = 1; len <= kSmallVecMaxL; ++len) h->small_units_by_len[len] = small_units_by_len[len];
     h->piece_units = piece_units;
     h->block_units = block_units;
     if (!small_segs.empty())
@@ -269,7 +290,7 @@ int build_plan(am_handle *h) {
         if (e != cudaSuccess) return cuda_fail(h, e);
     }
 
-    h->launches = (small_units ? 1 : 0) + (tile_short_units ? 1 : 0) + (tile_units > tile_short_units ? 1 : 0) + (piece_units ? 3 : 0) + (wide_units ? 1 : 0) + sp.launches();
+    h->launches = (small_units_by_len[1] ? 1 : 0) + (small_units_by_len[2] ? 1 : 0) + (small_units_by_len[3] ? 1 : 0) + (tile_short_units ? 1 : 0) + (tile_units > tile_short_units ? 1 : 0) + (piece_units ? 3 : 0) + (wide_units ? 1 : 0) + sp.launches();
     h->planned = true;
     return AM_OK;
 }
@@ -543,10 +564,16 @@ int adammini_step_ex(am_handle *h, void *const *params, const void *const *grads
         ss.statistic = sc.statistic;
         ss.stall = h->opt[AM_OPT_TEST_STALL] != 0;
         ss.wait_limit_ns = wait_limit_ns;
-        if (h->small_units) {
-            small_kernel<<<static_cast<unsigned>(h->small_units), kThreads, 0, stream>>>(
-                h->d_tensors, h->d_small_segs, h->n_small_segs, v, ss);
+        int64_t first = 0;
+        for (int len = 1; len <= kSmallVecMaxL; ++len) {
+            const int64_t units = h->small_units_by_len[len];
+            if (!units) continue;
+            const unsigned grid = static_cast<unsigned>(units);
+            if (len == 1) small_kernel<1><<<grid, kThreads, 0, stream>>>(h->d_tensors, h->d_small_segs, h->n_small_segs, v, ss, first);
+            else if (len == 2) small_kernel<2><<<grid, kThreads, 0, stream>>>(h->d_tensors, h->d_small_segs, h->n_small_segs, v, ss, first);
+            else small_kernel<3><<<grid, kThreads, 0, stream>>>(h->d_tensors, h->d_small_segs, h->n_small_segs, v, ss, first);
             AM_CUDA(h, cudaGetLastError());
+            first += units;
         }
         if (h->tile_units) {
             const int64_t n_short = h->tile_short_units, n_long = h->tile_units - n_short;
@@ -565,6 +592,7 @@ int adammini_step_ex(am_handle *h, void *const *params, const void *const *grads
     h->stream.bf16_copies = ex && ex->params_bf16;
     if (prof) AM_CUDA(h, cudaEventRecord(pev[1], stream));
     AM_CUDA(h, h->stream.launch_main(h->d_tensors, v, sc, h->error_word, stream));
+    AM_CUDA(h, h->stream.launch_edge(h->d_tensors, v, sc, h->error_word, stream));
     if (prof) AM_CUDA(h, cudaEventRecord(pev[2], stream));
     AM_CUDA(h, h->stream.launch_cluster(h->d_tensors, v, sc, h->error_word, stream));
     if (prof) AM_CUDA(h, cudaEventRecord(pev[3], stream));

@@ -30,6 +30,7 @@ struct am_handle {
     am::Seg *d_small_segs = nullptr, *d_piece_segs = nullptr, *d_block_segs = nullptr;
     int n_small_segs = 0, n_piece_segs = 0, n_block_segs = 0;
     int64_t small_units = 0, piece_units = 0, block_units = 0;
+    int64_t small_units_by_len[4] = {0, 0, 0, 0};   // units of the register kernel for block lengths 1, 2, 3 (index 0 unused)
     am::Seg *d_tile_segs = nullptr;      // short blocks handled a tile at a time
     int n_tile_segs = 0;
     int64_t tile_units = 0;

@@ -13,7 +13,7 @@ namespace am {
 
 constexpr int kThreads = 256;            // CTA size of the kernels in this file
 constexpr int kSmallMaxL = 64;           // blocks up to this length go to the short-block kernels
-constexpr int kSmallUnitVec = 4096;      // elements per CTA unit (L == 1, float4 path)
+constexpr int kSmallVecMaxL = 3;         // ... and up to this length, when aligned, straight through registers (small_kernel)
 constexpr int64_t kPieceMax = 32768;     // elements per partial sum, two-pass path
 constexpr int64_t kMaxPiecesPerBlock = 16384;
 constexpr int64_t kWideBlockPieces = 256;   // blocks with at least this many partial sums are finalized by a whole CTA
@@ -143,8 +143,8 @@ __device__ __forceinline__ double warp_sum(double x) {
 }
 
 // ---------------------------------------------------------------------------
-// Short blocks (L <= 64): float32 scalars throughout.  L == 1 with everything
-// 16-byte aligned runs here, one thread per four blocks (this is AdamW); every
+// Short blocks (L <= 64): float32 scalars throughout.  L == 1 (this is AdamW), 2 and 3
+// with everything 16-byte aligned run here, straight from registers; every
 // other case runs on the tile kernel (kernels_tile.cuh).
 // ---------------------------------------------------------------------------
 struct SmallScalars {
@@ -164,45 +164,107 @@ __device__ __forceinline__ float small_block_step(float mean_sq, float v_old, co
     return __fdiv_rn(s.lr_over_bc1, denom);
 }
 
-// L == 1, everything 16-byte aligned: four blocks per thread per round.
-template <int GD>
+// Blocks of one, two or three elements, everything 16-byte aligned: a thread takes
+// E = lcm(L, 4) consecutive elements per round (E / 4 16-byte accesses to each of g, m, p
+// and E / L whole blocks with their v), so nothing passes through shared memory and no
+// lane idles.  L == 1 is AdamW.
+template <int L> struct SmallVec {
+    static constexpr int E = L == 3 ? 12 : 4;                     // elements per thread per round
+    static constexpr int NB = E / L;                              // blocks per thread per round
+    static constexpr int kRounds = L == 3 ? 1 : 4;                // rounds per CTA unit
+    static constexpr int kUnit = kThreads * E * kRounds;          // elements per CTA unit
+};
+
+// Statistic of one block of L gradients (already scaled): mean of g*g, or an ablation variant.
+template <int L>
+__device__ __forceinline__ float small_block_statistic(const float *g, int statistic) {
+    if (L == 1) return g[0] * g[0];                               // every statistic of a one-element block
+    if (statistic == 0 || statistic == 3) {
+        float sum = g[0] * g[0];
+#pragma unroll
+        for (int k = 1; k < L; ++k) sum = fmaf(g[k], g[k], sum);
+        return statistic == 0 ? __fdiv_rn(sum, static_cast<float>(L)) : sum;
+    }
+    double acc = stat_identity(statistic);
+#pragma unroll
+    for (int k = 0; k < L; ++k) acc = stat_combine(acc, stat_term(g[k], statistic), statistic);
+    return static_cast<float>(stat_finish(acc, static_cast<double>(L), statistic));
+}
+
+template <int GD, int L>
 __device__ __forceinline__ void small_body(const DevTensor &t, int64_t local, float *__restrict__ v,
                                            const SmallScalars &sc) {
+    typedef SmallVec<L> V;
     const float lr_wd = t.wd ? sc.lr_wd : 0.f;
     const float gscale = effective_gscale(sc.gscale, sc.gscale_dev);
     float *vt = v + t.v_offset;
-    const int64_t base = local * kSmallUnitVec;
+    const int64_t base = local * V::kUnit;
 #pragma unroll
-    for (int r = 0; r < kSmallUnitVec / (kThreads * 4); ++r) {
-        const int64_t i = base + (static_cast<int64_t>(r) * kThreads + threadIdx.x) * 4;
+    for (int r = 0; r < V::kRounds; ++r) {
+        const int64_t i = base + (static_cast<int64_t>(r) * kThreads + threadIdx.x) * V::E;
         if (i >= t.numel) break;
-        const float4 g = load_g4<GD>(t.g, i, gscale);
-        float4 m = *reinterpret_cast<const float4 *>(t.m + i);
-        float4 p = *reinterpret_cast<const float4 *>(t.p + i);
-        float4 vv = *reinterpret_cast<const float4 *>(vt + i);
-        // (every statistic of a one-element block is g*g itself)
-        float st;
-        st = small_block_step(g.x * g.x, vv.x, sc, &vv.x); update_one(g.x, m.x, p.x, sc.beta1, sc.omb1, lr_wd, st);
-        st = small_block_step(g.y * g.y, vv.y, sc, &vv.y); update_one(g.y, m.y, p.y, sc.beta1, sc.omb1, lr_wd, st);
-        st = small_block_step(g.z * g.z, vv.z, sc, &vv.z); update_one(g.z, m.z, p.z, sc.beta1, sc.omb1, lr_wd, st);
-        st = small_block_step(g.w * g.w, vv.w, sc, &vv.w); update_one(g.w, m.w, p.w, sc.beta1, sc.omb1, lr_wd, st);
-        *reinterpret_cast<float4 *>(t.m + i) = m;
-        *reinterpret_cast<float4 *>(t.p + i) = p;
-        *reinterpret_cast<float4 *>(vt + i) = vv;
-        if (t.p_bf16) store_bf16x4(t.p_bf16 + i, p);
+        float g[V::E], m[V::E], p[V::E], vv[V::NB];
+#pragma unroll
+        for (int q = 0; q < V::E / 4; ++q) {
+            const float4 g4 = load_g4<GD>(t.g, i + 4 * q, gscale);
+            const float4 m4 = *reinterpret_cast<const float4 *>(t.m + i + 4 * q);
+            const float4 p4 = *reinterpret_cast<const float4 *>(t.p + i + 4 * q);
+            g[4 * q] = g4.x; g[4 * q + 1] = g4.y; g[4 * q + 2] = g4.z; g[4 * q + 3] = g4.w;
+            m[4 * q] = m4.x; m[4 * q + 1] = m4.y; m[4 * q + 2] = m4.z; m[4 * q + 3] = m4.w;
+            p[4 * q] = p4.x; p[4 * q + 1] = p4.y; p[4 * q + 2] = p4.z; p[4 * q + 3] = p4.w;
+        }
+        const int64_t b0 = i / L;                                 // exact: i is a multiple of E
+        if (V::NB == 4) {
+            const float4 v4 = *reinterpret_cast<const float4 *>(vt + b0);
+            vv[0] = v4.x; vv[1] = v4.y; vv[2] = v4.z; vv[3] = v4.w;
+        } else {
+            const float2 v2 = *reinterpret_cast<const float2 *>(vt + b0);
+            vv[0] = v2.x; vv[1] = v2.y;
+        }
+#pragma unroll
+        for (int b = 0; b < V::NB; ++b) {
+            const float st = small_block_step(small_block_statistic<L>(g + b * L, sc.statistic), vv[b], sc, &vv[b]);
+#pragma unroll
+            for (int k = 0; k < L; ++k) update_one(g[b * L + k], m[b * L + k], p[b * L + k], sc.beta1, sc.omb1, lr_wd, st);
+        }
+#pragma unroll
+        for (int q = 0; q < V::E / 4; ++q) {
+            const float4 m4 = make_float4(m[4 * q], m[4 * q + 1], m[4 * q + 2], m[4 * q + 3]);
+            const float4 p4 = make_float4(p[4 * q], p[4 * q + 1], p[4 * q + 2], p[4 * q + 3]);
+            *reinterpret_cast<float4 *>(t.m + i + 4 * q) = m4;
+            *reinterpret_cast<float4 *>(t.p + i + 4 * q) = p4;
+            if (t.p_bf16) store_bf16x4(t.p_bf16 + i + 4 * q, p4);
+        }
+        if (V::NB == 4) *reinterpret_cast<float4 *>(vt + b0) = make_float4(vv[0], vv[1], vv[2], vv[3]);
+        else *reinterpret_cast<float2 *>(vt + b0) = make_float2(vv[0], vv[1]);
     }
 }
 
-__global__ void __launch_bounds__(kThreads)
+// Whether a tensor of blocks of L elements can take small_kernel: every access above is aligned.
+__host__ __device__ inline bool small_vec_ok(int64_t L, int64_t numel, int64_t v_offset) {
+    if (L == 1) return numel % 4 == 0 && v_offset % 4 == 0;
+    if (L == 2) return numel % 4 == 0 && v_offset % 2 == 0;
+    if (L == 3) return numel % 12 == 0 && v_offset % 4 == 0;
+    return false;
+}
+__host__ __device__ inline int64_t small_vec_unit(int64_t L) {
+    return L == 3 ? SmallVec<3>::kUnit : SmallVec<1>::kUnit;
+}
+
+// One launch per block length present (the units of the segments of one length are
+// consecutive, starting at first_unit), so that the AdamW case keeps the registers it needs
+// and no more.
+template <int L>
+__global__ void __launch_bounds__(kThreads, L == 3 ? 3 : 4)
 small_kernel(const DevTensor *__restrict__ tensors, const Seg *__restrict__ segs, int n_segs,
-             float *__restrict__ v, SmallScalars sc) {
+             float *__restrict__ v, SmallScalars sc, int64_t first_unit) {
     if (step_skipped(sc.skip_flag)) return;
-    const int64_t unit = blockIdx.x;
+    const int64_t unit = first_unit + blockIdx.x;
     const Seg seg = segs[find_seg(segs, n_segs, unit)];
     const DevTensor &t = tensors[seg.tensor];
     const int64_t local = unit - seg.unit_begin;
-    if (t.gdtype == AM_BF16) small_body<AM_BF16>(t, local, v, sc);
-    else small_body<AM_F32>(t, local, v, sc);
+    if (t.gdtype == AM_BF16) small_body<AM_BF16, L>(t, local, v, sc);
+    else small_body<AM_F32, L>(t, local, v, sc);
 }
 
 // ---------------------------------------------------------------------------

@@ -111,6 +111,14 @@ struct StreamParams {
     int32_t pad;
 };
 
+// Long blocks whose starts are off the 16-byte grid: a stage carries the aligned middle of its
+// chunk; the up to seven elements before the first stage's chunk and after the last one's do
+// not pass through shared memory, the consumers fetch them from global memory.
+struct EdgeMeta {
+    const void *g;          // global address of the stage's first gradient
+    int32_t head, tail;     // elements before / after the stage's chunk that belong to the block (0..7)
+};
+
 struct Control {            // first kCtrlBytes of dynamic shared memory
     unsigned long long full[kMaxStages];     // producer -> consumers: the stage's copies have landed
     unsigned long long empty[kMaxStages];    // consumers -> producer: every consumer warp is done with the stage
@@ -124,6 +132,7 @@ struct Control {            // first kCtrlBytes of dynamic shared memory
     unsigned long long ibar[kItemSlots];     // cluster launches: "the next block index has arrived"
     long long next_item[kItemSlots];
     StageMeta meta[kMaxStages];
+    EdgeMeta edge[kMaxStages];               // launches of unaligned long blocks only
 };
 static_assert(sizeof(Control) <= kCtrlBytes, "control block fits its reservation");
 
@@ -395,12 +404,14 @@ __device__ __forceinline__ bool group_reduce(Control *ctl, GroupSync &gs, int *e
 // Template parameters keep the code of one launch small (the consumer loop is
 // sensitive to instruction-cache misses): GDM says which gradient dtypes the
 // launch's tensors have, COPY whether any tensor wants a bf16 copy, ST the block
-// statistic (StatOp; ST_SUM is Algorithm 1's mean).
+// statistic (StatOp; ST_SUM is Algorithm 1's mean), EDGES that the launch's blocks are
+// long ones that start off the 16-byte grid (see EdgeMeta).
 enum GradMode : int { GDM_F32 = 0, GDM_BF16 = 1, GDM_MIXED = 2 };
 
-template <bool CLUSTER, int GDM, bool COPY, int ST>
+template <bool CLUSTER, int GDM, bool COPY, int ST, bool EDGES>
 __global__ void __launch_bounds__(32 + kMaxConsumerWarps * 32, 1)
 stream_kernel(const __grid_constant__ StreamParams P) {
+    static_assert(!(EDGES && CLUSTER), "unaligned long blocks are handled by single CTAs");
     typedef typename StatAcc<ST>::T Acc;
     extern __shared__ __align__(128) unsigned char smem[];
     if (step_skipped(P.sc.skip_flag)) return;      // uniform over the grid: nobody reaches a barrier
@@ -577,11 +588,26 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                         begin = q * crank / csize * 16;
                         slice = (crank + 1 == csize ? t.L : q * (crank + 1) / csize * 16) - begin;
                     }
+                    int head = 0, tail = 0;
+                    if (EDGES) {
+                        // the aligned middle travels through the stages: 8 elements are 16 bytes of
+                        // bf16 gradients and 32 bytes of float32
+                        head = static_cast<int>((8 - ((local * t.L) & 7)) & 7);
+                        begin = head;
+                        slice = (t.L - head) & ~int64_t(7);
+                        tail = static_cast<int>(t.L - head - slice);
+                    }
                     const int64_t e0 = local * t.L + begin;
                     const int sum_cap = P.stage_bytes / gsz;
                     for (int64_t off = 0; off < slice && ok; off += sum_cap) {
                         const int c = static_cast<int>(slice - off < sum_cap ? slice - off : sum_cap);
                         if (!(ok = acquire())) break;
+                        if (EDGES) {
+                            EdgeMeta &em = ctl->edge[stage];
+                            em.g = gbase + (e0 + off) * gsz;
+                            em.head = off == 0 ? head : 0;
+                            em.tail = off + c == slice ? tail : 0;
+                        }
                         StageMeta &mt = ctl->meta[stage];
                         mt.m = nullptr; mt.p = nullptr; mt.v = P.v + t.v_offset + local; mt.pb = nullptr; mt.group = item_group;
                         mt.inv_L = inv_L;
@@ -601,6 +627,12 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                     for (int64_t off = 0; off < slice && ok; off += kStageElems) {
                         const int c = static_cast<int>(slice - off < kStageElems ? slice - off : kStageElems);
                         if (!(ok = acquire())) break;
+                        if (EDGES) {
+                            EdgeMeta &em = ctl->edge[stage];
+                            em.g = gbase + (e0 + off) * gsz;
+                            em.head = off == 0 ? head : 0;
+                            em.tail = off + c == slice ? tail : 0;
+                        }
                         StageMeta &mt = ctl->meta[stage];
                         mt.m = t.m + e0 + off; mt.p = t.p + e0 + off; mt.v = nullptr;
                         mt.pb = t.p_bf16 ? t.p_bf16 + e0 + off : nullptr; mt.group = item_group;
@@ -731,6 +763,18 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                 } else if (mt.kind == STAGE_SUM) {
                     if (bf16) sum_span<AM_BF16, ST>(gs, 0, mt.n, gtid, nthr, a0, a1, a2, a3);
                     else sum_span<AM_F32, ST>(gs, 0, mt.n, gtid, nthr, a0, a1, a2, a3);
+                    if (EDGES) {
+                        // the block's elements either side of the staged chunks, from global memory
+                        const EdgeMeta em = ctl->edge[stage];
+                        if (gtid < em.head) {
+                            const int64_t k = gtid - em.head;
+                            stat_acc_add<ST>(a0, bf16 ? load_g1<AM_BF16>(em.g, k, 1.f) : load_g1<AM_F32>(em.g, k, 1.f));
+                        }
+                        if (gtid >= 8 && gtid < 8 + em.tail) {
+                            const int64_t k = mt.n + (gtid - 8);
+                            stat_acc_add<ST>(a1, bf16 ? load_g1<AM_BF16>(em.g, k, 1.f) : load_g1<AM_F32>(em.g, k, 1.f));
+                        }
+                    }
                     if (!last_sum) {
                         __syncwarp();
                         if (lane == 0) mbar_arrive(&ctl->empty[stage]);
@@ -769,6 +813,19 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                 } else {   // STAGE_APPLY
                     if (bf16) apply_span<AM_BF16, COPY, CLUSTER>(gs, ms, ps, mt.m, mt.p, mt.pb, 0, mt.n, gtid, nthr, beta1, omb1, lr_wd, long_step);
                     else apply_span<AM_F32, COPY, CLUSTER>(gs, ms, ps, mt.m, mt.p, mt.pb, 0, mt.n, gtid, nthr, beta1, omb1, lr_wd, long_step);
+                    if (EDGES) {
+                        const EdgeMeta em = ctl->edge[stage];
+                        const bool is_head = gtid < em.head, is_tail = gtid >= 8 && gtid < 8 + em.tail;
+                        if (is_head || is_tail) {
+                            const int64_t k = is_head ? gtid - em.head : mt.n + (gtid - 8);
+                            const float g = bf16 ? load_g1<AM_BF16>(em.g, k, 1.f) : load_g1<AM_F32>(em.g, k, 1.f);
+                            float m = mt.m[k], p = mt.p[k];
+                            update_one(g, m, p, beta1, omb1, lr_wd, long_step);
+                            mt.m[k] = m;
+                            mt.p[k] = p;
+                            if (COPY && mt.pb) store_bf16(mt.pb + k, p);
+                        }
+                    }
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&ctl->empty[stage]);
                 }
@@ -797,21 +854,26 @@ struct StreamPlanInput {
     DeviceCaps caps;
     int ctas = 0, cluster_size = 0, threads = 0, groups = 0, chunk = 0, cluster_chunk = 0;
     struct Item { int tensor; am_table_row row; };
-    std::vector<Item> stream_tensors, cluster_tensors;
+    std::vector<Item> stream_tensors, cluster_tensors, edge_tensors;
 };
 
-// Which path a tensor with block length L (> 16) takes.
-inline int stream_classify(int64_t L, int32_t gdtype, bool cluster_ok) {
+// Which path a tensor with block length L (> 64) takes; *edges: its blocks start off the 16-byte
+// grid and run in the streaming kernel's launch for such blocks.
+inline int stream_classify(int64_t L, int32_t gdtype, bool cluster_ok, bool *edges) {
     const int64_t gsz = gdtype == AM_BF16 ? 2 : 4;
     const int64_t vec = 16 / gsz;                     // elements per 16 bytes of g
-    if (L % vec != 0) return PATH_TWOPASS;            // block starts would not be 16-byte aligned
+    *edges = false;
+    if (L % vec != 0) {                               // block starts are not 16-byte aligned
+        if (L > kStageElems && L * gsz <= kStreamMaxBlockBytes) { *edges = true; return PATH_STREAM; }
+        return PATH_TWOPASS;                          // (up to kStageElems elements the tile kernel takes them)
+    }
     if (L * gsz <= kStreamMaxBlockBytes) return PATH_STREAM;
     if (cluster_ok && L * gsz <= kClusterMaxBlockBytes && L % (kMaxCluster * vec) == 0) return PATH_CLUSTER;
     return PATH_TWOPASS;
 }
 
-inline void stream_add_tensor(StreamPlanInput &in, int index, const am_table_row &r, int path) {
-    (path == PATH_STREAM ? in.stream_tensors : in.cluster_tensors).push_back({index, r});
+inline void stream_add_tensor(StreamPlanInput &in, int index, const am_table_row &r, int path, bool edges) {
+    (path == PATH_CLUSTER ? in.cluster_tensors : edges ? in.edge_tensors : in.stream_tensors).push_back({index, r});
 }
 
 typedef void (*StreamKernelFn)(const StreamParams);
@@ -822,12 +884,12 @@ template <bool CLUSTER, int ST>
 inline StreamKernelFn stream_kernel_for(int gdm, bool copy) {
     if (ST != ST_SUM) copy = true;
     switch (gdm * 2 + (copy ? 1 : 0)) {
-    case 0: return stream_kernel<CLUSTER, GDM_F32, ST != ST_SUM, ST>;
-    case 1: return stream_kernel<CLUSTER, GDM_F32, true, ST>;
-    case 2: return stream_kernel<CLUSTER, GDM_BF16, ST != ST_SUM, ST>;
-    case 3: return stream_kernel<CLUSTER, GDM_BF16, true, ST>;
-    case 4: return stream_kernel<CLUSTER, GDM_MIXED, ST != ST_SUM, ST>;
-    default: return stream_kernel<CLUSTER, GDM_MIXED, true, ST>;
+    case 0: return stream_kernel<CLUSTER, GDM_F32, ST != ST_SUM, ST, false>;
+    case 1: return stream_kernel<CLUSTER, GDM_F32, true, ST, false>;
+    case 2: return stream_kernel<CLUSTER, GDM_BF16, ST != ST_SUM, ST, false>;
+    case 3: return stream_kernel<CLUSTER, GDM_BF16, true, ST, false>;
+    case 4: return stream_kernel<CLUSTER, GDM_MIXED, ST != ST_SUM, ST, false>;
+    default: return stream_kernel<CLUSTER, GDM_MIXED, true, ST, false>;
     }
 }
 template <bool CLUSTER>
@@ -842,12 +904,22 @@ inline StreamKernelFn stream_kernel_for(int gdm, bool copy, int st) {
 inline StreamKernelFn stream_kernel_for(bool cluster, int gdm, bool copy, int st) {
     return cluster ? stream_kernel_for<true>(gdm, copy, st) : stream_kernel_for<false>(gdm, copy, st);
 }
+// Unaligned long blocks: one instantiation per statistic, any gradient dtype, bf16 copies where asked for.
+inline StreamKernelFn stream_edge_kernel_for(int st) {
+    switch (st) {
+    case ST_MAX: return stream_kernel<false, GDM_MIXED, true, ST_MAX, true>;
+    case ST_MIN: return stream_kernel<false, GDM_MIXED, true, ST_MIN, true>;
+    case ST_SUM4: return stream_kernel<false, GDM_MIXED, true, ST_SUM4, true>;
+    default: return stream_kernel<false, GDM_MIXED, true, ST_SUM, true>;
+    }
+}
 
 struct StreamLaunch {
     std::vector<StreamSeg> segs;     // with sentinel
     std::vector<int64_t> bounds;
     int grid = 0, cluster = 1, n_stages = 0, stage_bytes = 0, g_region_bytes = 0, threads = 0, groups = 1, chunk = 0;
     int gdm = GDM_MIXED;
+    bool edges = false;              // the launch of unaligned long blocks
     unsigned long long *d_counter = nullptr;
     const StreamSeg *d_segs = nullptr;
     const int64_t *d_bounds = nullptr;
@@ -856,17 +928,17 @@ struct StreamLaunch {
 };
 
 struct StreamPlan {
-    StreamLaunch main, clus;
+    StreamLaunch main, clus, edge;
 
     size_t table_bytes() const {
-        return (main.segs.size() + clus.segs.size()) * sizeof(StreamSeg) + 256 +
-               (main.bounds.size() + clus.bounds.size()) * sizeof(int64_t) + 256 + 512;
+        return (main.segs.size() + clus.segs.size() + edge.segs.size()) * sizeof(StreamSeg) + 384 +
+               (main.bounds.size() + clus.bounds.size() + edge.bounds.size()) * sizeof(int64_t) + 384 + 768;
     }
-    int launches() const { return (main.active() ? 1 : 0) + (clus.active() ? 1 : 0); }
+    int launches() const { return (main.active() ? 1 : 0) + (clus.active() ? 1 : 0) + (edge.active() ? 1 : 0); }
 
     cudaError_t upload(char *base) {
         size_t off = 0;
-        for (StreamLaunch *L : {&main, &clus}) {
+        for (StreamLaunch *L : {&main, &clus, &edge}) {
             if (!L->active()) continue;
             cudaError_t e = cudaMemcpy(base + off, L->segs.data(), L->segs.size() * sizeof(StreamSeg), cudaMemcpyHostToDevice);
             if (e != cudaSuccess) return e;
@@ -915,7 +987,8 @@ struct StreamPlan {
             cfg.attrs = attr;
             cfg.numAttrs = 1;
         }
-        return cudaLaunchKernelEx(&cfg, stream_kernel_for(cluster, L.gdm, bf16_copies, stat_op_of(sc.statistic)), P);
+        const int st = stat_op_of(sc.statistic);
+        return cudaLaunchKernelEx(&cfg, L.edges ? stream_edge_kernel_for(st) : stream_kernel_for(cluster, L.gdm, bf16_copies, st), P);
     }
 
     cudaError_t launch_main(const DevTensor *tensors, float *v, const StepScalars &sc, int *error_word,
@@ -925,6 +998,10 @@ struct StreamPlan {
     cudaError_t launch_cluster(const DevTensor *tensors, float *v, const StepScalars &sc, int *error_word,
                                cudaStream_t stream) const {
         return clus.active() ? launch_one(clus, true, tensors, v, sc, error_word, stream) : cudaSuccess;
+    }
+    cudaError_t launch_edge(const DevTensor *tensors, float *v, const StepScalars &sc, int *error_word,
+                            cudaStream_t stream) const {
+        return edge.active() ? launch_one(edge, false, tensors, v, sc, error_word, stream) : cudaSuccess;
     }
 };
 
@@ -1037,7 +1114,7 @@ inline void stream_probe_clusters(DeviceCaps *caps, int block_threads) {
         cfg.attrs = attr;
         cfg.numAttrs = 1;
         int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, stream_kernel<true, GDM_MIXED, true, ST_SUM>, &cfg) == cudaSuccess && n > 0)
+        if (cudaOccupancyMaxActiveClusters(&n, stream_kernel<true, GDM_MIXED, true, ST_SUM, false>, &cfg) == cudaSuccess && n > 0)
             caps->resident[cs] = n;
         else
             (void)cudaGetLastError();
@@ -1090,19 +1167,22 @@ inline void stream_finish_plan(const StreamPlanInput &in, StreamPlan *plan) {
     int threads, groups;
     stream_consumer_shape(in.threads, in.groups, &threads, &groups);
     const int ctas = in.ctas > 0 ? in.ctas : in.caps.sm_count;
-    stream_build_launch(in.stream_tensors, false, ctas, in.caps.smem_optin, &plan->main);
-    plan->main.threads = threads;
-    plan->main.groups = groups;
-    plan->main.cluster = 1;
-    // work distribution: ranges of `chunk` items from a shared counter unless static ranges were asked for
-    if (in.chunk == kStaticRanges) plan->main.chunk = 0;
-    else if (in.chunk > 0) plan->main.chunk = in.chunk;
-    else {
-        // a workload of a couple of items per CTA gains nothing from the counter (and saves its memset)
-        const int64_t items = plan->main.bounds.empty() ? 0 : plan->main.bounds.back();     // in slots
-        plan->main.chunk = items <= 2 * static_cast<int64_t>(ctas)
-                               ? 0
-                               : static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(64, items / (int64_t(32) * std::max(ctas, 1)))));
+    for (StreamLaunch *L : {&plan->main, &plan->edge}) {
+        stream_build_launch(L == &plan->main ? in.stream_tensors : in.edge_tensors, false, ctas, in.caps.smem_optin, L);
+        L->edges = L == &plan->edge;
+        L->threads = threads;
+        L->groups = groups;
+        L->cluster = 1;
+        // work distribution: ranges of `chunk` items from a shared counter unless static ranges were asked for
+        if (in.chunk == kStaticRanges) L->chunk = 0;
+        else if (in.chunk > 0) L->chunk = in.chunk;
+        else {
+            // a workload of a couple of items per CTA gains nothing from the counter (and saves its memset)
+            const int64_t items = L->bounds.empty() ? 0 : L->bounds.back();     // in slots
+            L->chunk = items <= 2 * static_cast<int64_t>(ctas)
+                           ? 0
+                           : static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(64, items / (int64_t(32) * std::max(ctas, 1)))));
+        }
     }
     plan->clus = StreamLaunch();
     if (in.cluster_tensors.empty()) return;
@@ -1142,6 +1222,11 @@ inline cudaError_t stream_configure_kernels(size_t smem_optin) {
                                                                static_cast<int>(smem_optin));
                     if (e != cudaSuccess) return e;
                 }
+    for (int st = 0; st < 4; ++st) {
+        const cudaError_t e = cudaFuncSetAttribute(stream_edge_kernel_for(st), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                   static_cast<int>(smem_optin));
+        if (e != cudaSuccess) return e;
+    }
     return cudaSuccess;
 }
 

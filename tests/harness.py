@@ -166,7 +166,7 @@ class DeviceState:
 
 
 def mixed_workload():
-    """Every kernel family at once: tiny blocks, packed rows, long rows, a clustered head, a two-pass block."""
+    """Every kernel family at once: tiny blocks, packed rows, long rows (aligned and not), a clustered head, a two-pass block."""
     T = W.TensorSpec
     bf = dict(grad_dtype=W.BF16)
     tensors = [
@@ -177,6 +177,7 @@ def mixed_workload():
         T("head", 256, 4096, W.HEADS, n_heads=2, **bf),
         T("whole", 1, 3 << 20, W.WHOLE, **bf),
         T("odd", 5, 1001, W.ROWS, **bf),
+        T("longodd", 6, 10007, W.ROWS, **bf),
         T("f32rows", 64, 512, W.ROWS, grad_dtype=W.F32),
     ]
     return W.Workload("mixed", 61, tensors, W.GradRecipe(-4.0, -1.0), steps=3)

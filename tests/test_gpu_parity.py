@@ -670,6 +670,47 @@ def test_every_short_block_length(grad_dtype):
 
 
 @pytest.mark.parametrize("grad_dtype", [W.F32, W.BF16], ids=["f32", "bf16"])
+def test_blocks_of_two_and_three_elements(grad_dtype):
+    """Blocks of two and three elements whose tensors are 16-byte aligned throughout run
+    straight from registers (a thread takes 4 or 12 elements), several CTAs and a ragged
+    last one; the same lengths at offsets of v or element counts that break the alignment
+    stay on the tile kernel.  All against the oracle, also with an ablation statistic, a
+    gradient scale and a bf16 copy."""
+    gd = dict(grad_dtype=grad_dtype)
+    T = W.TensorSpec
+    tensors = [
+        T("a2", 2 * 4096 * 3 + 2 * 18, 2, W.ROWS, **gd),                 # L = 2: twelve full CTAs of 4096 elements and 72 elements
+        T("a3", 4 * 1024 * 2 + 4 * 7, 3, W.ROWS, apply_weight_decay=0, **gd),     # L = 3: eight full CTAs of 3072 elements and 84 elements
+        T("a1", 1, 4096 + 8, W.FIXED, fixed_block_len=1, **gd),
+        T("odd", 3, 5, W.ROWS, **gd),                                    # three blocks: what follows has an odd offset in v
+        T("b2", 1000, 2, W.ROWS, **gd),                                  # v offset odd: tile kernel
+        T("b3", 1001, 3, W.ROWS, **gd),                                  # 3003 elements: not a multiple of 12: tile kernel
+        T("c2", 1001, 2, W.ROWS, **gd),                                  # 2002 elements: not a multiple of 4: tile kernel
+    ]
+    w = W.Workload("tiny-blocks", 97 + grad_dtype, tensors, W.GradRecipe(-4.0, -1.0), steps=4)
+    opt = H.make_optimizer(w)
+    assert opt.query(B.Q_LAUNCHES_PER_STEP) == 4                         # lengths 1, 2, 3 from registers + one launch of tiles
+    assert opt.query(B.Q_ELEMENTS_SMALL) == w.numel
+    opt.close()
+    H.assert_parity(H.run_parity(w))
+    for statistic in (B.STAT_MAX, B.STAT_MIN, B.STAT_ONE_NORM, B.STAT_TWO_NORM):
+        H.assert_parity(H.run_parity(w, steps=2, statistic=statistic))
+    a, b = H.DeviceState(w, guarded=False), H.DeviceState(w, guarded=True)
+    copies = [H.Guarded(t.numel, torch.bfloat16, "cuda") for t in w.tensors]
+    oa, ob = H.make_optimizer(w), H.make_optimizer(w)
+    a.draw_grads(1)
+    for x, y in zip(a.g, b.g):
+        y.copy_(x * 0.5)
+    oa.step_ex(a.p, a.g, a.m, a.v, 1, grad_scale=0.5)
+    ob.step_ex(b.p, b.g, b.m, b.v, 1, params_bf16=[c.view for c in copies])
+    oa.sync_status(); ob.sync_status()
+    assert _same(a, b) and b.guards_intact()
+    for c, p in zip(copies, b.p):
+        assert torch.equal(c.view, p.to(torch.bfloat16)) and c.intact()
+    oa.close(); ob.close()
+
+
+@pytest.mark.parametrize("grad_dtype", [W.F32, W.BF16], ids=["f32", "bf16"])
 def test_unaligned_block_lengths_up_to_a_tile(grad_dtype):
     """Block lengths whose blocks start off the 16-byte grid, from just above the
     short-block limit to the tile size and one past it: several tiles each, so that
@@ -681,7 +722,10 @@ def test_unaligned_block_lengths_up_to_a_tile(grad_dtype):
     H.assert_parity(H.run_parity(w))
     H.assert_parity(H.run_parity(w, steps=2, statistic=B.STAT_MAX))
     opt = H.make_optimizer(w)
-    assert opt.query(B.Q_ELEMENTS_TWOPASS) == tensors[-1].numel          # only the 4097-element rows
+    assert opt.query(B.Q_ELEMENTS_TWOPASS) == 0
+    vec = 8 if grad_dtype == W.BF16 else 4                   # elements per 16 bytes of gradients
+    on_tiles = sum(t.numel for t in tensors if t.cols <= 4096 and t.cols % vec)
+    assert opt.query(B.Q_ELEMENTS_SMALL) == on_tiles and opt.query(B.Q_ELEMENTS_STREAM) == w.numel - on_tiles
     opt.close()
     a, b = H.DeviceState(w, guarded=False), H.DeviceState(w, guarded=True)
     copies = [H.Guarded(t.numel, torch.bfloat16, "cuda") for t in w.tensors]
@@ -693,6 +737,45 @@ def test_unaligned_block_lengths_up_to_a_tile(grad_dtype):
     ob.step_ex(b.p, b.g, b.m, b.v, 1, params_bf16=[c.view for c in copies], grad_scale=1.0)
     oa.sync_status(); ob.sync_status()
     assert _same(a, b) and b.guards_intact()
+    for c, p in zip(copies, b.p):
+        assert torch.equal(c.view, p.to(torch.bfloat16)) and c.intact()
+    oa.close(); ob.close()
+
+
+@pytest.mark.parametrize("grad_dtype", [W.F32, W.BF16], ids=["f32", "bf16"])
+def test_long_blocks_with_unaligned_starts_are_read_once(grad_dtype):
+    """Rows of more than 4096 elements whose byte length is not a multiple of 16 (so that
+    rows start at every offset within 32 bytes) stay on the single-read streaming kernel:
+    the aligned middle of every chunk is staged in shared memory, the up to seven elements
+    either side come from global memory.  Lengths around the stage sizes, a few rows each;
+    against the oracle, with guards, then with ablation statistics, a gradient scale and
+    bf16 copies.  Rows beyond 256 KB of gradients take the two-pass kernels as before."""
+    gsz = 2 if grad_dtype == W.BF16 else 4
+    lengths = [4097, 4099, 4101, 4103, 8191, 10007, 20481, 20489, 24577, 50257, 65543, 131063]
+    tensors = [W.TensorSpec(f"l{L}", 5 + i % 5, L, W.ROWS, grad_dtype=grad_dtype, apply_weight_decay=i % 2)
+               for i, L in enumerate(lengths)]
+    tensors.insert(3, W.TensorSpec("aligned", 7, 4104, W.ROWS, grad_dtype=grad_dtype))     # the ordinary launch beside it
+    w = W.Workload("long-unaligned", 99 + grad_dtype, tensors, W.GradRecipe(-4.0, -1.0), steps=3)
+    opt = H.make_optimizer(w)
+    beyond = sum(t.numel for t in tensors if t.cols * gsz > 256 * 1024)
+    assert opt.query(B.Q_ELEMENTS_TWOPASS) == beyond and opt.query(B.Q_ELEMENTS_STREAM) == w.numel - beyond
+    assert opt.query(B.Q_LAUNCHES_PER_STEP) == 2 + (3 if beyond else 0)
+    opt.close()
+    H.assert_parity(H.run_parity(w))
+    H.assert_parity(H.run_parity(w, steps=2, options={B.OPT_STREAM_CHUNK: 1, B.OPT_STREAM_THREADS: 128}))
+    for statistic in (B.STAT_MAX, B.STAT_TWO_NORM):
+        H.assert_parity(H.run_parity(w, steps=2, statistic=statistic))
+    a, b = H.DeviceState(w, guarded=False), H.DeviceState(w, guarded=True)
+    copies = [H.Guarded(t.numel, torch.bfloat16, "cuda") for t in w.tensors]
+    oa, ob = H.make_optimizer(w), H.make_optimizer(w, {B.OPT_STREAM_CTAS: 5, B.OPT_STREAM_GROUPS: 1})
+    for step in (1, 2):
+        a.draw_grads(step)
+        for x, y in zip(a.g, b.g):
+            y.copy_(x * 0.5)
+        oa.step_ex(a.p, a.g, a.m, a.v, step, grad_scale=0.5)
+        ob.step_ex(b.p, b.g, b.m, b.v, step, params_bf16=[c.view for c in copies])
+    oa.sync_status(); ob.sync_status()
+    assert _same(a, b) and b.guards_intact()                   # whatever the CTAs and groups, the same bits
     for c, p in zip(copies, b.p):
         assert torch.equal(c.view, p.to(torch.bfloat16)) and c.intact()
     oa.close(); ob.close()
