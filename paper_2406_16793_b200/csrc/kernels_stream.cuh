@@ -104,6 +104,7 @@ struct StreamParams {
     int32_t n_groups;
     int32_t chunk;              // > 0: items are handed out `chunk` at a time from *counter
     unsigned long long *counter;
+    unsigned long long *counter_next;   // the counter of this launch shape's NEXT launch: set to zero here (the two alternate)
     int64_t total_items;
     int64_t v_len;              // floats in v (staging never reads past it)
     unsigned long long wait_limit_ns;   // polling time after which a wait gives up
@@ -414,6 +415,9 @@ stream_kernel(const __grid_constant__ StreamParams P) {
     static_assert(!(EDGES && CLUSTER), "unaligned long blocks are handled by single CTAs");
     typedef typename StatAcc<ST>::T Acc;
     extern __shared__ __align__(128) unsigned char smem[];
+    // The work counter of the next launch of this shape starts at zero: the launch before this one
+    // used it and has ended (launches of one handle are ordered), so no separate clearing is enqueued.
+    if (blockIdx.x == 0 && threadIdx.x == 0 && P.counter_next) *P.counter_next = 0ull;
     if (step_skipped(P.sc.skip_flag)) return;      // uniform over the grid: nobody reaches a barrier
     Control *ctl = reinterpret_cast<Control *>(smem);
     unsigned char *stages = smem + kCtrlBytes;
@@ -920,7 +924,8 @@ struct StreamLaunch {
     int grid = 0, cluster = 1, n_stages = 0, stage_bytes = 0, g_region_bytes = 0, threads = 0, groups = 1, chunk = 0;
     int gdm = GDM_MIXED;
     bool edges = false;              // the launch of unaligned long blocks
-    unsigned long long *d_counter = nullptr;
+    unsigned long long *d_counter = nullptr;      // two counters, 64 bytes apart, used by alternate launches
+    mutable int counter_parity = 0;
     const StreamSeg *d_segs = nullptr;
     const int64_t *d_bounds = nullptr;
     bool active() const { return grid > 0; }
@@ -949,6 +954,9 @@ struct StreamPlan {
             L->d_bounds = reinterpret_cast<const int64_t *>(base + off);
             off += (L->bounds.size() * sizeof(int64_t) + 127) / 128 * 128;
             L->d_counter = reinterpret_cast<unsigned long long *>(base + off);
+            L->counter_parity = 0;
+            e = cudaMemset(base + off, 0, 128);
+            if (e != cudaSuccess) return e;
             off += 128;
         }
         return cudaSuccess;
@@ -968,11 +976,10 @@ struct StreamPlan {
         P.n_groups = L.groups;
         P.v_len = v_len;
         P.wait_limit_ns = wait_limit_ns; P.stall_after = stall_after; P.pad = 0;
-        P.chunk = L.chunk; P.counter = L.d_counter; P.total_items = L.bounds.empty() ? 0 : L.bounds.back();
-        if (P.chunk > 0) {
-            cudaError_t e = cudaMemsetAsync(L.d_counter, 0, sizeof(unsigned long long), stream);
-            if (e != cudaSuccess) return e;
-        }
+        P.chunk = L.chunk; P.total_items = L.bounds.empty() ? 0 : L.bounds.back();
+        P.counter = L.d_counter + 8 * L.counter_parity;
+        P.counter_next = L.d_counter + 8 * (L.counter_parity ^ 1);
+        L.counter_parity ^= 1;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(L.grid);
         cfg.blockDim = dim3(32 + L.threads * L.groups);

@@ -751,7 +751,7 @@ def test_long_blocks_with_unaligned_starts_are_read_once(grad_dtype):
     against the oracle, with guards, then with ablation statistics, a gradient scale and
     bf16 copies.  Rows beyond 256 KB of gradients take the two-pass kernels as before."""
     gsz = 2 if grad_dtype == W.BF16 else 4
-    lengths = [4097, 4099, 4101, 4103, 8191, 10007, 20481, 20489, 24577, 50257, 65543, 131063]
+    lengths = [4097, 4099, 4101, 4103, 8191, 8199, 8209, 10007, 20481, 20489, 24577, 50257, 65543, 131063]
     tensors = [W.TensorSpec(f"l{L}", 5 + i % 5, L, W.ROWS, grad_dtype=grad_dtype, apply_weight_decay=i % 2)
                for i, L in enumerate(lengths)]
     tensors.insert(3, W.TensorSpec("aligned", 7, 4104, W.ROWS, grad_dtype=grad_dtype))     # the ordinary launch beside it

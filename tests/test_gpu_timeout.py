@@ -26,7 +26,7 @@ def rows_workload():
     """Single-CTA streaming kernel: packed rows and long rows re-read from L2, aligned and
     not (the latter in a launch of their own)."""
     return W.Workload("stall-rows", 71, [T("rows", 600, 4096, W.ROWS, **BF), T("short", 3000, 768, W.ROWS, **BF),
-                                         T("long", 300, 11008, W.ROWS, **BF), T("longodd", 150, 10007, W.ROWS, **BF)], W.GradRecipe(-4.0, -1.0), steps=2)
+                                         T("long", 300, 11008, W.ROWS, **BF), T("longodd", 150, 10007, W.ROWS, **BF), T("held", 300, 4099, W.ROWS, **BF)], W.GradRecipe(-4.0, -1.0), steps=2)
 
 
 def heads_workload():
