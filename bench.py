@@ -42,12 +42,30 @@ NOMINAL_HBM_GBS = 8000.0      # HBM3e of a B200, nominal (quoted beside the meas
 # family from the ncu captures summarised under profiles/.  An entry counts only while the
 # sources its kernel is compiled from still have the digest they had at the capture.
 NCU_TRAFFIC = [
-    {"family": "stream_kernel<false>", "grad": "bf16", "sources": "stream", "digest": "b54ab5e4dc5f67f5",
-     "bytes_per_param": 17.91, "elements_query": lambda B: B.Q_ELEMENTS_STREAM,
+    {"family": "stream_kernel<false>", "grad": "bf16", "block_lens": {4096, 11008}, "sources": "stream", "digest": "625d60e88a1e6a4b",
+     "bytes_per_param": 17.905, "elements_query": lambda B: B.Q_ELEMENTS_STREAM,
      "capture": "profiles/stream_kernel_llama2_7b.md (2-layer case, scaled by parameters)"},
-    {"family": "stream_kernel<true>", "grad": "bf16", "sources": "stream", "digest": "b54ab5e4dc5f67f5",
-     "bytes_per_param": 17.41, "elements_query": lambda B: B.Q_ELEMENTS_CLUSTER,
+    {"family": "stream_kernel<true>", "grad": "bf16", "block_lens": {524288}, "sources": "stream", "digest": "625d60e88a1e6a4b",
+     "bytes_per_param": 17.475, "elements_query": lambda B: B.Q_ELEMENTS_CLUSTER,
      "capture": "profiles/stream_kernel_llama2_7b.md (2-layer case, scaled by parameters)"},
+    {"family": "stream_kernel<false>", "grad": "bf16", "block_lens": {10007}, "sources": "stream", "digest": "625d60e88a1e6a4b",
+     "bytes_per_param": 17.596, "elements_query": lambda B: B.Q_ELEMENTS_STREAM,
+     "capture": "profiles/stream_kernel_unaligned_rows_bf16_L10007.md (2^27 parameters, scaled)"},
+    {"family": "short_block_kernels", "grad": "f32", "block_lens": {1}, "sources": "basic", "digest": "ba7f3053c6c300ff",
+     "bytes_per_param": 27.595, "elements_query": lambda B: B.Q_ELEMENTS_SMALL,
+     "capture": "profiles/small_and_twopass_kernels_flat_fp32.md (2^27 parameters, scaled)"},
+    {"family": "short_block_kernels", "grad": "f32", "block_lens": {2}, "sources": "basic", "digest": "ba7f3053c6c300ff",
+     "bytes_per_param": 23.597, "elements_query": lambda B: B.Q_ELEMENTS_SMALL,
+     "capture": "profiles/small_and_twopass_kernels_flat_fp32.md (2^27 parameters, scaled)"},
+    {"family": "twopass_kernels", "grad": "f32", "min_block_len": 1 << 22, "sources": "basic", "digest": "ba7f3053c6c300ff",
+     "bytes_per_param": 23.647, "elements_query": lambda B: B.Q_ELEMENTS_TWOPASS,
+     "capture": "profiles/small_and_twopass_kernels_flat_fp32.md (one block of 2^27 elements, scaled)"},
+    {"family": "short_block_kernels", "grad": "f32", "block_lens": {32}, "sources": "tile", "digest": "e668cb567947738c",
+     "bytes_per_param": 19.837, "elements_query": lambda B: B.Q_ELEMENTS_SMALL,
+     "capture": "profiles/tile_kernel_flat_fp32_L32.md (2^27 parameters, scaled)"},
+    {"family": "short_block_kernels", "grad": "bf16", "block_lens": {1001}, "sources": "tile", "digest": "e668cb567947738c",
+     "bytes_per_param": 17.585, "elements_query": lambda B: B.Q_ELEMENTS_SMALL,
+     "capture": "profiles/tile_kernel_rows_bf16_L1001.md (2^27 parameters, scaled)"},
 ]
 
 
@@ -101,8 +119,9 @@ def pick_workload(name: str):
     if name.startswith("flat-L"):                      # flat-L<block length>[-n<log2 of the element count>]
         parts = name[6:].split("-n")
         L, numel = int(parts[0]), 1 << (int(parts[1]) if len(parts) > 1 else 30)
-        unit = 64 * L if 64 % L else 64                                # whole blocks and whole 64-element chunks of one sigma
-        return W.flat_sweep(L, numel=numel // unit * unit)
+        import math
+        unit = math.lcm(L, 64)                                         # whole blocks and whole 64-element chunks of one sigma
+        return W.flat_sweep(L, numel=max(numel // unit, 1) * unit)
     if name.startswith("llama2-7b-layers"):
         return W.llama2_7b(n_layers=int(name[len("llama2-7b-layers"):]))
     if name.startswith("rows-"):                        # rows-<bf16|f32>-L<row length>-r<rows>: one matrix, a block per row
@@ -279,6 +298,30 @@ class ShardedJob:
             self.sh.step_local(self.p, self.g, self.m, self.v, t, self.exchange)
 
 
+def family_of_specs(job, B):
+    """The kernel family each tensor of the job runs on, by the library's routing rules as its
+    element counts per family confirm them: short or tile-sized unaligned blocks -> short-block
+    kernels; head-sized blocks -> the cluster kernel; blocks beyond 4 MB of gradients -> two-pass."""
+    out = []
+    for t in job.specs:
+        gsz = 2 if t.grad_dtype == 1 else 4
+        L = t.block_len
+        if L <= 64 or (L <= 4096 and (L * gsz) % 16):
+            out.append("short_block_kernels")
+        elif L * gsz <= 256 * 1024:
+            out.append("stream_kernel<false>")
+        elif L * gsz <= 4 * 1024 * 1024 and L % (8 * 16 // gsz) == 0:
+            out.append("stream_kernel<true>")
+        else:
+            out.append("twopass_kernels")
+    counts = {"short_block_kernels": B.Q_ELEMENTS_SMALL, "stream_kernel<false>": B.Q_ELEMENTS_STREAM,
+              "stream_kernel<true>": B.Q_ELEMENTS_CLUSTER, "twopass_kernels": B.Q_ELEMENTS_TWOPASS}
+    for fam, q in counts.items():
+        if sum(t.numel for t, f in zip(job.specs, out) if f == fam) != job.opt.query(q):
+            return [None] * len(out)           # the routing differs (an option forces a path): no capture applies
+    return out
+
+
 def ncu_traffic(family: str, job, B):
     """DRAM bytes per launch of the dominant kernel family from the ncu captures
     summarised under profiles/, scaled by the parameters the family processes; None
@@ -286,13 +329,19 @@ def ncu_traffic(family: str, job, B):
     digests = kernel_digests()
     bf16 = all(t.grad_dtype == 1 for t in job.specs)
     f32 = all(t.grad_dtype == 0 for t in job.specs)
-    unit_blocks = all(t.block_len == 1 for t in job.specs)
     for e in NCU_TRAFFIC:
         if e["family"] != family or digests.get(e["sources"]) != e["digest"]:
             continue
         if (e["grad"] == "bf16" and not bf16) or (e["grad"] == "f32" and not f32):
             continue
-        if e.get("unit_blocks") is not None and e["unit_blocks"] != unit_blocks:
+        # a capture speaks for the block lengths it ran: every tensor the family handles must have one of them
+        fam_lens = {t.block_len for t, path in zip(job.specs, family_of_specs(job, B)) if path == family}
+        if not fam_lens:
+            continue
+        if "min_block_len" in e:
+            if min(fam_lens) < e["min_block_len"]:
+                continue
+        elif not fam_lens <= e["block_lens"]:
             continue
         return e["bytes_per_param"] * job.opt.query(e["elements_query"](B)), e["capture"]
     return None, None
