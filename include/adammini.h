@@ -286,10 +286,12 @@ typedef enum {
     AM_Q_TOTAL_ELEMENTS    = 3,
     AM_Q_ELEMENTS_SMALL    = 4, /* elements routed to the short-block kernels (block_len <= 64, and blocks of
                                    up to 4096 elements whose starts are not 16-byte aligned) */
-    AM_Q_ELEMENTS_STREAM   = 5, /* ... to the single-launch streaming kernel */
+    AM_Q_ELEMENTS_STREAM   = 5, /* ... to the streaming kernel (its launch for rows, and the one for blocks of more
+                                   than 4096 elements, up to 256 KB of gradients, whose starts are not 16-byte
+                                   aligned) */
     AM_Q_ELEMENTS_CLUSTER  = 6, /* ... to the cluster kernel (head-sized blocks) */
-    AM_Q_ELEMENTS_TWOPASS  = 7, /* ... to the two-pass path (blocks beyond on-chip/L2 reach, or longer than 4096
-                                   elements with unaligned starts) */
+    AM_Q_ELEMENTS_TWOPASS  = 7, /* ... to the two-pass path (blocks beyond on-chip/L2 reach: more than 4 MB of
+                                   gradients, or more than 256 KB with unaligned starts; parts of blocks) */
     AM_Q_ALGORITHMIC_BYTES = 8, /* bytes one step must move: per tensor g once (twice for blocks beyond
                                    on-chip/L2 reach), m and p read+written, v read+written */
     AM_Q_BYTES_SMALL       = 9, /* the same, split by the kernel family that handles the tensor */

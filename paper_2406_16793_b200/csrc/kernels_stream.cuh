@@ -765,20 +765,23 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&ctl->empty[stage]);
                 } else if (mt.kind == STAGE_SUM) {
-                    if (bf16) sum_span<AM_BF16, ST>(gs, 0, mt.n, gtid, nthr, a0, a1, a2, a3);
-                    else sum_span<AM_F32, ST>(gs, 0, mt.n, gtid, nthr, a0, a1, a2, a3);
+                    // (unaligned blocks: the block's elements either side of the staged chunks come from
+                    // global memory; their loads are issued first, so that the pass over the stage covers
+                    // their latency)
+                    bool edge_mine = false;
+                    float edge_g = 0.f;
                     if (EDGES) {
-                        // the block's elements either side of the staged chunks, from global memory
                         const EdgeMeta em = ctl->edge[stage];
-                        if (gtid < em.head) {
-                            const int64_t k = gtid - em.head;
-                            stat_acc_add<ST>(a0, bf16 ? load_g1<AM_BF16>(em.g, k, 1.f) : load_g1<AM_F32>(em.g, k, 1.f));
-                        }
-                        if (gtid >= 8 && gtid < 8 + em.tail) {
-                            const int64_t k = mt.n + (gtid - 8);
-                            stat_acc_add<ST>(a1, bf16 ? load_g1<AM_BF16>(em.g, k, 1.f) : load_g1<AM_F32>(em.g, k, 1.f));
+                        const bool is_head = gtid < em.head, is_tail = gtid >= 8 && gtid < 8 + em.tail;
+                        edge_mine = is_head || is_tail;
+                        if (edge_mine) {
+                            const int64_t k = is_head ? gtid - em.head : mt.n + (gtid - 8);
+                            edge_g = bf16 ? load_g1<AM_BF16>(em.g, k, 1.f) : load_g1<AM_F32>(em.g, k, 1.f);
                         }
                     }
+                    if (bf16) sum_span<AM_BF16, ST>(gs, 0, mt.n, gtid, nthr, a0, a1, a2, a3);
+                    else sum_span<AM_F32, ST>(gs, 0, mt.n, gtid, nthr, a0, a1, a2, a3);
+                    if (EDGES && edge_mine) stat_acc_add<ST>(a0, edge_g);
                     if (!last_sum) {
                         __syncwarp();
                         if (lane == 0) mbar_arrive(&ctl->empty[stage]);
@@ -815,20 +818,27 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                         if (gtid == 0 && (mt.flags & SF_WRITE_V)) *mt.v = vn;
                     }
                 } else {   // STAGE_APPLY
-                    if (bf16) apply_span<AM_BF16, COPY, CLUSTER>(gs, ms, ps, mt.m, mt.p, mt.pb, 0, mt.n, gtid, nthr, beta1, omb1, lr_wd, long_step);
-                    else apply_span<AM_F32, COPY, CLUSTER>(gs, ms, ps, mt.m, mt.p, mt.pb, 0, mt.n, gtid, nthr, beta1, omb1, lr_wd, long_step);
-                    if (EDGES) {
+                    bool edge_mine = false;
+                    int64_t edge_k = 0;
+                    float edge_g = 0.f, edge_m = 0.f, edge_p = 0.f;
+                    if (EDGES) {        // edge elements: loads first, update and stores after the pass over the stage
                         const EdgeMeta em = ctl->edge[stage];
                         const bool is_head = gtid < em.head, is_tail = gtid >= 8 && gtid < 8 + em.tail;
-                        if (is_head || is_tail) {
-                            const int64_t k = is_head ? gtid - em.head : mt.n + (gtid - 8);
-                            const float g = bf16 ? load_g1<AM_BF16>(em.g, k, 1.f) : load_g1<AM_F32>(em.g, k, 1.f);
-                            float m = mt.m[k], p = mt.p[k];
-                            update_one(g, m, p, beta1, omb1, lr_wd, long_step);
-                            mt.m[k] = m;
-                            mt.p[k] = p;
-                            if (COPY && mt.pb) store_bf16(mt.pb + k, p);
+                        edge_mine = is_head || is_tail;
+                        if (edge_mine) {
+                            edge_k = is_head ? gtid - em.head : mt.n + (gtid - 8);
+                            edge_g = bf16 ? load_g1<AM_BF16>(em.g, edge_k, 1.f) : load_g1<AM_F32>(em.g, edge_k, 1.f);
+                            edge_m = mt.m[edge_k];
+                            edge_p = mt.p[edge_k];
                         }
+                    }
+                    if (bf16) apply_span<AM_BF16, COPY, CLUSTER>(gs, ms, ps, mt.m, mt.p, mt.pb, 0, mt.n, gtid, nthr, beta1, omb1, lr_wd, long_step);
+                    else apply_span<AM_F32, COPY, CLUSTER>(gs, ms, ps, mt.m, mt.p, mt.pb, 0, mt.n, gtid, nthr, beta1, omb1, lr_wd, long_step);
+                    if (EDGES && edge_mine) {
+                        update_one(edge_g, edge_m, edge_p, beta1, omb1, lr_wd, long_step);
+                        mt.m[edge_k] = edge_m;
+                        mt.p[edge_k] = edge_p;
+                        if (COPY && mt.pb) store_bf16(mt.pb + edge_k, edge_p);
                     }
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&ctl->empty[stage]);

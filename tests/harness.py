@@ -82,8 +82,8 @@ class ShortBlockScale:
     with operands of opposite sign.  float32 then carries an absolute error of the
     order of an ulp of the OPERANDS, so the ratio to |m_t| says nothing about the
     arithmetic; in a block of one, two or three elements all of them can do so at
-    once (seen in the seeded tests: see the design notes), and the block's RMS is
-    then no better a scale.  The scale kept here is the magnitude of those operands,
+    once (the seeded tests hold two-element blocks whose two entries of m are both below
+    1e-2 of their operands), and the block's RMS is then no better a scale.  The scale kept here is the magnitude of those operands,
     followed along the oracle's own trajectory of that element:
         S_m(t) = max(|m_t|, (1-beta1)|g_t| + beta1 S_m(t-1)),  S_m(0) = 0
         S_p(t) = max(|p_t|, S_p(t-1)),                         S_p(0) = |p_0|
