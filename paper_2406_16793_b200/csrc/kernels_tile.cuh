@@ -347,7 +347,7 @@ tile_kernel(const DevTensor *__restrict__ tensors, const Seg *__restrict__ segs,
     float *sg = reinterpret_cast<float *>(bar + 2);
     if (step_skipped(sc.skip_flag)) return;
     const int64_t unit = first_unit + blockIdx.x;
-    const Seg seg = segs[find_seg(segs, n_segs, unit)];
+    const Seg seg = segs[find_seg_warp(segs, n_segs, unit)];
     const DevTensor &t = tensors[seg.tensor];
     const int64_t tile = unit - seg.unit_begin;
     if (t.L > kSmallMaxL) {
