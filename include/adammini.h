@@ -251,11 +251,13 @@ typedef enum {
     AM_OPT_PROFILE        = 4, /* n > 0: record CUDA events around each kernel family of every step, keeping
                                   the latest n steps (n <= 4096); read them with adammini_get_profile.
                                   Setting the option again restarts the record */
-    AM_OPT_STREAM_CHUNK   = 5, /* how the streaming kernel's CTAs share the work: 0 = automatic (CTAs take
-                                  up to 64 work items at a time from a shared counter, which evens out
-                                  bandwidth differences between SMs; fixed ranges for tiny workloads);
-                                  1..4096 = that many items at a time; 1000000 = every CTA walks its own
-                                  fixed, cost-balanced range.  Results are bit-identical in every mode */
+    AM_OPT_STREAM_CHUNK   = 5, /* how the streaming kernel's CTAs share the work: 0 = automatic (CTAs take one
+                                  work item at a time -- a stage of packed blocks, or one long block -- from
+                                  a shared counter: this evens out bandwidth differences between SMs and
+                                  keeps all CTAs on one neighbourhood of memory; fixed ranges for tiny
+                                  workloads); 1..4096 = that many items at a time; 1000000 = every CTA
+                                  walks its own fixed, cost-balanced range.  Results are bit-identical in
+                                  every mode */
     AM_OPT_CLUSTER_CHUNK  = 6, /* the same for the cluster kernel, in blocks handed to a cluster at a time */
     AM_OPT_STATISTIC      = 7, /* block statistic that feeds v: 0 = mean(g*g), Algorithm 1.  The ablation
                                   of the paper's appendix ("Ablation Studies on the Design of Adam-mini"),
