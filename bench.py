@@ -42,29 +42,29 @@ NOMINAL_HBM_GBS = 8000.0      # HBM3e of a B200, nominal (quoted beside the meas
 # family from the ncu captures summarised under profiles/.  An entry counts only while the
 # sources its kernel is compiled from still have the digest they had at the capture.
 NCU_TRAFFIC = [
-    {"family": "stream_kernel<false>", "grad": "bf16", "block_lens": {4096, 11008}, "sources": "stream", "digest": "e474a406306c3448",
-     "bytes_per_param": 17.909, "elements_query": lambda B: B.Q_ELEMENTS_STREAM,
+    {"family": "stream_kernel<false>", "grad": "bf16", "block_lens": {4096, 11008}, "sources": "stream", "digest": "02a849eb5e16e77e",
+     "bytes_per_param": 17.905, "elements_query": lambda B: B.Q_ELEMENTS_STREAM,
      "capture": "profiles/stream_kernel_llama2_7b.md (2-layer case, scaled by parameters)"},
-    {"family": "stream_kernel<true>", "grad": "bf16", "block_lens": {524288}, "sources": "stream", "digest": "e474a406306c3448",
-     "bytes_per_param": 17.440, "elements_query": lambda B: B.Q_ELEMENTS_CLUSTER,
+    {"family": "stream_kernel<true>", "grad": "bf16", "block_lens": {524288}, "sources": "stream", "digest": "02a849eb5e16e77e",
+     "bytes_per_param": 17.434, "elements_query": lambda B: B.Q_ELEMENTS_CLUSTER,
      "capture": "profiles/stream_kernel_llama2_7b.md (2-layer case, scaled by parameters)"},
-    {"family": "stream_kernel<false>", "grad": "bf16", "block_lens": {10007}, "sources": "stream", "digest": "e474a406306c3448",
-     "bytes_per_param": 17.590, "elements_query": lambda B: B.Q_ELEMENTS_STREAM,
+    {"family": "stream_kernel<false>", "grad": "bf16", "block_lens": {10007}, "sources": "stream", "digest": "02a849eb5e16e77e",
+     "bytes_per_param": 17.592, "elements_query": lambda B: B.Q_ELEMENTS_STREAM,
      "capture": "profiles/stream_kernel_unaligned_rows_bf16_L10007.md (2^27 parameters, scaled)"},
-    {"family": "short_block_kernels", "grad": "f32", "block_lens": {1}, "sources": "basic", "digest": "b2d1acce62e6fc5f",
-     "bytes_per_param": 27.594, "elements_query": lambda B: B.Q_ELEMENTS_SMALL,
+    {"family": "short_block_kernels", "grad": "f32", "block_lens": {1}, "sources": "basic", "digest": "85b9245f3da5fdb0",
+     "bytes_per_param": 27.587, "elements_query": lambda B: B.Q_ELEMENTS_SMALL,
      "capture": "profiles/small_and_twopass_kernels_flat_fp32.md (2^27 parameters, scaled)"},
-    {"family": "short_block_kernels", "grad": "f32", "block_lens": {2}, "sources": "basic", "digest": "b2d1acce62e6fc5f",
-     "bytes_per_param": 23.599, "elements_query": lambda B: B.Q_ELEMENTS_SMALL,
+    {"family": "short_block_kernels", "grad": "f32", "block_lens": {2}, "sources": "basic", "digest": "85b9245f3da5fdb0",
+     "bytes_per_param": 23.597, "elements_query": lambda B: B.Q_ELEMENTS_SMALL,
      "capture": "profiles/small_and_twopass_kernels_flat_fp32.md (2^27 parameters, scaled)"},
-    {"family": "twopass_kernels", "grad": "f32", "min_block_len": 1 << 22, "sources": "basic", "digest": "b2d1acce62e6fc5f",
-     "bytes_per_param": 23.654, "elements_query": lambda B: B.Q_ELEMENTS_TWOPASS,
+    {"family": "twopass_kernels", "grad": "f32", "min_block_len": 1 << 22, "sources": "basic", "digest": "85b9245f3da5fdb0",
+     "bytes_per_param": 23.650, "elements_query": lambda B: B.Q_ELEMENTS_TWOPASS,
      "capture": "profiles/small_and_twopass_kernels_flat_fp32.md (one block of 2^27 elements, scaled)"},
-    {"family": "short_block_kernels", "grad": "f32", "block_lens": {32}, "sources": "tile", "digest": "ce631954a4b99910",
-     "bytes_per_param": 19.833, "elements_query": lambda B: B.Q_ELEMENTS_SMALL,
+    {"family": "short_block_kernels", "grad": "f32", "block_lens": {32}, "sources": "tile", "digest": "d087d6ca571e955b",
+     "bytes_per_param": 19.841, "elements_query": lambda B: B.Q_ELEMENTS_SMALL,
      "capture": "profiles/tile_kernel_flat_fp32_L32.md (2^27 parameters, scaled)"},
-    {"family": "short_block_kernels", "grad": "bf16", "block_lens": {1001}, "sources": "tile", "digest": "ce631954a4b99910",
-     "bytes_per_param": 17.582, "elements_query": lambda B: B.Q_ELEMENTS_SMALL,
+    {"family": "short_block_kernels", "grad": "bf16", "block_lens": {1001}, "sources": "tile", "digest": "d087d6ca571e955b",
+     "bytes_per_param": 17.591, "elements_query": lambda B: B.Q_ELEMENTS_SMALL,
      "capture": "profiles/tile_kernel_rows_bf16_L1001.md (2^27 parameters, scaled)"},
 ]
 

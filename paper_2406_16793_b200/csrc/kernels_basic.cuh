@@ -126,20 +126,11 @@ __device__ __forceinline__ double warp_stat(double x, int statistic) {
     return x;
 }
 
-// Segment lookup: the last segment whose unit_begin is <= unit.
-__device__ __forceinline__ int find_seg(const Seg *segs, int n_segs, int64_t unit) {
-    int lo = 0, hi = n_segs - 1;
-    while (lo < hi) {
-        const int mid = (lo + hi + 1) >> 1;
-        if (segs[mid].unit_begin <= unit) lo = mid; else hi = mid - 1;
-    }
-    return lo;
-}
-
-// The same lookup by a whole (converged) warp: 32 probes per round, so a table of up to 1024
-// segments takes two dependent loads instead of ten.  Every lane returns the result.  A CTA of
-// these kernels lives for a few microseconds, and nothing can be requested from memory before
-// its segment is known: on a table of 94 matrices the tile kernel went from 0.96 to 1.00 of the
+// Segment lookup: the last segment whose unit_begin is <= unit, by a whole (converged) warp:
+// 32 probes per round, so a table of up to 1024 segments takes two dependent loads where a
+// binary search by one thread takes ten.  Every lane returns the result.  A CTA of these
+// kernels lives for a few microseconds, and nothing can be requested from memory before its
+// segment is known: on a table of 94 matrices the tile kernel went from 0.96 to 1.00 of the
 // measured copy bandwidth with this.
 __device__ __forceinline__ int find_seg_warp(const Seg *segs, int n_segs, int64_t unit) {
     const int lane = threadIdx.x & 31;

@@ -1,7 +1,8 @@
 // The single-read streaming kernels.
 //
-// One persistent CTA per SM.  A producer thread takes work items (from a
-// global counter, a range at a time, or from a fixed range of its own) and
+// One persistent CTA per SM.  A producer thread takes work items (one at a
+// time from a global counter, so that all CTAs stay on one neighbourhood of
+// memory and share open DRAM pages; or from a fixed range of its own) and
 // moves gradients, first moments, parameters and the blocks' old v from HBM
 // into a ring of shared-memory stages with bulk asynchronous copies
 // (cp.async.bulk, completion counted on an mbarrier).  The consumer warps,
@@ -25,6 +26,10 @@
 // depend on the number of CTAs or groups or on how the work was handed out; the
 // threads per group and the cluster size fix that order and so can change the
 // last bit of a sum.
+//
+// Blocks longer than a stage whose starts are off the 16-byte grid run in a
+// launch of their own (template argument EDGES): the aligned middle of every
+// chunk is staged, the few elements either side come from global memory.
 //
 // Every wait is bounded: a wait that gives up sets the abort flag and the
 // handle's error word, and all roles leave through the common exit.
