@@ -139,7 +139,11 @@ int adammini_set_hparams(am_handle *h, const am_hparams *hp);
  * Asynchronous: work is enqueued on the stream and the call returns without
  * synchronising.  params, m and v are updated in place.  Calls on one handle
  * must be issued from one thread at a time and ordered on one stream (or
- * otherwise serialised), because they share the handle's scratch. */
+ * otherwise serialised), because they share the handle's scratch.
+ * A step cannot be recorded into a CUDA graph (t and the hyper-parameters are
+ * kernel arguments, and successive launches take turns on two work counters,
+ * so a replay would repeat a stale step): a stream that is capturing is refused
+ * with AM_ERR_INVALID_ARGUMENT and nothing is enqueued. */
 int adammini_step(am_handle *h, void *const *params, const void *const *grads, void *const *m,
                   float *v, int64_t step, void *cuda_stream);
 

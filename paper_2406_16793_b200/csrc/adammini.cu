@@ -517,6 +517,12 @@ int adammini_step_ex(am_handle *h, void *const *params, const void *const *grads
     int dev = -1;
     AM_CUDA(h, cudaGetDevice(&dev));
     if (dev != h->device) return AM_ERR_INVALID_ARGUMENT;
+    // A step is not a replayable graph node: t and the hyper-parameters are kernel arguments, the
+    // tensor table is re-uploaded when a pointer changes, and consecutive launches of a shape take
+    // turns on two work counters.  A capturing stream is refused before anything is enqueued.
+    cudaStreamCaptureStatus capture = cudaStreamCaptureStatusNone;
+    AM_CUDA(h, cudaStreamIsCapturing(stream, &capture));
+    if (capture != cudaStreamCaptureStatusNone) return AM_ERR_INVALID_ARGUMENT;
 
     int rc = refresh_pointers(h, params, grads, m, ex ? ex->params_bf16 : nullptr, stream);
     if (rc != AM_OK) return rc;

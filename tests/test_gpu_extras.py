@@ -114,6 +114,41 @@ def test_skip_flag_leaves_the_state_untouched():
     oa.close(); ob.close()
 
 
+@pytest.mark.filterwarnings("ignore:The CUDA Graph is empty")
+def test_a_capturing_stream_is_refused():
+    """A step carries t and the learning rate as kernel arguments and alternates
+    between two work counters, so a graph replay would repeat a stale step: the
+    call refuses a stream that is being captured, enqueues nothing, and the
+    handle steps normally afterwards."""
+    w = mixed_workload()
+    a = H.DeviceState(w, guarded=False)
+    b = H.DeviceState(w, guarded=False)
+    oa, ob = H.make_optimizer(w), H.make_optimizer(w)
+    a.draw_grads(1)
+    for x, y in zip(a.g, b.g):
+        y.copy_(x)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    torch.cuda.synchronize()
+    before = [x.clone() for x in b.p + b.m + [b.v]]
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        graph.capture_begin()
+        try:
+            with pytest.raises(B.AdamMiniError) as info:
+                ob.step(b.p, b.g, b.m, b.v, 1, stream=side.cuda_stream)
+        finally:
+            graph.capture_end()
+    assert info.value.status == -1                                # AM_ERR_INVALID_ARGUMENT
+    torch.cuda.synchronize()
+    assert all(torch.equal(x, y) for x, y in zip(before, b.p + b.m + [b.v]))
+    oa.step(a.p, a.g, a.m, a.v, 1)
+    ob.step(b.p, b.g, b.m, b.v, 1)
+    ob.sync_status()
+    assert _same(a, b)
+    oa.close(); ob.close()
+
+
 @pytest.mark.parametrize("statistic", [B.STAT_MAX, B.STAT_MIN, B.STAT_ONE_NORM, B.STAT_TWO_NORM],
                          ids=["max", "min", "one-norm", "two-norm"])
 @pytest.mark.parametrize("grad_dtype", [W.F32, W.BF16], ids=["f32", "bf16"])
