@@ -252,9 +252,11 @@ typedef enum {
     AM_OPT_STREAM_THREADS = 3, /* threads per consumer group of the streaming kernels, a multiple of 32
                                   from 64 to 512 (0 = default 256; anything else is rejected);
                                   groups x threads is capped at 512 */
-    AM_OPT_PROFILE        = 4, /* n > 0: record CUDA events around each kernel family of every step, keeping
+    AM_OPT_PROFILE        = 4, /* n > 0: record CUDA events around each kernel family of every step (one
+                                  at the start, one behind every family that launches something), keeping
                                   the latest n steps (n <= 4096); read them with adammini_get_profile.
-                                  Setting the option again restarts the record */
+                                  Setting the option again, or an option that changes the launch plan,
+                                  restarts the record */
     AM_OPT_STREAM_CHUNK   = 5, /* how the streaming kernel's CTAs share the work: 0 = automatic (CTAs take one
                                   work item at a time -- a stage of packed blocks, or one long block -- from
                                   a shared counter: this evens out bandwidth differences between SMs and

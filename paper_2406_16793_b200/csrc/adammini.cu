@@ -290,9 +290,19 @@ int build_plan(am_handle *h) {
         if (e != cudaSuccess) return cuda_fail(h, e);
     }
 
+    h->prof_steps = 0;       // recorded steps belong to the plan that launched them
     h->launches = (small_units_by_len[1] ? 1 : 0) + (small_units_by_len[2] ? 1 : 0) + (small_units_by_len[3] ? 1 : 0) + (tile_short_units ? 1 : 0) + (tile_units > tile_short_units ? 1 : 0) + (piece_units ? 3 : 0) + (wide_units ? 1 : 0) + sp.launches();
     h->planned = true;
     return AM_OK;
+}
+
+// Kernel families in the order a step launches them (and adammini_get_profile reports them):
+// short blocks, streaming launches, cluster launch, two-pass kernels.
+inline void active_families(const am_handle *h, bool active[4]) {
+    active[0] = h->small_units > 0 || h->tile_units > 0;
+    active[1] = h->stream.main.active() || h->stream.edge.active();
+    active[2] = h->stream.clus.active();
+    active[3] = h->piece_units > 0;
 }
 
 // Refresh the device tensor table if any data pointer changed.
@@ -553,7 +563,13 @@ int adammini_step_ex(am_handle *h, void *const *params, const void *const *grads
     h->stream.stall_after = static_cast<int>(std::min<int64_t>(h->opt[AM_OPT_TEST_STALL], 1 << 30));
     const bool prof = h->opt[AM_OPT_PROFILE] != 0;
     cudaEvent_t *pev = prof ? &h->prof_ev[(h->prof_steps % h->opt[AM_OPT_PROFILE]) * 5] : nullptr;
-    if (prof) AM_CUDA(h, cudaEventRecord(pev[0], stream));
+    // An event behind every family that launches something (none behind the others: on steps of a
+    // few hundred microseconds each event costs a percent).
+    bool fam[4] = {false, false, false, false};
+    if (prof) {
+        active_families(h, fam);
+        AM_CUDA(h, cudaEventRecord(pev[0], stream));
+    }
     if (h->small_units || h->tile_units) {
         SmallScalars ss;
         ss.beta1 = sc.beta1;
@@ -596,12 +612,12 @@ int adammini_step_ex(am_handle *h, void *const *params, const void *const *grads
         }
     }
     h->stream.bf16_copies = ex && ex->params_bf16;
-    if (prof) AM_CUDA(h, cudaEventRecord(pev[1], stream));
+    if (fam[0]) AM_CUDA(h, cudaEventRecord(pev[1], stream));
     AM_CUDA(h, h->stream.launch_main(h->d_tensors, v, sc, h->error_word, stream));
     AM_CUDA(h, h->stream.launch_edge(h->d_tensors, v, sc, h->error_word, stream));
-    if (prof) AM_CUDA(h, cudaEventRecord(pev[2], stream));
+    if (fam[1]) AM_CUDA(h, cudaEventRecord(pev[2], stream));
     AM_CUDA(h, h->stream.launch_cluster(h->d_tensors, v, sc, h->error_word, stream));
-    if (prof) AM_CUDA(h, cudaEventRecord(pev[3], stream));
+    if (fam[2]) AM_CUDA(h, cudaEventRecord(pev[3], stream));
     if (h->piece_units) {
         twopass_partial_kernel<<<static_cast<unsigned>(h->piece_units), kThreads, 0, stream>>>(
             h->d_tensors, h->d_piece_segs, h->n_piece_segs, h->d_partials, sc.gscale, sc.gscale_dev, sc.skip_flag, sc.statistic);
@@ -620,10 +636,8 @@ int adammini_step_ex(am_handle *h, void *const *params, const void *const *grads
             h->d_tensors, h->d_piece_segs, h->n_piece_segs, h->d_block_steps, sc);
         AM_CUDA(h, cudaGetLastError());
     }
-    if (prof) {
-        AM_CUDA(h, cudaEventRecord(pev[4], stream));
-        ++h->prof_steps;
-    }
+    if (fam[3]) AM_CUDA(h, cudaEventRecord(pev[4], stream));
+    if (prof) ++h->prof_steps;
     return AM_OK;
 }
 
@@ -632,13 +646,21 @@ int adammini_get_profile(am_handle *h, float *ms, int32_t *n_steps) {
     const int64_t ring = h->opt[AM_OPT_PROFILE];
     const int64_t n = std::min(h->prof_steps, ring);
     double sum[4] = {0.0, 0.0, 0.0, 0.0};
+    bool fam[4];
+    active_families(h, fam);
+    int last = 0;                       // the last event a step records
+    for (int k = 0; k < 4; ++k)
+        if (fam[k]) last = k + 1;
     for (int64_t s = 0; s < n; ++s) {
         cudaEvent_t *ev = &h->prof_ev[s * 5];
-        AM_CUDA(h, cudaEventSynchronize(ev[4]));
+        AM_CUDA(h, cudaEventSynchronize(ev[last]));
+        int before = 0;                 // the event recorded before family k's launches
         for (int k = 0; k < 4; ++k) {
+            if (!fam[k]) continue;      // (launches nothing: no time, no event)
             float x = 0.f;
-            AM_CUDA(h, cudaEventElapsedTime(&x, ev[k], ev[k + 1]));
+            AM_CUDA(h, cudaEventElapsedTime(&x, ev[before], ev[k + 1]));
             sum[k] += x;
+            before = k + 1;
         }
     }
     for (int k = 0; k < 4; ++k) ms[k] = static_cast<float>(sum[k] / static_cast<double>(n));
