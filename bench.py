@@ -101,6 +101,37 @@ def kernel_digest() -> str:
     return kernel_digests()["stream"]
 
 
+def ring_copy_ceiling(opt, dev, load_bytes: int, store_bytes: int, reps: int = 10):
+    """What the device's memory gives a kernel that reads load_bytes and writes store_bytes per
+    item and computes nothing: the library's copy through its ring of bulk loads and bulk stores
+    (adammini_probe_ring_copy), timed here with events over 4 GiB of items."""
+    import torch
+    n_items = (4 << 30) // 40960
+    try:
+        src = torch.ones(max(n_items * load_bytes, 16), dtype=torch.uint8, device=dev)
+        dst = torch.zeros(max(n_items * store_bytes, 16), dtype=torch.uint8, device=dev)
+    except torch.OutOfMemoryError:
+        return None
+    for _ in range(3):
+        opt.probe_ring_copy(src, dst, n_items, load_bytes, store_bytes)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        opt.probe_ring_copy(src, dst, n_items, load_bytes, store_bytes)
+    e1.record()
+    torch.cuda.synchronize(dev)
+    opt.sync_status()
+    ms = e0.elapsed_time(e1) / reps
+    del src, dst
+    return {"gbs": n_items * (load_bytes + store_bytes) / (ms * 1e-3) / 1e9, "ms_per_launch": ms,
+            "read_bytes_per_item": load_bytes, "written_bytes_per_item": store_bytes, "items": n_items}
+
+
+def update_mix(grad_f32: bool):
+    """Bytes a stage of 4096 elements reads (g, m, p) and writes (m, p), scaled to a 40960-byte read."""
+    return (40960, 27296) if grad_f32 else (40960, 32768)
+
+
 def measured_peak_gbs():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -436,6 +467,17 @@ def run_ours(args):
                 "whole_step_gbs": whole_gbs, "whole_step_frac": whole_gbs / peak,
                 "whole_step_frac_of_nominal": whole_gbs / NOMINAL_HBM_GBS}
 
+    if not args.no_ring_copy:
+        # the ceiling for the update's own mix of reads and writes (and, on request, for other mixes)
+        ring = ring_copy_ceiling(opt, dev, *update_mix(w.tensors[0].grad_dtype != W.BF16))
+        if ring:
+            ring["what"] = "bulk-load / bulk-store ring of this library with no arithmetic, the update's read:write mix"
+            roofline["ring_copy"] = ring
+            roofline["frac_of_ring_copy"] = achieved / ring["gbs"]
+        if args.ring_copy_modes:
+            roofline["ring_copy_modes"] = [ring_copy_ceiling(opt, dev, *(int(x) for x in mode.split(":")))
+                                           for mode in args.ring_copy_modes.split(",")]
+
     e2e = None
     if not args.no_e2e:
         if args.shard == "flat" and opt.query(B.Q_PART_TENSORS) > 0:
@@ -541,6 +583,8 @@ def main():
                     help="none: every rank steps its own copy of the table (weak scaling); blocks / flat: the ranks "
                          "share ONE table as whole-block shards / as flat shards with one exchange of part sums (strong scaling)")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-ring-copy", action="store_true", help="skip the copy-through-the-ring ceiling measurement")
+    ap.add_argument("--ring-copy-modes", default="", help="further read:write byte mixes per item to time through the ring, e.g. 40960:40960,40960:0,0:40960")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

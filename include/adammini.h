@@ -335,6 +335,23 @@ int32_t adammini_choose_cluster_size(const int32_t *resident_clusters, int64_t l
  * (may be NULL) receives the number of steps averaged. */
 int adammini_get_profile(am_handle *h, float *ms, int32_t *n_steps);
 
+/* Measurement aid (no step of Algorithm 1 runs here): a copy through the streaming kernel's
+ * ring of shared-memory stages with nothing in between -- bulk asynchronous loads, bulk
+ * asynchronous stores, one persistent CTA per SM, items handed out one at a time.  Item i reads
+ * load_bytes at src + i * load_bytes and writes store_bytes (the first store_bytes of what it
+ * read) at dst + i * store_bytes.  Timed by the caller with events on the stream, n_items *
+ * (load_bytes + store_bytes) / time is what this device's memory gives a kernel with that mix
+ * of reads and writes: the ceiling for the update's 10 bytes read and 8 written per parameter.
+ *   src, dst : DEVICE, 16-byte aligned, at least n_items * load_bytes / store_bytes long
+ *              (either may be NULL when its byte count is 0).
+ *   load_bytes, store_bytes : multiples of 16 from 0 to 40960, not both 0; when both are
+ *              set, store_bytes <= load_bytes.
+ * Asynchronous on cuda_stream (which must not be capturing); waits inside are bounded like a
+ * step's, and a wait that gives up is reported by adammini_sync_status.  Uses the handle's
+ * device only, none of its tensors. */
+int adammini_probe_ring_copy(am_handle *h, const void *src, void *dst, int64_t n_items, int32_t load_bytes,
+                             int32_t store_bytes, void *cuda_stream);
+
 /* The CUDA error code (cudaError_t as int) of the last AM_ERR_CUDA on this handle; with
  * h == NULL, of the calling thread's last adammini_create that failed with AM_ERR_CUDA. */
 int adammini_last_cuda_error(const am_handle *h);

@@ -72,6 +72,8 @@ _SIGNATURES = {
                                         ctypes.POINTER(ctypes.c_void_p), ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p,
                                         ctypes.POINTER(StepExtras)]),
     "adammini_part_sums": (ctypes.c_int, [ctypes.c_void_p, ctypes.POINTER(ctypes.c_void_p), ctypes.c_void_p, ctypes.c_void_p]),
+    "adammini_probe_ring_copy": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32,
+                                                ctypes.c_int32, ctypes.c_void_p]),
     "adammini_step_host": (ctypes.c_int, [ctypes.c_void_p, ctypes.POINTER(ctypes.c_void_p), ctypes.POINTER(ctypes.c_void_p),
                                           ctypes.POINTER(ctypes.c_void_p), ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64]),
     "adammini_step_tensor_noalloc": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
@@ -279,6 +281,15 @@ class AdamMini:
         tensors, in table order) into `out`, a device float64 tensor."""
         ga = _ptr_array(_data_ptrs(grads))
         _check(load().adammini_part_sums(self._h, ga, int(out.data_ptr()), stream or None), self._h)
+
+    def probe_ring_copy(self, src, dst, n_items: int, load_bytes: int, store_bytes: int, stream: int = 0) -> None:
+        """Measurement aid: a copy through the streaming kernel's ring with no arithmetic
+        (item i reads load_bytes at src + i * load_bytes and writes store_bytes at
+        dst + i * store_bytes).  src/dst: device tensors, raw addresses or None.  Asynchronous."""
+        sp = 0 if src is None else (int(src.data_ptr()) if hasattr(src, "data_ptr") else int(src))
+        dp = 0 if dst is None else (int(dst.data_ptr()) if hasattr(dst, "data_ptr") else int(dst))
+        _check(load().adammini_probe_ring_copy(self._h, sp or None, dp or None, int(n_items), int(load_bytes), int(store_bytes),
+                                               stream or None), self._h)
 
     def step_host(self, params: Sequence, grads: Sequence, m: Sequence, v, step: int,
                   staging_bytes: int = 0) -> None:

@@ -16,6 +16,7 @@
 #include "kernels_basic.cuh"
 #include "kernels_stream.cuh"
 #include "kernels_tile.cuh"
+#include "kernels_probe.cuh"
 #include "host_state.h"
 
 using namespace am;
@@ -244,6 +245,7 @@ int build_plan(am_handle *h) {
     const size_t o_wide_segs = take(sizeof(Seg) * std::max<size_t>(wide_segs.size(), 1));
     const size_t o_part_segs = take(sizeof(Seg) * std::max<size_t>(part_segs.size(), 1));
     const size_t o_part_list = take(sizeof(int32_t) * std::max<size_t>(part_tensors.size(), 1));
+    const size_t o_probe = take(128);
     h->arena_bytes = off;
     AM_CUDA(h, cudaMalloc(&h->arena, h->arena_bytes));
     char *base = static_cast<char *>(h->arena);
@@ -256,6 +258,7 @@ int build_plan(am_handle *h) {
     h->d_piece_segs = reinterpret_cast<Seg *>(base + o_piece);
     h->d_block_segs = reinterpret_cast<Seg *>(base + o_block);
     h->d_partials = reinterpret_cast<double *>(base + o_partials);
+    h->d_probe_counter = reinterpret_cast<unsigned long long *>(base + o_probe);
     h->d_block_steps = reinterpret_cast<float *>(base + o_steps);
     h->n_small_segs = static_cast<int>(small_segs.size());
     h->n_piece_segs = static_cast<int>(piece_segs.size());
@@ -379,6 +382,8 @@ int adammini_create(const am_partition *part, const am_hparams *hp, am_handle **
     if (e == cudaSuccess) *h->error_word = 0;
     if (e == cudaSuccess) e = stream_configure_kernels(h->caps.smem_optin);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(tile_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileSmemBytes);
+    if (e == cudaSuccess && h->caps.smem_optin >= kCtrlBytes + 2 * static_cast<size_t>(kProbeStageBytes))
+        e = cudaFuncSetAttribute(ring_copy_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(h->caps.smem_optin));
     if (e != cudaSuccess) {
         g_create_cuda_error = static_cast<int>(e);
         adammini_destroy(h);
@@ -665,6 +670,39 @@ int adammini_get_profile(am_handle *h, float *ms, int32_t *n_steps) {
     }
     for (int k = 0; k < 4; ++k) ms[k] = static_cast<float>(sum[k] / static_cast<double>(n));
     if (n_steps) *n_steps = static_cast<int32_t>(n);
+    return AM_OK;
+}
+
+int adammini_probe_ring_copy(am_handle *h, const void *src, void *dst, int64_t n_items, int32_t load_bytes,
+                             int32_t store_bytes, void *cuda_stream) {
+    if (!h || !h->planned || n_items < 0) return AM_ERR_INVALID_ARGUMENT;
+    if (load_bytes < 0 || store_bytes < 0 || load_bytes > kProbeStageBytes || store_bytes > kProbeStageBytes ||
+        load_bytes % 16 != 0 || store_bytes % 16 != 0 || (load_bytes == 0 && store_bytes == 0) ||
+        (load_bytes > 0 && store_bytes > load_bytes))
+        return AM_ERR_INVALID_ARGUMENT;
+    if ((load_bytes > 0 && !src) || (store_bytes > 0 && !dst)) return AM_ERR_INVALID_ARGUMENT;
+    if (!aligned16(src) || !aligned16(dst)) return AM_ERR_MISALIGNED;
+    if (n_items > (int64_t(1) << 40) / kProbeStageBytes) return AM_ERR_TOO_LARGE;
+    const int n_stages = h->caps.smem_optin > kCtrlBytes
+                             ? std::min<int>(kMaxStages, static_cast<int>((h->caps.smem_optin - kCtrlBytes) / kProbeStageBytes)) : 0;
+    if (n_stages < 2) return AM_ERR_TOO_LARGE;          // the device's shared memory does not hold a ring
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    int dev = -1;
+    AM_CUDA(h, cudaGetDevice(&dev));
+    if (dev != h->device) return AM_ERR_INVALID_ARGUMENT;
+    cudaStreamCaptureStatus capture = cudaStreamCaptureStatusNone;
+    AM_CUDA(h, cudaStreamIsCapturing(stream, &capture));
+    if (capture != cudaStreamCaptureStatusNone) return AM_ERR_INVALID_ARGUMENT;
+    if (n_items == 0) return AM_OK;
+    AM_CUDA(h, cudaMemsetAsync(h->d_probe_counter, 0, sizeof(unsigned long long), stream));
+    const unsigned long long limit_ns =
+        h->opt[AM_OPT_WAIT_LIMIT_US] ? static_cast<unsigned long long>(h->opt[AM_OPT_WAIT_LIMIT_US]) * 1000ull : kWaitTimeoutNs;
+    const unsigned grid = static_cast<unsigned>(std::min<int64_t>(h->caps.sm_count, n_items));
+    const size_t smem = kCtrlBytes + static_cast<size_t>(n_stages) * kProbeStageBytes;
+    ring_copy_kernel<<<grid, kProbeThreads, smem, stream>>>(static_cast<const unsigned char *>(src), static_cast<unsigned char *>(dst),
+                                                            n_items, load_bytes, store_bytes, n_stages, h->d_probe_counter,
+                                                            h->error_word, limit_ns);
+    AM_CUDA(h, cudaGetLastError());
     return AM_OK;
 }
 

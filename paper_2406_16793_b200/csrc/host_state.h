@@ -43,6 +43,7 @@ struct am_handle {
     int n_parts = 0;
     int64_t part_units = 0;
     double *d_partials = nullptr;
+    unsigned long long *d_probe_counter = nullptr;   // work counter of adammini_probe_ring_copy
     float *d_block_steps = nullptr;
     am::StreamPlan stream;
     am::DeviceCaps caps;                 // SMs, shared memory, L2, resident clusters per cluster size
