@@ -207,14 +207,12 @@ __device__ __forceinline__ uint32_t map_to_rank(uint32_t local_smem_addr, uint32
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_smem_addr), "r"(rank));
     return r;
 }
-__device__ __forceinline__ void st_cluster_f64(uint32_t cluster_addr, double x) {
-    asm volatile("st.shared::cluster.f64 [%0], %1;" ::"r"(cluster_addr), "d"(x) : "memory");
-}
-__device__ __forceinline__ void st_cluster_s64(uint32_t cluster_addr, long long x) {
-    asm volatile("st.shared::cluster.s64 [%0], %1;" ::"r"(cluster_addr), "l"(x) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+// Asynchronous 8-byte store into a peer CTA's shared memory that counts as 8 bytes of
+// complete_tx on that CTA's mbarrier: value and signal travel together, no fence on the sender's
+// side (a release there waits for every global store the thread still has in flight).
+__device__ __forceinline__ void st_async_cluster_b64(uint32_t cluster_addr, unsigned long long bits, uint32_t cluster_bar) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b64 [%0], %1, [%2];"
+                 ::"r"(cluster_addr), "l"(bits), "r"(cluster_bar) : "memory");
 }
 __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release;\n\tbarrier.cluster.wait.acquire;" ::: "memory");
@@ -440,7 +438,7 @@ stream_kernel(const __grid_constant__ StreamParams P) {
             mbar_init(&ctl->empty[s], n_cwarps);
         }
         for (int k = 0; k < kMaxGroups; ++k) mbar_init(&ctl->redbar[k], n_gwarps);
-        for (int k = 0; k < kExchangeSlots; ++k) mbar_init(&ctl->xbar[k], csize);
+        for (int k = 0; k < kExchangeSlots; ++k) mbar_init(&ctl->xbar[k], 1);      // armed by its own CTA, completed by the peers' bytes
         for (int k = 0; k < kItemSlots; ++k) mbar_init(&ctl->ibar[k], 1);
         ctl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -497,19 +495,31 @@ stream_kernel(const __grid_constant__ StreamParams P) {
             const bool dynamic = !CLUSTER && P.chunk > 0;
             const bool cdynamic = CLUSTER && P.chunk > 0;
             uint32_t published = 0, taken = 0;
-            auto cluster_publish = [&]() {
-                const long long idx = static_cast<long long>(atomicAdd(P.counter, static_cast<unsigned long long>(P.chunk)));
+            // The first CTA asks the counter for a block index when it takes one (two blocks ahead of
+            // use) and sends it on after the block's first APPLY stage, by which time the counter has
+            // answered; the sends are asynchronous stores that complete the peers' barriers themselves.
+            long long pub_idx = 0;
+            bool pub_pending = false;
+            auto publish_begin = [&]() {
+                pub_idx = static_cast<long long>(atomicAdd(P.counter, static_cast<unsigned long long>(P.chunk)));
+                pub_pending = true;
+            };
+            auto publish_finish = [&]() {
                 const uint32_t slot = published & (kItemSlots - 1);
                 ++published;
+                pub_pending = false;
                 const uint32_t item = smem_addr(&ctl->next_item[slot]), bar = smem_addr(&ctl->ibar[slot]);
-                for (uint32_t r = 0; r < csize; ++r) {
-                    st_cluster_s64(map_to_rank(item, r), idx);
-                    mbar_arrive_remote(map_to_rank(bar, r));
-                }
+                for (uint32_t r = 0; r < csize; ++r)
+                    st_async_cluster_b64(map_to_rank(item, r), static_cast<unsigned long long>(pub_idx), map_to_rank(bar, r));
+            };
+            auto cluster_publish = [&]() {
+                publish_begin();
+                publish_finish();
             };
             auto cluster_take = [&]() -> int64_t {
                 const uint32_t slot = taken & (kItemSlots - 1), par = (taken / kItemSlots) & 1u;
                 ++taken;
+                mbar_arrive_expect_tx(&ctl->ibar[slot], 8u);     // (the index may have landed already: the byte count is signed)
                 if (!wait_phase_one<true>(&ctl->ibar[slot], par, ctl, P.error_word, 5, P.wait_limit_ns)) { ok = false; return P.total_items; }
                 return *reinterpret_cast<volatile long long *>(&ctl->next_item[slot]);
             };
@@ -545,10 +555,11 @@ stream_kernel(const __grid_constant__ StreamParams P) {
             for (; ok; ++it) {
                 if (it >= hi) {
                     if (cdynamic) {
+                        if (pub_pending) publish_finish();
                         it = cluster_take();
                         if (!ok || it >= P.total_items) break;
                         hi = it + P.chunk < P.total_items ? it + P.chunk : P.total_items;
-                        if (crank == 0) cluster_publish();
+                        if (crank == 0) publish_begin();
                     } else {
                         if (!dynamic || next >= P.total_items) break;
                         it = next;
@@ -658,11 +669,16 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                         bulk_load(st + P.g_region_bytes, t.m + e0 + off, c * 4, &ctl->full[stage]);
                         bulk_load(st + P.g_region_bytes + kStageElems * 4, t.p + e0 + off, c * 4, &ctl->full[stage]);
                         advance();
+                        if (CLUSTER && pub_pending) publish_finish();
                     }
                 }
                 if (++item_group == P.n_groups) item_group = 0;
                 it += sg.slots - 1;             // the loop's increment then lands on the next item
             }
+            // One index more than the cluster takes is always on its way (the first CTA runs two ahead
+            // and the last take is the one that finds nothing left): wait for it, so that no store is
+            // still travelling towards this CTA's shared memory when it retires.
+            if (cdynamic && ok) (void)cluster_take();
             if (ok && acquire()) {
                 ctl->meta[stage].kind = STAGE_DONE;
                 mbar_arrive(&ctl->full[stage]);
@@ -809,12 +825,12 @@ stream_kernel(const __grid_constant__ StreamParams P) {
                             // a group barrier of every peer has ordered the earlier reads before it.
                             const uint32_t slot = long_seen & (kExchangeSlots - 1);
                             if (gtid == 0) {
+                                mbar_arrive_expect_tx(&ctl->xbar[slot], 8u * csize);    // this CTA's turn of the slot: one sum per CTA
                                 const uint32_t part = smem_addr(&ctl->xpart[slot][crank]);
                                 const uint32_t bar = smem_addr(&ctl->xbar[slot]);
-                                for (uint32_t r = 0; r < csize; ++r) {
-                                    st_cluster_f64(map_to_rank(part, r), tot);
-                                    mbar_arrive_remote(map_to_rank(bar, r));
-                                }
+                                for (uint32_t r = 0; r < csize; ++r)
+                                    st_async_cluster_b64(map_to_rank(part, r), static_cast<unsigned long long>(__double_as_longlong(tot)),
+                                                         map_to_rank(bar, r));
                             }
                             if (!wait_phase<true>(&ctl->xbar[slot], (long_seen / kExchangeSlots) & 1u, ctl, P.error_word, 4, P.wait_limit_ns)) break;
                             tot = ctl->xpart[slot][0];
