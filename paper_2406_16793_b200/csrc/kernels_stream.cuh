@@ -1174,12 +1174,14 @@ inline void stream_probe_clusters(DeviceCaps *caps, int block_threads) {
 // clusters resident than a larger one is passed over (it only idles SMs).
 //
 // kL2ShareForHeads is a measured boundary, not a derived one (B200, 126 MB of
-// L2 in two halves, resident = 148/74/45/33/26/22/15/15 for sizes 1..8): 45
-// clusters x 1 MB ran at 0.94 of the copy bandwidth against 0.97 for 33 x 1 MB,
-// and 22 x 2 MB at 0.95 against 0.93 for 33 x 2 MB; 74 x 0.31 MB and 45 x 0.5 MB
-// (1.01 and 0.99) beat the clusters of 4 that a fixed rule had given them (0.83
-// and 0.93).
-constexpr double kL2ShareForHeads = 0.353;
+// L2 in two halves, resident = 148/74/45/33/26/22/15/15 for sizes 1..8).  With
+// the exchange done by asynchronous stores a larger cluster costs nothing extra,
+// and fewer clusters that hold less in L2 beat many: on 1 MB blocks 22 clusters
+// of 6 and 15 of 8 run at 1.00-1.02 of the copy bandwidth against 0.98 for 33 of
+// 4 and 0.93 for 74 of 2 (in long runs under the power cap 6 is ahead of 8 by
+// 1 %, in short ones 8 by as much); 2 MB blocks reach 1.02 with 15 of 8 against
+// 0.98 with 22 of 6; blocks of 0.3 to 0.5 MB run at 1.02-1.05 with 3 to 6 CTAs.
+constexpr double kL2ShareForHeads = 0.18;
 
 inline int choose_cluster_size(const int *resident, int64_t l2_bytes, int64_t block_bytes) {
     int largest = 0;
@@ -1263,8 +1265,8 @@ inline void stream_finish_plan(const StreamPlanInput &in, StreamPlan *plan) {
     // Launch shape for head-sized blocks: the cluster size follows from the largest block, the L2
     // size and how many clusters of each size fit the device (choose_cluster_size), unless the
     // caller fixed it (then the largest size up to the caller's that can run).  Clusters take one
-    // block at a time from the shared counter; clusters of the largest size, which hold the
-    // biggest blocks, walk fixed ranges (measured).
+    // block at a time from the shared counter (fixed ranges, which keep every cluster in a region
+    // of its own, ran 7 % slower on Llama-2-7B's heads).
     int64_t max_block_bytes = 0;
     for (const auto &it : in.cluster_tensors)
         max_block_bytes = std::max(max_block_bytes, it.row.block_len * (it.row.grad_dtype == AM_BF16 ? 2 : 4));
@@ -1277,7 +1279,7 @@ inline void stream_finish_plan(const StreamPlanInput &in, StreamPlan *plan) {
     }
     if (cluster_size == 0) return;
     int chunk = in.cluster_chunk;
-    if (chunk == 0) chunk = (in.cluster_size == 0 && cluster_size == kMaxCluster) ? kStaticRanges : 1;
+    if (chunk == 0) chunk = 1;
     stream_build_launch(in.cluster_tensors, true, in.caps.resident[cluster_size], in.caps.smem_optin, &plan->clus);
     plan->clus.grid *= cluster_size;          // bounds are per cluster
     plan->clus.cluster = cluster_size;

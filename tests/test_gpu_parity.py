@@ -227,9 +227,9 @@ def test_launch_options_are_validated():
 
 def test_cluster_shape_follows_the_device():
     """The cluster size of a table is what the chooser gives for the properties the handle
-    read from this device; on a B200 (148 SMs, 126 MB of L2) that is 33 clusters of 4 for
-    bf16 heads of 128 x 4096 and 22 clusters of 6 for the same heads with float32 gradients."""
-    for gd, block_bytes, on_b200 in ((W.BF16, 1 << 20, (33, 4)), (W.F32, 2 << 20, (22, 6))):
+    read from this device; on a B200 (148 SMs, 126 MB of L2) that is 22 clusters of 6 for
+    bf16 heads of 128 x 4096 and 15 clusters of 8 for the same heads with float32 gradients."""
+    for gd, block_bytes, on_b200 in ((W.BF16, 1 << 20, (22, 6)), (W.F32, 2 << 20, (15, 8))):
         w = W.Workload("heads", 78, [W.TensorSpec("q", 8192, 4096, W.HEADS, n_heads=64, grad_dtype=gd)],
                        W.GradRecipe(-5.0, -1.0), steps=1)
         opt = H.make_optimizer(w)

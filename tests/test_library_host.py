@@ -180,20 +180,20 @@ def test_cluster_size_follows_l2_size_and_resident_clusters():
     MB = 1 << 20
     b200 = [0, 148, 74, 45, 33, 26, 22, 15, 15]        # resident clusters of 1..8 CTAs, 126 MB of L2
     choose = lambda caps, l2, block: binding.choose_cluster_size(caps, l2, block)
-    assert choose(b200, 126 * MB, 1 * MB) == 4          # bf16 heads of 128 x 4096
-    assert choose(b200, 126 * MB, 2 * MB) == 6          # the same heads with float32 gradients
+    assert choose(b200, 126 * MB, 1 * MB) == 6          # bf16 heads of 128 x 4096: 22 x 1 MB is within the share, 26 x 1 MB not
+    assert choose(b200, 126 * MB, 2 * MB) == 8          # the same heads with float32 gradients
     assert choose(b200, 126 * MB, 4 * MB) == 8          # nothing fits the share: the largest size
     assert choose(b200, 126 * MB, 3 * MB) == 8          # 7 keeps no more clusters than 8: passed over
-    assert choose(b200, 126 * MB, 320 * 1024) == 2
-    assert choose(b200, 126 * MB, 512 * 1024) == 2
+    assert choose(b200, 126 * MB, 320 * 1024) == 3      # 74 x 0.31 MB is just over the share, 45 x 0.31 MB within
+    assert choose(b200, 126 * MB, 512 * 1024) == 3      # 45 x 0.5 MB
     # monotone in the block size and in the L2 size
     sizes = [choose(b200, 126 * MB, k * 64 * 1024) for k in range(4, 65)]
     assert sizes == sorted(sizes)
-    by_l2 = [choose(b200, l2 * MB, 1 * MB) for l2 in (32, 64, 126, 256, 512)]
-    assert by_l2 == sorted(by_l2, reverse=True) and by_l2[0] == 8 and by_l2[-1] == 1
+    by_l2 = [choose(b200, l2 * MB, 1 * MB) for l2 in (32, 64, 126, 256, 512, 2048)]
+    assert by_l2 == sorted(by_l2, reverse=True) and by_l2 == [8, 8, 6, 3, 2, 1]
     # a device half the size with twice the cache per SM keeps smaller clusters
     small = [0, 74, 37, 24, 18, 14, 12, 10, 9]
-    assert choose(small, 126 * MB, 1 * MB) == 2
+    assert choose(small, 126 * MB, 1 * MB) == 4
     # clusters of some sizes cannot run; none at all -> 0 (the two-pass kernels take such blocks)
     assert choose([0, 148, 74, 0, 33, 0, 0, 0, 0], 126 * MB, 2 * MB) == 4
     assert choose([0] * 9, 126 * MB, 1 * MB) == 0
