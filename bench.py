@@ -42,14 +42,14 @@ NOMINAL_HBM_GBS = 8000.0      # HBM3e of a B200, nominal (quoted beside the meas
 # family from the ncu captures summarised under profiles/.  An entry counts only while the
 # sources its kernel is compiled from still have the digest they had at the capture.
 NCU_TRAFFIC = [
-    {"family": "stream_kernel<false>", "grad": "bf16", "block_lens": {4096, 11008}, "sources": "stream", "digest": "02a849eb5e16e77e",
-     "bytes_per_param": 17.905, "elements_query": lambda B: B.Q_ELEMENTS_STREAM,
+    {"family": "stream_kernel<false>", "grad": "bf16", "block_lens": {4096, 11008}, "sources": "stream", "digest": "bb2178e8f2c7d6a3",
+     "bytes_per_param": 17.909, "elements_query": lambda B: B.Q_ELEMENTS_STREAM,
      "capture": "profiles/stream_kernel_llama2_7b.md (2-layer case, scaled by parameters)"},
-    {"family": "stream_kernel<true>", "grad": "bf16", "block_lens": {524288}, "sources": "stream", "digest": "02a849eb5e16e77e",
-     "bytes_per_param": 17.434, "elements_query": lambda B: B.Q_ELEMENTS_CLUSTER,
+    {"family": "stream_kernel<true>", "grad": "bf16", "block_lens": {524288}, "sources": "stream", "digest": "bb2178e8f2c7d6a3",
+     "bytes_per_param": 17.201, "elements_query": lambda B: B.Q_ELEMENTS_CLUSTER,
      "capture": "profiles/stream_kernel_llama2_7b.md (2-layer case, scaled by parameters)"},
-    {"family": "stream_kernel<false>", "grad": "bf16", "block_lens": {10007}, "sources": "stream", "digest": "02a849eb5e16e77e",
-     "bytes_per_param": 17.592, "elements_query": lambda B: B.Q_ELEMENTS_STREAM,
+    {"family": "stream_kernel<false>", "grad": "bf16", "block_lens": {10007}, "sources": "stream", "digest": "bb2178e8f2c7d6a3",
+     "bytes_per_param": 17.595, "elements_query": lambda B: B.Q_ELEMENTS_STREAM,
      "capture": "profiles/stream_kernel_unaligned_rows_bf16_L10007.md (2^27 parameters, scaled)"},
     {"family": "short_block_kernels", "grad": "f32", "block_lens": {1}, "sources": "basic", "digest": "85b9245f3da5fdb0",
      "bytes_per_param": 27.587, "elements_query": lambda B: B.Q_ELEMENTS_SMALL,
@@ -60,11 +60,11 @@ NCU_TRAFFIC = [
     {"family": "twopass_kernels", "grad": "f32", "min_block_len": 1 << 22, "sources": "basic", "digest": "85b9245f3da5fdb0",
      "bytes_per_param": 23.650, "elements_query": lambda B: B.Q_ELEMENTS_TWOPASS,
      "capture": "profiles/small_and_twopass_kernels_flat_fp32.md (one block of 2^27 elements, scaled)"},
-    {"family": "short_block_kernels", "grad": "f32", "block_lens": {32}, "sources": "tile", "digest": "d087d6ca571e955b",
-     "bytes_per_param": 19.841, "elements_query": lambda B: B.Q_ELEMENTS_SMALL,
+    {"family": "short_block_kernels", "grad": "f32", "block_lens": {32}, "sources": "tile", "digest": "c7d52bfd623def44",
+     "bytes_per_param": 19.839, "elements_query": lambda B: B.Q_ELEMENTS_SMALL,
      "capture": "profiles/tile_kernel_flat_fp32_L32.md (2^27 parameters, scaled)"},
-    {"family": "short_block_kernels", "grad": "bf16", "block_lens": {1001}, "sources": "tile", "digest": "d087d6ca571e955b",
-     "bytes_per_param": 17.591, "elements_query": lambda B: B.Q_ELEMENTS_SMALL,
+    {"family": "short_block_kernels", "grad": "bf16", "block_lens": {1001}, "sources": "tile", "digest": "c7d52bfd623def44",
+     "bytes_per_param": 17.584, "elements_query": lambda B: B.Q_ELEMENTS_SMALL,
      "capture": "profiles/tile_kernel_rows_bf16_L1001.md (2^27 parameters, scaled)"},
 ]
 
