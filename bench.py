@@ -474,6 +474,7 @@ def run_ours(args):
             ring["what"] = "bulk-load / bulk-store ring of this library with no arithmetic, the update's read:write mix"
             roofline["ring_copy"] = ring
             roofline["frac_of_ring_copy"] = achieved / ring["gbs"]
+            roofline["whole_step_frac_of_ring_copy"] = whole_gbs / ring["gbs"]
         if args.ring_copy_modes:
             roofline["ring_copy_modes"] = [ring_copy_ceiling(opt, dev, *(int(x) for x in mode.split(":")))
                                            for mode in args.ring_copy_modes.split(",")]
